@@ -1,0 +1,333 @@
+#!/usr/bin/env python
+"""Benchmark of the integer LSTM forward pass.
+
+  python bench.py --gpus N --steps K --warmup W            # this library (CUDA, sm_100a)
+  python bench.py --impl reference --steps K --warmup W    # the CPU oracle, as a reported baseline
+
+A "step" is one pass of the whole hot path (input projection + recurrent steps of every layer)
+over one batch: the production-shaped configuration 5 (8 layers, layer norm + projection,
+input 640, cell 2048, projection 640, T = 300) at batch 256.  The metric is batch*timesteps/s.
+With N > 1 (torchrun) every rank runs the same workload on its own GPU: batch rows are
+independent, there is no collective on the data path, scaling is weak.  Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "quantized LSTM batch*timesteps/sec"
+UNIT = "batch*timesteps/s"
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [v.strip() for v in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def algorithmic_ops(layers, B, T):
+    """int8 multiply-accumulates counted as 2 ops, per pass: (projection GEMMs, recurrent + projection matmuls)."""
+    gemm = rec = 0
+    for q in layers:
+        G = 3 if (q.flags & 8) else 4
+        gemm += 2 * T * B * G * q.n_cell * q.n_input
+        rec += 2 * T * B * G * q.n_cell * q.n_output
+        if q.flags & 1:
+            rec += 2 * T * B * q.n_output * q.n_cell
+    return gemm, rec
+
+
+def oracle_sample(w_full_index, threads_hint, T_sample, rows_n):
+    """Times the CPU oracle, as it stands, on `rows_n` batch rows x T_sample steps of the workload."""
+    from oracle import qlstm_ref
+    from workloads import make_workload
+    rows = list(range(rows_n))
+    w = make_workload(w_full_index, rows=rows, T=T_sample)
+    h0, c0 = w.initial_state()
+    t0 = time.perf_counter()
+    qlstm_ref.run(w.layers, w.x, h0, c0)
+    dt = time.perf_counter() - t0
+    return rows_n * T_sample / dt, dt, qlstm_ref.num_threads()
+
+
+def run_reference(args):
+    """The reference arm: the oracle on the host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import qlstm_ref
+    cores = qlstm_ref.num_threads()
+    rows_n, T_s = max(1, min(args.batch, cores)), 8
+    for _ in range(args.warmup):
+        oracle_sample(args.config, cores, 2, rows_n)
+    times = []
+    for _ in range(args.steps):
+        v, dt, _ = oracle_sample(args.config, cores, T_s, rows_n)
+        times.append(dt)
+    total = sum(times)
+    value = rows_n * T_s * args.steps / total
+    sample = f"{rows_n} batch rows x {T_s} timesteps of config {args.config} per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": f"config5-ln-proj-8x2048 batch {args.batch} T {args.T}", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--config", type=int, default=5)
+    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--T", type=int, default=None)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-latency", action="store_true")
+    args = ap.parse_args()
+
+    from workloads import CONFIGS, make_workload
+    if args.T is None:
+        args.T = CONFIGS[args.config].T
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_2101_05453_b200 as qlstm
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = make_workload(args.config, batch=args.batch, T=args.T)
+    T, B = w.T, w.B
+    O = w.layers[-1].n_output
+    peaks = measured_peaks()
+
+    q = qlstm.QLSTM(w.layers, T, B, device=local)
+    stream = torch.cuda.current_stream().cuda_stream
+    h0, c0 = w.initial_state()
+    x = torch.from_numpy(w.x).to(dev)
+    h_init = torch.from_numpy(h0).to(dev)
+    c_init = torch.from_numpy(c0).to(dev)
+    h = h_init.clone()
+    c = c_init.clone()
+    y = torch.zeros((T, B, O), dtype=torch.int8, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)     # > L2 (126 MB)
+
+    def one_step(profile=False):
+        h.copy_(h_init)
+        c.copy_(c_init)
+        flush.zero_()                                                  # evict L2 between timed passes
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        q.run(x, T, B, h, c, y, stream=stream)
+        b.record()
+        return a, b
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    q.last_status()
+    torch.cuda.synchronize()
+    q.set_profiling(True)
+    q.get_profile(reset=True)
+
+    sampler = ClockSampler(local)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    events = [one_step() for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    q.last_status()
+    if dist is not None:
+        dist.barrier()
+    clocks = sampler.stop()
+    step_ms = [a.elapsed_time(b) for a, b in events]
+    total_ms = sum(step_ms)
+    prof = q.get_profile(reset=True)
+    q.set_profiling(False)
+    if dist is not None:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    value = world * B * T * args.steps / (total_ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry point: H2D of x, h, c and D2H of y, h, c inside the timed region
+    xh = torch.from_numpy(w.x).pin_memory()
+    hh = torch.from_numpy(h0.copy()).pin_memory()
+    ch = torch.from_numpy(c0.copy()).pin_memory()
+    yh = torch.empty((T, B, O), dtype=torch.int8).pin_memory()
+    h0t, c0t = torch.from_numpy(h0), torch.from_numpy(c0)
+    e2e_times = []
+    for i in range(2 + min(args.steps, 5)):
+        hh.copy_(h0t)
+        ch.copy_(c0t)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        q.run_host_raw(xh.data_ptr(), T, B, hh.data_ptr(), ch.data_ptr(), yh.data_ptr())
+        dt = time.perf_counter() - t0
+        if i >= 2:
+            e2e_times.append(dt)
+    e2e_t = sum(e2e_times) / len(e2e_times)
+    if dist is not None:
+        t = torch.tensor([e2e_t], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_t = float(t.item())
+    h2d = xh.numel() + hh.numel() + ch.numel() * 2
+    d2h = yh.numel() + hh.numel() + ch.numel() * 2
+    e2e = {"value": world * B * T / e2e_t, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    e2e_matches = bool(np.array_equal(yh.numpy(), y.cpu().numpy()))
+
+    # ---- rooflines.  Input projection: dense int8 contraction on the tensor cores.  Recurrent kernel: the slower of
+    # its int8 matmuls at tensor peak and its per-step bytes; both are far below the time it takes, which is
+    # integer-ALU and barrier time (reported as measured).
+    gemm_ops, rec_ops = algorithmic_ops(w.layers, B, T)
+    int8_peak = 2.0 * peaks["bf16_tflops_sustained"]          # TOP/s: bf16 measured x nominal int8:bf16 ratio of 2
+    n_l = len(w.layers)
+    proj_ms = prof["projection_ms"] / max(args.steps, 1)
+    rec_ms = prof["recurrent_ms"] / max(args.steps, 1)
+    proj_tops = gemm_ops / (proj_ms * 1e-3) / 1e12 if proj_ms > 0 else 0.0
+    rec_tops = rec_ops / (rec_ms * 1e-3) / 1e12 if rec_ms > 0 else 0.0
+    roof_proj = {"kernel": "input_projection", "bound": "tensor", "achieved": proj_tops, "peak": int8_peak,
+                 "unit": "TOP/s", "frac": proj_tops / int8_peak, "traffic": None,
+                 "peak_source": f"2 x bf16 sustained, {peaks['source']}", "ms_per_launch": proj_ms / n_l}
+    roof_rec = {"kernel": "recurrent", "bound": "tensor", "achieved": rec_tops, "peak": int8_peak, "unit": "TOP/s",
+                "frac": rec_tops / int8_peak, "traffic": None,
+                "peak_source": f"2 x bf16 sustained, {peaks['source']}", "ms_per_launch": rec_ms / n_l,
+                "us_per_layer_step": 1e3 * rec_ms / (n_l * T)}
+    dominant = roof_rec if rec_ms >= proj_ms else roof_proj
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": f"config{args.config}-{w.config.name} batch {B} T {T}",
+                       "layers": n_l, "n_input": w.layers[0].n_input, "n_cell": w.layers[0].n_cell,
+                       "n_output": O, "l2": "256 MiB buffer written between timed passes; X workspace "
+                       f"{T * B * w.layers[0].n_cell * 8 / 1e6:.0f} MB per layer exceeds L2"},
+            "clocks": clocks, "e2e": e2e, "e2e_matches_device_run": e2e_matches,
+            "gpu_launches": prof["projection_launches"] + prof["recurrent_launches"] + prof["other_launches"],
+            "roofline": dominant, "roofline_projection": roof_proj, "roofline_recurrent": roof_rec}
+
+    if rank == 0:
+        if not args.no_latency and args.config == 5:
+            # batch-1 per-step latency on the same model
+            w1 = make_workload(5, batch=1, T=T)
+            q1 = qlstm.QLSTM(w1.layers, T, 1, device=local)
+            x1 = torch.from_numpy(w1.x).to(dev)
+            hi, ci = w1.initial_state()
+            h1, c1 = torch.from_numpy(hi).to(dev), torch.from_numpy(ci).to(dev)
+            y1 = torch.zeros((T, 1, O), dtype=torch.int8, device=dev)
+            ts = []
+            for i in range(5):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                q1.run(x1, T, 1, h1, c1, y1, stream=stream)
+                b.record()
+                torch.cuda.synchronize()
+                if i >= 2:
+                    ts.append(a.elapsed_time(b))
+            q1.last_status()
+            ms = statistics.median(ts)
+            line["latency_batch1"] = {"us_per_timestep_whole_stack": 1e3 * ms / T,
+                                      "us_per_layer_step": 1e3 * ms / (T * n_l), "ms_per_pass": ms}
+            q1.close()
+        if not args.no_cpu_baseline:
+            from oracle import qlstm_ref
+            cores = qlstm_ref.num_threads()
+            rows_n = max(1, min(B, cores))
+            v0, dt0, _ = oracle_sample(args.config, cores, 2, rows_n)
+            T_s = int(max(2, min(T, 15.0 / (dt0 / 2))))
+            v, dt, cores = oracle_sample(args.config, cores, T_s, rows_n)
+            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": f"{rows_n} batch rows x {T_s} timesteps of the same workload, {dt:.1f} s"}
+        print(json.dumps(line))
+    q.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

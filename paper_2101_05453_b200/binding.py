@@ -1,0 +1,244 @@
+"""Thin ctypes binding of libqlstm.so: argument marshalling only.
+
+Every step of the integer LSTM runs inside the library's CUDA kernels; this module only
+converts numpy / torch arguments into the plain pointers and sizes of the C ABI
+(include/qlstm.h) and turns error codes into exceptions.  There is no fallback: if the
+library is missing or no sm_100 device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+from . import build as _build
+
+OK = 0
+ERR_ARG, ERR_DIM, ERR_RANGE, ERR_NOMEM, ERR_CUDA, ERR_LAUNCH, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6, -7
+IMPL_AUTO, IMPL_SIMPLE, IMPL_FAST = 0, 1, 2
+
+EXPORTS = ["qlstm_create", "qlstm_run", "qlstm_run_host", "qlstm_input_projection", "qlstm_last_status",
+           "qlstm_destroy", "qlstm_strerror", "qlstm_trace_bytes", "qlstm_set_impl", "qlstm_set_profiling",
+           "qlstm_get_profile", "qlstm_device_info"]
+
+
+class Scale(C.Structure):
+    _fields_ = [("multiplier", C.c_int32), ("shift", C.c_int32)]
+
+
+class Layer(C.Structure):
+    _fields_ = [
+        ("n_input", C.c_int32), ("n_cell", C.c_int32), ("n_output", C.c_int32),
+        ("flags", C.c_uint32), ("cell_int_bits", C.c_int32),
+        ("zp_x", C.c_int32), ("zp_m", C.c_int32), ("zp_h", C.c_int32),
+        ("W", C.c_void_p * 4), ("R", C.c_void_p * 4), ("P", C.c_void_p * 4),
+        ("b", C.c_void_p * 4), ("L", C.c_void_p * 4),
+        ("W_proj", C.c_void_p), ("b_proj", C.c_void_p),
+        ("eff_x", Scale * 4), ("eff_h", Scale * 4), ("eff_c", Scale * 4), ("eff_ln", Scale * 4),
+        ("eff_m", Scale), ("eff_proj", Scale),
+    ]
+
+
+class Profile(C.Structure):
+    _fields_ = [("projection_ms", C.c_double), ("projection_launches", C.c_int),
+                ("recurrent_ms", C.c_double), ("recurrent_launches", C.c_int),
+                ("other_ms", C.c_double), ("other_launches", C.c_int)]
+
+
+class QlstmError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__(f"{what}: {strerror(code)} ({code})")
+        self.code = code
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib():
+    """Loads libqlstm.so, building it first if the sources are newer.  Raises if that fails."""
+    global _lib
+    if _lib is None:
+        path = _build.build() if os.environ.get("QLSTM_NO_BUILD") != "1" else _build.LIB
+        L = C.CDLL(path)
+        L.qlstm_create.restype = C.c_int
+        L.qlstm_create.argtypes = [C.POINTER(Layer), C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_void_p)]
+        L.qlstm_run.restype = C.c_int
+        L.qlstm_run.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p,
+                                C.c_void_p, C.c_void_p]
+        L.qlstm_run_host.restype = C.c_int
+        L.qlstm_run_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.qlstm_input_projection.restype = C.c_int
+        L.qlstm_input_projection.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
+        L.qlstm_last_status.restype = C.c_int
+        L.qlstm_last_status.argtypes = [C.c_void_p]
+        L.qlstm_destroy.restype = None
+        L.qlstm_destroy.argtypes = [C.c_void_p]
+        L.qlstm_strerror.restype = C.c_char_p
+        L.qlstm_strerror.argtypes = [C.c_int]
+        L.qlstm_trace_bytes.restype = C.c_size_t
+        L.qlstm_trace_bytes.argtypes = [C.c_void_p, C.c_int, C.c_int]
+        L.qlstm_set_impl.restype = C.c_int
+        L.qlstm_set_impl.argtypes = [C.c_void_p, C.c_int, C.c_int]
+        L.qlstm_set_profiling.restype = C.c_int
+        L.qlstm_set_profiling.argtypes = [C.c_void_p, C.c_int]
+        L.qlstm_get_profile.restype = C.c_int
+        L.qlstm_get_profile.argtypes = [C.c_void_p, C.POINTER(Profile), C.c_int]
+        L.qlstm_device_info.restype = C.c_int
+        L.qlstm_device_info.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().qlstm_strerror(code).decode()
+
+
+def _check(code: int, what: str):
+    if code != OK:
+        raise QlstmError(code, what)
+
+
+def _ptr(a: Optional[np.ndarray], dtype, keep: list):
+    if a is None:
+        return None
+    a = np.ascontiguousarray(a, dtype)
+    keep.append(a)
+    return a.ctypes.data
+
+
+def pack_layers(layers: Sequence, keep: list):
+    """Marshals layer descriptions (objects with the fields of qlstm_layer_t) into a C array."""
+    arr = (Layer * len(layers))()
+    for d, q in zip(arr, layers):
+        d.n_input, d.n_cell, d.n_output = q.n_input, q.n_cell, q.n_output
+        d.flags, d.cell_int_bits = q.flags, q.cell_int_bits
+        d.zp_x, d.zp_m, d.zp_h = q.zp_x, q.zp_m, q.zp_h
+        for g in range(4):
+            d.W[g] = _ptr(q.W[g], np.int8, keep)
+            d.R[g] = _ptr(q.R[g], np.int8, keep)
+            d.P[g] = _ptr(q.P[g], np.int16, keep)
+            d.b[g] = _ptr(q.b[g], np.int32, keep)
+            d.L[g] = _ptr(q.L[g], np.int16, keep)
+            d.eff_x[g] = Scale(*map(int, q.eff_x[g]))
+            d.eff_h[g] = Scale(*map(int, q.eff_h[g]))
+            d.eff_c[g] = Scale(*map(int, q.eff_c[g]))
+            d.eff_ln[g] = Scale(*map(int, q.eff_ln[g]))
+        d.W_proj = _ptr(q.W_proj, np.int8, keep)
+        d.b_proj = _ptr(q.b_proj, np.int32, keep)
+        d.eff_m = Scale(*map(int, q.eff_m))
+        d.eff_proj = Scale(*map(int, q.eff_proj))
+    return arr
+
+
+def _dev_ptr(t) -> int:
+    """Device pointer of a torch CUDA tensor (must be contiguous) or a raw int address."""
+    if isinstance(t, int):
+        return t
+    if t is None:
+        return 0
+    assert t.is_cuda and t.is_contiguous()
+    return t.data_ptr()
+
+
+class QLSTM:
+    """Handle of one integer LSTM stack on one GPU (qlstm_create / qlstm_run / qlstm_destroy)."""
+
+    def __init__(self, layers: Sequence, max_T: int, max_B: int, device: int = 0):
+        keep: list = []
+        arr = pack_layers(layers, keep)
+        h = C.c_void_p()
+        _check(lib().qlstm_create(arr, len(layers), max_T, max_B, device, C.byref(h)), "qlstm_create")
+        self._h = h
+        self.device = device
+        self.dims = [(q.n_input, q.n_cell, q.n_output, 3 if (q.flags & 8) else 4) for q in layers]
+        self.max_T, self.max_B = max_T, max_B
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().qlstm_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    def run(self, x, T: int, B: int, h, c, y, trace=None, stream: int = 0, check: bool = False):
+        """qlstm_run on device tensors (torch CUDA tensors or raw addresses).  Asynchronous."""
+        _check(lib().qlstm_run(self._h, _dev_ptr(x), T, B, _dev_ptr(h), _dev_ptr(c), _dev_ptr(y), _dev_ptr(trace),
+                               stream), "qlstm_run")
+        if check:
+            self.last_status()
+
+    def run_host(self, x: np.ndarray, h: np.ndarray, c: np.ndarray):
+        """qlstm_run_host on numpy arrays: returns (y, h, c) as new arrays."""
+        x = np.ascontiguousarray(x, np.int8)
+        T, B, _ = x.shape
+        h = np.array(h, np.int8, copy=True)
+        c = np.array(c, np.int16, copy=True)
+        y = np.empty((T, B, self.dims[-1][2]), np.int8)
+        _check(lib().qlstm_run_host(self._h, x.ctypes.data, T, B, h.ctypes.data, c.ctypes.data, y.ctypes.data),
+               "qlstm_run_host")
+        return y, h, c
+
+    def run_host_raw(self, x_ptr: int, T: int, B: int, h_ptr: int, c_ptr: int, y_ptr: int):
+        _check(lib().qlstm_run_host(self._h, x_ptr, T, B, h_ptr, c_ptr, y_ptr), "qlstm_run_host")
+
+    def input_projection(self, layer: int, x, rows: int, out, stream: int = 0):
+        _check(lib().qlstm_input_projection(self._h, layer, _dev_ptr(x), rows, _dev_ptr(out), stream),
+               "qlstm_input_projection")
+
+    def last_status(self):
+        _check(lib().qlstm_last_status(self._h), "qlstm_last_status")
+
+    def trace_bytes(self, T: int, B: int) -> int:
+        return lib().qlstm_trace_bytes(self._h, T, B)
+
+    def set_impl(self, projection: int = IMPL_AUTO, recurrent: int = IMPL_AUTO):
+        _check(lib().qlstm_set_impl(self._h, projection, recurrent), "qlstm_set_impl")
+
+    def set_profiling(self, on: bool):
+        _check(lib().qlstm_set_profiling(self._h, int(on)), "qlstm_set_profiling")
+
+    def get_profile(self, reset: bool = True) -> dict:
+        p = Profile()
+        _check(lib().qlstm_get_profile(self._h, C.byref(p), int(reset)), "qlstm_get_profile")
+        return {k: getattr(p, k) for k, _ in Profile._fields_}
+
+    def device_info(self):
+        a, b = C.c_int(), C.c_int()
+        _check(lib().qlstm_device_info(self._h, C.byref(a), C.byref(b)), "qlstm_device_info")
+        return a.value, b.value
+
+
+def parse_trace(buf: np.ndarray, dims: Sequence, T: int, B: int):
+    """Splits a trace buffer (uint8 array, layout of include/qlstm.h) into per-layer dicts of arrays [T, ...]."""
+    out, off = [], 0
+    for (_, Cn, O, _) in dims:
+        bc, bo = B * Cn, B * O
+        fields = [("acc", np.int32, (4, B, Cn)), ("pacc", np.int32, (B, O)), ("xg", np.int16, (4, B, Cn)),
+                  ("pre", np.int16, (4, B, Cn)), ("ain", np.int16, (4, B, Cn)), ("gate", np.int16, (4, B, Cn)),
+                  ("c", np.int16, (B, Cn)), ("m", np.int8, (B, Cn)), ("h", np.int8, (B, O))]
+        rec = (16 * bc + 4 * bo + 32 * bc + 2 * bc + bc + bo + 15) & ~15
+        sect = buf[off:off + T * rec].reshape(T, rec)
+        d, o = {}, 0
+        for name, dt, shape in fields:
+            n = int(np.prod(shape)) * np.dtype(dt).itemsize
+            d[name] = np.ascontiguousarray(sect[:, o:o + n]).view(dt).reshape((T,) + shape)
+            o += n
+        out.append(d)
+        off += T * rec
+    return out

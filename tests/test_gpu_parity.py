@@ -1,0 +1,229 @@
+"""Parity of the CUDA path against the CPU oracle, bit for bit, through the C ABI (needs a B200)."""
+import copy
+
+import numpy as np
+import pytest
+
+from oracle import qlstm_ref as R
+from tests.gpu_util import assert_trace_equal, run_gpu
+from workloads import make_workload, random_layer_stack
+
+pytestmark = pytest.mark.gpu
+
+SIMPLE, FAST, AUTO = 1, 2, 0
+
+
+def oracle(w, trace=False, x=None, h0=None, c0=None):
+    hh, cc = w.initial_state()
+    if h0 is not None:
+        hh, cc = h0, c0
+    return R.run(w.layers, w.x if x is None else x, hh, cc, trace=trace)
+
+
+def check_equal(got, want, what):
+    for name, g, r in zip(("y", "h", "c"), got[:3], want[:3]):
+        if not np.array_equal(g, r):
+            bad = np.argwhere(g != r)
+            raise AssertionError(f"{what}: {name} differs at {len(bad)} places, first {bad[0]}: "
+                                 f"gpu {g[tuple(bad[0])]} oracle {r[tuple(bad[0])]}")
+
+
+# ------------------------------------------------------------------ every tensor at every step
+
+@pytest.mark.parametrize("index", [1, 2])
+def test_trace_parity_small_configs(index):
+    w = make_workload(index)
+    want = oracle(w, trace=True)
+    got = run_gpu(w, impl=(SIMPLE, SIMPLE), trace=True)
+    assert_trace_equal(got[3], want[3], f"config {index}")
+    check_equal(got, want, f"config {index}")
+
+
+VARIANTS = [
+    dict(),
+    dict(projection=True),
+    dict(peephole=True),
+    dict(layernorm=True),
+    dict(cifg=True),
+    dict(projection=True, peephole=True, layernorm=True),
+    dict(projection=True, layernorm=True),
+    dict(peephole=True, cifg=True),
+    dict(layernorm=True, cifg=True, projection=True),
+    dict(peephole=True, layernorm=True, cifg=True, projection=True),
+]
+
+
+@pytest.mark.parametrize("kw", VARIANTS, ids=lambda k: "+".join(sorted(k)) or "basic")
+def test_trace_parity_variants_ragged_shapes(kw):
+    # odd widths: nothing is a multiple of a tile, a warp or a vector
+    w = random_layer_stack(40 + len(kw), 2, 19, 37, 23, T=7, B=5, **kw)
+    want = oracle(w, trace=True)
+    got = run_gpu(w, impl=(SIMPLE, SIMPLE), trace=True)
+    assert_trace_equal(got[3], want[3], str(kw))
+    check_equal(got, want, str(kw))
+
+
+@pytest.mark.parametrize("kw", VARIANTS, ids=lambda k: "+".join(sorted(k)) or "basic")
+def test_auto_path_parity_variants(kw):
+    # shapes that span several tiles of the fast kernels plus a ragged tail
+    w = random_layer_stack(60 + len(kw), 2, 48, 176, 80, T=9, B=11, **kw)
+    want = oracle(w)
+    got = run_gpu(w, impl=(AUTO, AUTO))
+    check_equal(got, want, str(kw))
+
+
+def test_trace_parity_config3_slice():
+    w = make_workload(3, batch=3, T=6)
+    want = oracle(w, trace=True)
+    got = run_gpu(w, impl=(SIMPLE, SIMPLE), trace=True)
+    assert_trace_equal(got[3], want[3], "config 3")
+
+
+# ------------------------------------------------------------------ the five configurations
+
+@pytest.mark.parametrize("index,kw", [
+    (1, {}), (2, {}),
+    (3, dict(batch=32, T=24)),
+    (4, dict(batch=64, T=24)),
+    (5, dict(batch=1, T=24)),
+    (5, dict(batch=8, T=24)),
+    (5, dict(batch=64, T=6)),
+])
+def test_config_parity(index, kw):
+    w = make_workload(index, **kw)
+    want = oracle(w)
+    got = run_gpu(w)
+    check_equal(got, want, f"config {index} {kw}")
+
+
+@pytest.mark.parametrize("index,rows", [(3, [0, 13, 31]), (4, [0, 40, 63]), (5, [0, 100, 255])])
+def test_full_size_parity_on_sampled_rows(index, rows):
+    """Full T and full batch on the GPU in the launch configuration the benchmark times; the oracle
+    recomputes sampled batch rows one by one (rows never interact)."""
+    w = make_workload(index)
+    got = run_gpu(w)
+    ws = make_workload(index, rows=rows)
+    want = oracle(ws)
+    y = got[0][:, rows]
+    assert np.array_equal(y, want[0]), f"config {index}: y differs on sampled rows"
+    off_h = off_c = 0
+    offs_h = offs_c = 0
+    for q in w.layers:
+        hg = got[1][off_h:off_h + w.B * q.n_output].reshape(w.B, q.n_output)[rows]
+        cg = got[2][off_c:off_c + w.B * q.n_cell].reshape(w.B, q.n_cell)[rows]
+        hr = want[1][offs_h:offs_h + len(rows) * q.n_output].reshape(len(rows), q.n_output)
+        cr = want[2][offs_c:offs_c + len(rows) * q.n_cell].reshape(len(rows), q.n_cell)
+        assert np.array_equal(hg, hr) and np.array_equal(cg, cr)
+        off_h += w.B * q.n_output
+        off_c += w.B * q.n_cell
+        offs_h += len(rows) * q.n_output
+        offs_c += len(rows) * q.n_cell
+
+
+# ------------------------------------------------------------------ pieces and edge cases
+
+@pytest.mark.parametrize("impl", [SIMPLE, AUTO])
+def test_input_projection_matches_oracle(impl):
+    import torch
+    import paper_2101_05453_b200 as qlstm
+    w = random_layer_stack(77, 1, 96, 200, 200, T=5, B=70, peephole=True)
+    _, _, _, tr = oracle(w, trace=True)
+    q = w.layers[0]
+    rows = w.T * w.B
+    with qlstm.QLSTM(w.layers, w.T, w.B) as hnd:
+        hnd.set_impl(impl, impl)
+        xd = torch.from_numpy(w.x).cuda()
+        out = torch.zeros((rows, q.n_cell, 4), dtype=torch.int16, device="cuda")
+        hnd.input_projection(0, xd, rows, out, stream=torch.cuda.current_stream().cuda_stream)
+        hnd.last_status()
+        got = out.cpu().numpy().reshape(w.T, w.B, q.n_cell, 4).transpose(0, 3, 1, 2)
+    assert np.array_equal(got, tr[0]["xg"])
+
+
+def test_streaming_equivalence_and_state_carry():
+    import paper_2101_05453_b200 as qlstm
+    w = random_layer_stack(81, 2, 32, 64, 48, projection=True, layernorm=True, T=10, B=6)
+    want = oracle(w)
+    with qlstm.QLSTM(w.layers, w.T, w.B) as hnd:
+        y1, h1, c1, _ = run_gpu(w, handle=hnd, x=w.x[:3])
+        y2, h2, c2, _ = run_gpu(w, handle=hnd, x=w.x[3:], h0=h1, c0=c1)
+    check_equal((np.concatenate([y1, y2]), h2, c2), want, "streaming")
+
+
+def test_run_host_matches_device_run():
+    import paper_2101_05453_b200 as qlstm
+    w = make_workload(2)
+    want = oracle(w)
+    h0, c0 = w.initial_state()
+    with qlstm.QLSTM(w.layers, w.T, w.B) as hnd:
+        got = hnd.run_host(w.x, h0, c0)
+    check_equal(got, want, "run_host")
+
+
+def test_deterministic_run_to_run():
+    w = make_workload(3, batch=16, T=10)
+    a = run_gpu(w)
+    b = run_gpu(w)
+    check_equal(a, b, "determinism")
+
+
+def test_empty_inputs_and_limits():
+    import torch
+    import paper_2101_05453_b200 as qlstm
+    w = make_workload(1)
+    with qlstm.QLSTM(w.layers, 4, 2) as hnd:
+        x = torch.zeros((4, 2, 16), dtype=torch.int8, device="cuda")
+        h = torch.full((64,), 5, dtype=torch.int8, device="cuda")
+        c = torch.full((64,), 9, dtype=torch.int16, device="cuda")
+        y = torch.zeros((4, 2, 32), dtype=torch.int8, device="cuda")
+        hnd.run(x, 0, 2, h, c, y)          # T = 0: no-op
+        hnd.run(x, 4, 0, h, c, y)          # B = 0: no-op
+        hnd.last_status()
+        assert int(h[0]) == 5 and int(c[0]) == 9
+        with pytest.raises(qlstm.QlstmError) as e:
+            hnd.run(x, 5, 2, h, c, y)      # beyond max_T
+        assert e.value.code == qlstm.ERR_ARG
+        with pytest.raises(qlstm.QlstmError) as e:
+            hnd.run(None, 4, 2, h, c, y)
+        assert e.value.code == qlstm.ERR_ARG
+
+
+def test_folded_bias_out_of_range_is_rejected():
+    import paper_2101_05453_b200 as qlstm
+    w = make_workload(1)
+    bad = copy.deepcopy(w.layers[0])
+    bad.R[1][:] = 127
+    bad.zp_h = bad.zp_m = -128
+    bad.b[1][:] = 2 ** 31 - 1              # b - zp_h * sum(R) leaves int32
+    with pytest.raises(qlstm.QlstmError) as e:
+        qlstm.QLSTM([bad], 4, 1)
+    assert e.value.code == qlstm.ERR_RANGE
+
+
+def test_saturating_extremes_match_oracle():
+    """Hand-built layer whose every clamp engages: accumulator + bias, gate sum, cell update."""
+    from workloads.quantize import QLayer
+    C = 8
+    q = QLayer(4, C, C, 0, 0, -128, -128, -128)
+    for g in range(4):
+        q.W[g] = np.full((C, 4), 127, np.int8)
+        q.R[g] = np.full((C, C), 127 if g != 2 else -127, np.int8)
+        q.b[g] = np.full(C, 2 ** 31 - 1 - 127 * 128 * C, np.int32)
+        q.eff_x[g] = (1 << 30, 5)
+        q.eff_h[g] = ((1 << 31) - 1, -10)
+    q.eff_m = (1 << 30, -21)
+    x = np.full((3, 2, 4), 127, np.int8)
+
+    class W:
+        layers = [q]
+        B, T = 2, 3
+
+        def initial_state(self):
+            return np.full(2 * C, 127, np.int8), np.full(2 * C, 32767, np.int16)
+    w = W()
+    w.x = x
+    want = oracle(w, trace=True)
+    got = run_gpu(w, impl=(SIMPLE, SIMPLE), trace=True)
+    assert_trace_equal(got[3], want[3], "extremes")
+    got2 = run_gpu(w)
+    check_equal(got2, want, "extremes auto")
