@@ -29,6 +29,7 @@ struct FastScratch {
 };
 
 int fast_layer_init(FastLayer &f, const LayerParams &p, int max_T, int max_B, int sm_count);
+int fast_projection_init(FastLayer &f, const LayerParams &p);
 void fast_layer_destroy(FastLayer &f);
 int fast_scratch_init(FastScratch &s, int max_B, int maxC, int maxO, int maxN, int sm_count);
 void fast_scratch_destroy(FastScratch &s);
@@ -36,7 +37,7 @@ int fast_persistent_blocks(const FastScratch &s);
 
 bool fast_projection_supported(const FastLayer &f, const LayerParams &p);
 cudaError_t launch_projection_fast(const FastLayer &f, const LayerParams &p, const int8_t *x, int rows, int16_t *X,
-                                   int sm_count, cudaStream_t st);
+                                   int sm_count, int *status, cudaStream_t st);
 
 bool fast_recurrent_supported(const FastLayer &f, const LayerParams &p, int B);
 int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastScratch &s, const int16_t *X, int T, int B,

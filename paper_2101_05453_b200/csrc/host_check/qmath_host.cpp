@@ -12,6 +12,11 @@ void qmh_mbqm_many(const int32_t *x, int n, int32_t mult, int32_t shift, int32_t
 {
     for (int i = 0; i < n; ++i) out[i] = ql::mbqm(x[i], ql::Scale{mult, shift});
 }
+void qmh_fast_rescale_many(const int32_t *x, int n, int32_t mult, int32_t shift, int32_t *out)
+{
+    ql::FastScale f = ql::make_fast_scale(ql::Scale{mult, shift});
+    for (int i = 0; i < n; ++i) out[i] = ql::fast_rescale(x[i], f);
+}
 uint64_t qmh_isqrt(uint64_t v) { return ql::isqrt64(v); }
 void qmh_layernorm_row(const int16_t *q, int n, const int16_t *L, const int32_t *b, int32_t mult, int32_t shift, int16_t *out)
 {

@@ -237,7 +237,7 @@ int run_projection(qlstm *q, LayerHost &L, const int8_t *x, int rows, int16_t *X
     int impl = q->impl_proj;
     if (impl == 2 && !fast_ok) return QLSTM_ERR_DIM;
     bool use_fast = (impl == 2) || (impl == 0 && fast_ok);
-    cudaError_t e = use_fast ? launch_projection_fast(L.fast, L.p, x, rows, X, q->sm_count, st)
+    cudaError_t e = use_fast ? launch_projection_fast(L.fast, L.p, x, rows, X, q->sm_count, q->status, st)
                              : launch_projection_simple(L.p, x, rows, X, st);
     g.done(1);
     return e == cudaSuccess ? QLSTM_OK : QLSTM_ERR_CUDA;

@@ -47,6 +47,29 @@ QL_HD int32_t mbqm(int32_t x, Scale s)
     return p < 0 ? -(int32_t)q : (int32_t)q;
 }
 
+// The same rescale for shift <= 0 with its constants pre-computed, in 32-bit registers:
+//   round(round(|x| M / 2^31) / 2^R) = floor((2 |x| M + 2^31 + [R>0] 2^(31+R)) / 2^(32+R))
+// (nested floors collapse), i.e. the high word of one 32x32+64 multiply-add, shifted right by R.
+struct FastScale { uint32_t m2, add_hi; int32_t rshift; };
+
+QL_HD FastScale make_fast_scale(Scale s)
+{
+    int R = s.shift < 0 ? -s.shift : 0;
+    FastScale f;
+    f.m2 = (uint32_t)s.mult * 2u;
+    f.add_hi = R > 0 ? (1u << (R - 1)) : 0u;
+    f.rshift = R;
+    return f;
+}
+
+QL_HD int32_t fast_rescale(int32_t x, const FastScale &f)
+{
+    uint32_t a = x < 0 ? (uint32_t)0 - (uint32_t)x : (uint32_t)x;
+    uint64_t p = (uint64_t)a * f.m2 + (((uint64_t)f.add_hi << 32) | 0x80000000ull);
+    uint32_t q = (uint32_t)(p >> 32) >> f.rshift;
+    return x < 0 ? (int32_t)((uint32_t)0 - q) : (int32_t)q;
+}
+
 // n / d, d > 0, |n| + d/2 < 2^63
 QL_HD int64_t rdiv(int64_t n, int64_t d)
 {

@@ -48,6 +48,29 @@ def test_rescale_against_oracle(H):
         assert np.array_equal(out[::17], want), (M, s)
 
 
+def test_fast_rescale_against_oracle(H):
+    """The pre-computed single multiply-add form used in the kernels' epilogues (shift <= 0)."""
+    rng = np.random.default_rng(3)
+    xs = np.concatenate([rng.integers(-2 ** 31, 2 ** 31, 30000), np.arange(-70000, 70000, 3),
+                         [-2 ** 31, 2 ** 31 - 1, 0, 1, -1, 2 ** 30, -2 ** 30, 2 ** 30 + 1]]).astype(np.int32)
+    scales = [((1 << 31) - 1, 0), (1 << 30, 0), (1 << 30, -1), (1 << 30, -31), (0, 0), ((1 << 31) - 1, -31)] + \
+        [(int(rng.integers(1 << 30, 1 << 31)), int(s)) for s in range(-31, 1)]
+    out = np.empty_like(xs)
+    ref = np.empty_like(xs)
+    for M, s in scales:
+        H.qmh_fast_rescale_many(xs.ctypes.data_as(C.c_void_p), len(xs), M, s, out.ctypes.data_as(C.c_void_p))
+        H.qmh_mbqm_many(xs.ctypes.data_as(C.c_void_p), len(xs), M, s, ref.ctypes.data_as(C.c_void_p))
+        assert np.array_equal(out, ref), (M, s)            # all points: against the plain form (itself checked above)
+        want = np.array([R.mbqm(int(x), (M, s)) for x in xs[::23]], np.int32)
+        assert np.array_equal(out[::23], want), (M, s)     # a subsample directly against the oracle
+    # ties: x * M / 2^31 exactly half-way, then a second half-way in the right shift
+    for x in (1, -1, 3, -3, 5, -5, 7, -7, 1 << 20, -(1 << 20)):
+        for s in (0, -1, -2, -5):
+            xs1 = np.array([x], np.int32)
+            H.qmh_fast_rescale_many(xs1.ctypes.data_as(C.c_void_p), 1, 1 << 30, s, out.ctypes.data_as(C.c_void_p))
+            assert out[0] == R.mbqm(x, (1 << 30, s))
+
+
 def test_isqrt(H):
     import math
     rng = np.random.default_rng(1)
