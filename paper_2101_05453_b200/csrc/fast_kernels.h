@@ -8,38 +8,48 @@
 
 namespace ql {
 
+// Device scratch of the persistent recurrent kernel, shared by all layers of a handle.
+struct FastScratch {
+    int Bpad = 0;                // max batch rounded up to 128: rows of the MMA operands
+    int sm_count = 0;
+    int8_t *hbuf = nullptr;      // [2][Bpad][max O]  h^{t-1} / h^t, the recurrent matmul's A operand
+    int8_t *mbuf = nullptr;      // [Bpad][max C]     hidden state m, the projection's A operand
+    int32_t *pre = nullptr;      // [max B][max N]    gate sums between the matmul and elementwise phases
+                                 //                   (int16 values, or int32 X+H when a peephole follows)
+    unsigned *bar = nullptr;     // [0] grid-barrier counter, [1] abort word
+    size_t hbuf_bytes = 0, mbuf_bytes = 0;
+};
+
 struct FastLayer {
     bool proj_ok = false;        // tensor-core projection usable for this layer
-    bool rec_ok = false;         // persistent recurrent kernel usable for this layer
     CUtensorMap map_W;           // W [N][I] int8, K-major, 128B swizzle
-    int proj_block_n = 0;
-    // persistent kernel tiling
-    int cells_per_cta = 0, n_cta = 0, proj_cols_per_cta = 0;
-    CUtensorMap map_R, map_Wproj;
-    void *dev_aux = nullptr;
+    // persistent recurrent kernel plan
+    bool rec_ok = false;
+    int grid = 0;                // CTAs of the cooperative launch (one per SM)
+    int cpc = 0;                 // cells per CTA in the matmul phase
+    int n_cta_a = 0;             // CTAs that own cells
+    int nc_pad = 0;              // UMMA N of the recurrent matmul (multiple of 16)
+    int pn = 0, npn = 0;         // projection: N-slice width and number of N slices
+    int kb_h = 0, kb_c = 0;      // 128-byte k-blocks of the recurrent / projection matmul
+    int stages = 0;
+    size_t smem = 0;
+    CUtensorMap map_R, map_Wp, map_h, map_m;
 };
 
-struct FastScratch {
-    int persistent_blocks = 0;
-    int8_t *hbuf = nullptr;      // padded double-buffered h operand
-    int8_t *mbuf = nullptr;      // padded m operand
-    long long *ln_part = nullptr;
-    unsigned *bar = nullptr;     // grid barrier words
-    int max_B = 0;
-};
-
-int fast_layer_init(FastLayer &f, const LayerParams &p, int max_T, int max_B, int sm_count);
-int fast_projection_init(FastLayer &f, const LayerParams &p);
-void fast_layer_destroy(FastLayer &f);
 int fast_scratch_init(FastScratch &s, int max_B, int maxC, int maxO, int maxN, int sm_count);
 void fast_scratch_destroy(FastScratch &s);
-int fast_persistent_blocks(const FastScratch &s);
+
+int fast_layer_init(FastLayer &f, const LayerParams &p, const FastScratch &s, int max_T, int max_B);
+void fast_layer_destroy(FastLayer &f);
+int fast_projection_init(FastLayer &f, const LayerParams &p);
+int fast_recurrent_init(FastLayer &f, const LayerParams &p, const FastScratch &s, int max_B);
 
 bool fast_projection_supported(const FastLayer &f, const LayerParams &p);
 cudaError_t launch_projection_fast(const FastLayer &f, const LayerParams &p, const int8_t *x, int rows, int16_t *X,
                                    int sm_count, int *status, cudaStream_t st);
 
 bool fast_recurrent_supported(const FastLayer &f, const LayerParams &p, int B);
+// h / c are the caller's state (B rows); y is [T][B][O].  Returns a qlstm_error.
 int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastScratch &s, const int16_t *X, int T, int B,
                           int8_t *h, int16_t *c, int8_t *y, int *status, cudaStream_t st, int *launches);
 

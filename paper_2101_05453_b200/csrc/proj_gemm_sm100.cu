@@ -178,13 +178,14 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
                 bias[i * 32 + lane] = n < p.N ? p.bx[n] : 0;
             }
             __syncwarp();
-            if (!wait_or_abort(&ctl->tmem_full[buf], acc_phase, abort_flag)) break;
+            if (!__all_sync(0xffffffffu, wait_or_abort(&ctl->tmem_full[buf], acc_phase, abort_flag))) break;
             ptx::tc_fence_after();
             const int row = m0 + quarter * 32 + lane;
 #pragma unroll 1
             for (int ch = 0; ch < 4; ++ch) {
                 const int col = half * 128 + ch * 32, cw = ch * 32;
                 uint32_t r[32];
+                __syncwarp();             // the TMEM load is warp-collective: reconverge after the per-row branch
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + col), r);
                 ptx::tmem_ld_wait();
                 const int n_first = n0 + col;

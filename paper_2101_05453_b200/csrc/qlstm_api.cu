@@ -296,13 +296,11 @@ int qlstm_create(const qlstm_layer_t *layers, int n_layers, int max_T, int max_B
     if (ok && cudaStreamCreateWithFlags(&q->own_stream, cudaStreamNonBlocking) != cudaSuccess) { ok = false; rc = QLSTM_ERR_CUDA; }
     if (ok) {
         cudaMemset(q->status, 0, 4 * sizeof(int));
-        for (int l = 0; l < n_layers && ok; ++l) {
-            int frc = fast_layer_init(q->layers[l].fast, q->layers[l].p, max_T, max_B, q->sm_count);
-            if (frc != QLSTM_OK) { ok = false; rc = frc; }
-        }
-    }
-    if (ok) {
         int frc = fast_scratch_init(q->fscratch, max_B, (int)maxC, (int)maxO, (int)maxN, q->sm_count);
+        if (frc != QLSTM_OK) { ok = false; rc = frc; }
+    }
+    for (int l = 0; l < n_layers && ok; ++l) {
+        int frc = fast_layer_init(q->layers[l].fast, q->layers[l].p, q->fscratch, max_T, max_B);
         if (frc != QLSTM_OK) { ok = false; rc = frc; }
     }
     if (!ok) { qlstm_destroy(q); return rc; }
@@ -464,7 +462,7 @@ int qlstm_device_info(qlstm_t *q, int *sm_count, int *persistent_blocks)
 {
     if (!q) return QLSTM_ERR_ARG;
     if (sm_count) *sm_count = q->sm_count;
-    if (persistent_blocks) *persistent_blocks = fast_persistent_blocks(q->fscratch);
+    if (persistent_blocks) *persistent_blocks = q->layers.empty() ? 0 : (q->layers[0].fast.rec_ok ? q->layers[0].fast.grid : 0);
     return QLSTM_OK;
 }
 

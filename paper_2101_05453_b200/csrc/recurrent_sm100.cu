@@ -1,0 +1,712 @@
+// Persistent recurrent kernel: all T steps of one LSTM layer in one cooperative launch.
+//
+// Per step, three phases separated by grid-wide barriers (each phase partitions the work its own way):
+//
+//   A  recurrent matmul   partitioned by gate rows.  CTA i keeps the rows of R for cells
+//                         [i*cpc, (i+1)*cpc) resident in shared memory for the whole sequence, streams
+//                         h^{t-1} (int8 [B][O]) through a TMA ring and runs tcgen05.mma kind::i8 with the
+//                         batch as M and its gate rows as N.  Epilogue: + folded bias (saturating),
+//                         rescale to the gate format, + the input projection X_t -> gate sums to L2.
+//   B  elementwise        partitioned by (batch row, cell chunk).  Integer layer norm (statistics over the
+//                         whole row), integer sigmoid / tanh, CIFG coupling, peephole terms, int16 cell
+//                         update, hidden state requantised to int8.
+//   C  projection         partitioned by (batch tile, output slice); W_proj slice resident in shared memory,
+//                         m^t streamed through the same TMA ring; epilogue requantises to int8 h^t.
+//
+// Layer norm needs every cell of a row before any activation, and the projection needs every m before any
+// h, so these barriers are inherent to the method (Section 3.2.6, 3.2.8); only the data that crosses
+// CTAs (gate sums, m, h) goes through L2, the weights never move after the prologue.
+//
+// Every wait is bounded.  A wait that runs out sets the abort word; all CTAs observe it at the next
+// barrier, leave the time loop together, free their tensor memory and return; the host reports
+// QLSTM_ERR_TIMEOUT and the context stays usable.
+#include <cstring>
+
+#include "../../include/qlstm.h"
+#include "fast_kernels.h"
+#include "sm100_ptx.cuh"
+#include "tma_host.h"
+
+namespace ql {
+
+namespace {
+
+constexpr int RTHREADS = 320;                 // warp 0 TMA producer, warp 1 MMA issuer, warps 2..9 epilogue
+constexpr int A_STAGE_BYTES = 128 * 128;      // one k-block of the A operand: 128 rows x 128 bytes
+constexpr int MAX_STAGES = 6;
+constexpr unsigned long long SPIN_LIMIT_NS = 2000000000ull;   // 2 s per grid barrier
+
+struct RecParams {
+    int T, B, MT, Bpad;
+    int C, O, G, N;
+    uint32_t flags;
+    int m_bits, zp_m, zp_h;
+    int cpc, n_cta_a, nc_pad;
+    int pn, npn, n_ptiles;
+    int kb_h, kb_c, stages;
+    int chunks, chunk_cells, units_per_cta;
+    int fast_rescale_ok;          // every rescale of this layer has shift <= 0
+    const int16_t *X;             // [T][B][N]
+    int16_t *c;                   // [B][C]
+    int8_t *y;                    // [T][B][O]
+    int8_t *hbuf, *mbuf;
+    int32_t *pre;
+    unsigned *bar;
+    int *status;
+    const int32_t *bh, *bp, *bln;
+    const int16_t *P, *L;
+    Scale eff_h[4], eff_c[4], eff_ln[4], eff_m, eff_proj;
+    FastScale f_h[4], f_proj;
+    int gate_slot[4];             // canonical gate -> slot, -1 if absent
+};
+
+struct RecCtl {
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[3], w_full;
+    uint32_t tmem_base;
+    int abort_flag;
+    long long red_sum[10][4], red_sq[10][4];
+    long long stat_mean[4], stat_sigma[4];
+};
+
+__device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    for (uint32_t i = 0; i < (1u << 20); ++i) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ unsigned ld_acquire(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ unsigned long long globaltimer()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// Grid-wide barrier on a monotonic counter.  Global writes made before it by any thread of any CTA are
+// visible after it to every thread and to TMA loads (async proxy) of every CTA.
+__device__ __forceinline__ void grid_sync(const RecParams &p, unsigned &epoch, volatile int *abort_flag)
+{
+    fence_proxy_async_all();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        ++epoch;
+        const unsigned target = epoch * gridDim.x;
+        __threadfence();
+        atomicAdd(p.bar, 1u);
+        const unsigned long long t0 = globaltimer();
+        unsigned spins = 0;
+        while (ld_acquire(p.bar) < target) {
+            if (ld_acquire(p.bar + 1) != 0u) { *abort_flag = 1; break; }
+            if ((++spins & 1023u) == 0u && globaltimer() - t0 > SPIN_LIMIT_NS) {
+                atomicExch(p.bar + 1, 1u);
+                *abort_flag = 1;
+                break;
+            }
+        }
+        if (*abort_flag) atomicExch(p.bar + 1, 1u);
+        __threadfence();
+    }
+    __syncthreads();
+    fence_proxy_async_all();
+}
+
+__device__ __forceinline__ int32_t rescale_sel(int32_t x, const Scale &s, const FastScale &f, int fast_ok)
+{
+    return fast_ok ? fast_rescale(x, f) : mbqm(x, s);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Phase A epilogue for one thread = one batch row: NC gate sums of this CTA.
+//   out = sat16( X + sat16(rescale(sat32(acc + bh), eff_h)) )            (no peephole: final gate sum, int16)
+//   out = X + sat16(rescale(...))                                        (peephole: int32, finished in phase B)
+__device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, int b, int t, int n0, int n_cnt,
+                                            const int32_t *bh_s, bool row_valid)
+{
+    const bool peep = (p.flags & F_PEEPHOLE) != 0;
+    const int16_t *xrow = p.X + ((size_t)t * p.B + b) * p.N + n0;
+    for (int col = 0; col < p.nc_pad; col += 16) {
+        uint32_t r[16];
+        __syncwarp();                 // the TMEM load is warp-collective: reconverge after the per-row branch
+        ptx::tmem_ld_32x16(taddr + (uint32_t)col, r);
+        ptx::tmem_ld_wait();
+        if (!row_valid || col >= n_cnt) continue;
+        int32_t out[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int n = col + j;
+            if (n < n_cnt) {
+                const int gi = (p.G == 4) ? (j & 3) : (n % 3);
+                int32_t acc = sat32((int64_t)(int32_t)r[j] + bh_s[n]);
+                int32_t H = sat16(rescale_sel(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
+                int32_t X = xrow[n];
+                out[j] = peep ? X + H : sat16(X + H);
+            } else {
+                out[j] = 0;
+            }
+        }
+        if (peep) {
+            int32_t *dst = p.pre + (size_t)b * p.N + n0 + col;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (col + j < n_cnt) dst[j] = out[j];
+        } else {
+            int16_t *dst = (int16_t *)p.pre + (size_t)b * p.N + n0 + col;
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+                if (col + j < n_cnt) dst[j] = (int16_t)out[j];
+        }
+    }
+}
+
+// Phase C epilogue for one thread = one batch row: PN outputs of the projection tile.
+__device__ __forceinline__ void phase_c_row(const RecParams &p, uint32_t taddr, int b, int t, int p0, int8_t *h_next,
+                                            bool row_valid)
+{
+    for (int col = 0; col < p.pn; col += 16) {
+        uint32_t r[16];
+        __syncwarp();
+        ptx::tmem_ld_32x16(taddr + (uint32_t)col, r);
+        ptx::tmem_ld_wait();
+        if (!row_valid || p0 + col >= p.O) continue;
+        uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int o = p0 + col + j;
+            int32_t hq = 0;
+            if (o < p.O) {
+                int32_t acc = sat32((int64_t)(int32_t)r[j] + p.bp[o]);
+                hq = sat8(rescale_sel(acc, p.eff_proj, p.f_proj, p.fast_rescale_ok) + p.zp_h);
+            }
+            w[j >> 2] |= (uint32_t)(hq & 0xff) << (8 * (j & 3));
+        }
+        // O is a multiple of 16, so a 16-wide group is either fully inside or fully outside
+        uint4 v = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4 *>(h_next + (size_t)b * p.O + p0 + col) = v;
+        *reinterpret_cast<uint4 *>(p.y + ((size_t)t * p.B + b) * p.O + p0 + col) = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Phase B helpers
+
+struct GateStats { LnStats s[4]; };
+
+// Block-wide reduction of per-gate sum / sum of squares; result for gate slots in `mask` lands in ctl->stat_*.
+__device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, long long (&sum)[4], long long (&sq)[4], int G, int n)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int g = 0; g < G; ++g) {
+        long long a = sum[g], b = sq[g];
+        for (int o = 16; o > 0; o >>= 1) {
+            a += __shfl_down_sync(0xffffffffu, a, o);
+            b += __shfl_down_sync(0xffffffffu, b, o);
+        }
+        if (lane == 0) { ctl->red_sum[warp][g] = a; ctl->red_sq[warp][g] = b; }
+    }
+    __syncthreads();
+    if (threadIdx.x < G) {
+        long long a = 0, b = 0;
+        for (int w = 0; w < RTHREADS / 32; ++w) { a += ctl->red_sum[w][threadIdx.x]; b += ctl->red_sq[w][threadIdx.x]; }
+        LnStats st = ln_stats(a, b, n);
+        ctl->stat_mean[threadIdx.x] = st.mean;
+        ctl->stat_sigma[threadIdx.x] = st.sigma;
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ int32_t ln_gate(const RecParams &p, const RecCtl *ctl, int32_t pre, int n, int gi)
+{
+    LnStats st;
+    st.mean = ctl->stat_mean[gi];
+    st.sigma = ctl->stat_sigma[gi];
+    return ln_apply(pre, st, p.L[n], p.bln[n], p.eff_ln[gi]);
+}
+
+__device__ __forceinline__ void store_hidden(const RecParams &p, int b, int u, int t, int32_t m, int8_t *h_next)
+{
+    if (p.flags & F_PROJECTION) {
+        p.mbuf[(size_t)b * p.C + u] = (int8_t)m;
+    } else {
+        h_next[(size_t)b * p.O + u] = (int8_t)m;
+        p.y[((size_t)t * p.B + b) * p.O + u] = (int8_t)m;
+    }
+}
+
+// Elementwise phase for the units of this CTA.  `row_s` is a shared buffer of C*G int16 plus C int16.
+__device__ void phase_b(const RecParams &p, RecCtl *ctl, int t, int8_t *h_next, int16_t *row_s)
+{
+    const bool ln = (p.flags & F_LAYERNORM) != 0, peep = (p.flags & F_PEEPHOLE) != 0, cifg = (p.flags & F_CIFG) != 0;
+    const int G = p.G;
+    const int si = p.gate_slot[0], sf = p.gate_slot[1], sz = p.gate_slot[2], so = p.gate_slot[3];
+    const int total_units = p.B * p.chunks;
+    int u_begin = blockIdx.x * p.units_per_cta, u_end = u_begin + p.units_per_cta;
+    if (u_end > total_units) u_end = total_units;
+    int stats_row = -1;
+    const int16_t *pre16 = (const int16_t *)p.pre;
+
+    for (int unit = u_begin; unit < u_end; ++unit) {
+        const int b = unit / p.chunks, ch = unit % p.chunks;
+        const int k0 = ch * p.chunk_cells;
+        const int k1 = (k0 + p.chunk_cells < p.C) ? k0 + p.chunk_cells : p.C;
+        int16_t *c_row = p.c + (size_t)b * p.C;
+
+        if (ln && peep) {
+            // the unit is a whole row: gate sums need the peephole term before their statistics
+            int16_t *pre_s = row_s, *cnew_s = row_s + (size_t)p.C * G;
+            const int32_t *xh = p.pre + (size_t)b * p.N;
+            long long sum[4] = {0, 0, 0, 0}, sq[4] = {0, 0, 0, 0};
+            for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
+                const int32_t c_old = c_row[u];
+                for (int gi = 0; gi < G; ++gi) {
+                    if (gi == so) continue;
+                    const int n = u * G + gi;
+                    int32_t v = xh[n];
+                    if (gi != sz) v += sat16(mbqm((int32_t)p.P[n] * c_old, p.eff_c[gi]));
+                    v = sat16(v);
+                    pre_s[n] = (int16_t)v;
+                    sum[gi] += v;
+                    sq[gi] += (long long)v * v;
+                }
+            }
+            block_reduce_stats(ctl, sum, sq, G, p.C);
+            long long sum_o[4] = {0, 0, 0, 0}, sq_o[4] = {0, 0, 0, 0};
+            for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
+                const int nb = u * G;
+                int32_t f = sigmoid_q(ln_gate(p, ctl, pre_s[nb + sf], nb + sf, sf), 3);
+                int32_t z = tanh_q(ln_gate(p, ctl, pre_s[nb + sz], nb + sz, sz), 3);
+                int32_t i;
+                if (cifg) { i = 32768 - f; if (i > 32767) i = 32767; }
+                else i = sigmoid_q(ln_gate(p, ctl, pre_s[nb + si], nb + si, si), 3);
+                int32_t c_new = cell_update(i, z, f, c_row[u], p.m_bits);
+                c_row[u] = (int16_t)c_new;
+                cnew_s[u] = (int16_t)c_new;
+                int32_t v = sat16(xh[nb + so] + sat16(mbqm((int32_t)p.P[nb + so] * c_new, p.eff_c[so])));
+                pre_s[nb + so] = (int16_t)v;
+                sum_o[so] += v;
+                sq_o[so] += (long long)v * v;
+            }
+            __syncthreads();          // statistics of i, f, z are consumed; the slots are reused for o
+            block_reduce_stats(ctl, sum_o, sq_o, G, p.C);
+            for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
+                const int n = u * G + so;
+                int32_t o = sigmoid_q(ln_gate(p, ctl, pre_s[n], n, so), 3);
+                store_hidden(p, b, u, t, hidden_q(o, cnew_s[u], p.m_bits, p.eff_m, p.zp_m), h_next);
+            }
+            __syncthreads();
+            continue;
+        }
+
+        if (ln && b != stats_row) {
+            const int16_t *row = pre16 + (size_t)b * p.N;
+            long long sum[4] = {0, 0, 0, 0}, sq[4] = {0, 0, 0, 0};
+            for (int u = threadIdx.x; u < p.C; u += RTHREADS)
+                for (int gi = 0; gi < G; ++gi) {
+                    long long v = row[u * G + gi];
+                    sum[gi] += v;
+                    sq[gi] += v * v;
+                }
+            __syncthreads();          // previous unit may still read the statistics
+            block_reduce_stats(ctl, sum, sq, G, p.C);
+            stats_row = b;
+        }
+
+        for (int u = k0 + threadIdx.x; u < k1; u += RTHREADS) {
+            const int nb = u * G;
+            const int32_t c_old = c_row[u];
+            int32_t af, az, ai = 0, ao_part;
+            if (peep) {
+                const int32_t *xh = p.pre + (size_t)b * p.N + nb;
+                af = sat16(xh[sf] + sat16(mbqm((int32_t)p.P[nb + sf] * c_old, p.eff_c[sf])));
+                az = sat16(xh[sz]);
+                if (!cifg) ai = sat16(xh[si] + sat16(mbqm((int32_t)p.P[nb + si] * c_old, p.eff_c[si])));
+                ao_part = xh[so];
+            } else {
+                const int16_t *pr = pre16 + (size_t)b * p.N + nb;
+                af = pr[sf]; az = pr[sz];
+                if (!cifg) ai = pr[si];
+                ao_part = pr[so];
+                if (ln) {
+                    af = ln_gate(p, ctl, af, nb + sf, sf);
+                    az = ln_gate(p, ctl, az, nb + sz, sz);
+                    if (!cifg) ai = ln_gate(p, ctl, ai, nb + si, si);
+                    ao_part = ln_gate(p, ctl, ao_part, nb + so, so);
+                }
+            }
+            int32_t f = sigmoid_q(af, 3), z = tanh_q(az, 3), i;
+            if (cifg) { i = 32768 - f; if (i > 32767) i = 32767; }
+            else i = sigmoid_q(ai, 3);
+            int32_t c_new = cell_update(i, z, f, c_old, p.m_bits);
+            c_row[u] = (int16_t)c_new;
+            int32_t ao = ao_part;
+            if (peep) ao = sat16(ao_part + sat16(mbqm((int32_t)p.P[nb + so] * c_new, p.eff_c[so])));
+            int32_t o = sigmoid_q(ao, 3);
+            store_hidden(p, b, u, t, hidden_q(o, c_new, p.m_bits, p.eff_m, p.zp_m), h_next);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+
+__global__ void __launch_bounds__(RTHREADS, 1)
+k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_R,
+                  const __grid_constant__ CUtensorMap map_m, const __grid_constant__ CUtensorMap map_Wp, RecParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const bool proj = (p.flags & F_PROJECTION) != 0;
+    // layout: [ring stages][R slice][Wproj slice][row buffer][bias slice][control]
+    uint8_t *ring = smem;
+    uint8_t *R_s = ring + (size_t)p.stages * A_STAGE_BYTES;
+    uint8_t *Wp_s = R_s + (size_t)p.kb_h * p.nc_pad * 128;
+    uint8_t *after_w = Wp_s + (proj ? (size_t)p.kb_c * p.pn * 128 : 0);
+    int16_t *row_s = (int16_t *)after_w;
+    const size_t row_bytes = ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE)) ? ((size_t)p.C * p.G + p.C) * 2 : 0;
+    int32_t *bh_s = (int32_t *)(after_w + ((row_bytes + 15) & ~(size_t)15));
+    RecCtl *ctl = (RecCtl *)(bh_s + p.nc_pad);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int cta = blockIdx.x;
+    volatile int *abort_flag = &ctl->abort_flag;
+    const bool has_cells = cta < p.n_cta_a;
+    const bool has_ptile = proj && cta < p.n_ptiles;
+    const int n0 = cta * p.cpc * p.G;
+    int n_cnt = p.cpc * p.G;
+    if (n0 + n_cnt > p.N) n_cnt = p.N - n0;
+    const int tile_mi = has_ptile ? cta / p.npn : 0, tile_p0 = has_ptile ? (cta % p.npn) * p.pn : 0;
+    const uint32_t acc_cols_a = (uint32_t)(p.MT * p.nc_pad);
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < acc_cols_a + (uint32_t)(proj ? p.pn : 0)) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&ctl->full[s], 1); ptx::mbar_init(&ctl->empty[s], 1); }
+        for (int i = 0; i < 3; ++i) ptx::mbar_init(&ctl->acc_full[i], 1);
+        ptx::mbar_init(&ctl->w_full, 1);
+        ctl->abort_flag = 0;
+        ptx::fence_barrier_init();
+        ptx::prefetch_tensormap(&map_h);
+        ptx::prefetch_tensormap(&map_R);
+        if (proj) { ptx::prefetch_tensormap(&map_m); ptx::prefetch_tensormap(&map_Wp); }
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(&ctl->tmem_base, tmem_cols);
+        ptx::tmem_relinquish();
+    }
+    for (int i = threadIdx.x; i < p.nc_pad; i += RTHREADS) bh_s[i] = (has_cells && i < n_cnt) ? p.bh[n0 + i] : 0;
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    // resident weights: one TMA box per k-block
+    if (threadIdx.x == 0) {
+        uint32_t bytes = 0;
+        if (has_cells) bytes += (uint32_t)(p.kb_h * p.nc_pad * 128);
+        if (has_ptile) bytes += (uint32_t)(p.kb_c * p.pn * 128);
+        if (bytes) {
+            ptx::mbar_arrive_expect_tx(&ctl->w_full, bytes);
+            if (has_cells)
+                for (int kb = 0; kb < p.kb_h; ++kb)
+                    ptx::tma_load_2d(R_s + (size_t)kb * p.nc_pad * 128, &map_R, &ctl->w_full, kb * 128, n0);
+            if (has_ptile)
+                for (int kb = 0; kb < p.kb_c; ++kb)
+                    ptx::tma_load_2d(Wp_s + (size_t)kb * p.pn * 128, &map_Wp, &ctl->w_full, kb * 128, tile_p0);
+        } else {
+            ptx::mbar_arrive(&ctl->w_full);
+        }
+    }
+    if (warp == 1 && lane == 0) wait_or_abort(&ctl->w_full, 0, abort_flag);
+    __syncthreads();
+
+    unsigned epoch = 0;
+    int stage = 0; uint32_t ring_phase = 0;      // advanced identically by producer and MMA issuer
+    const uint32_t idesc_a = ptx::idesc_i8(128, p.nc_pad), idesc_c = ptx::idesc_i8(128, p.pn);
+
+    for (int t = 0; t < p.T; ++t) {
+        const int cur = t & 1;
+        int8_t *h_next = p.hbuf + (size_t)(cur ^ 1) * p.Bpad * p.O;
+        const uint32_t par = (uint32_t)t & 1u;
+
+        // ================= phase A: gate sums =================
+        if (has_cells) {
+            if (warp == 0) {
+                if (lane == 0) {
+                    for (int mi = 0; mi < p.MT && !*abort_flag; ++mi)
+                        for (int kb = 0; kb < p.kb_h; ++kb) {
+                            if (!wait_or_abort(&ctl->empty[stage], ring_phase ^ 1, abort_flag)) break;
+                            ptx::mbar_arrive_expect_tx(&ctl->full[stage], A_STAGE_BYTES);
+                            ptx::tma_load_2d(ring + (size_t)stage * A_STAGE_BYTES, &map_h, &ctl->full[stage], kb * 128,
+                                             cur * p.Bpad + mi * 128);
+                            if (++stage == p.stages) { stage = 0; ring_phase ^= 1; }
+                        }
+                }
+                __syncwarp();
+            } else if (warp == 1) {
+                if (lane == 0) {
+                    ptx::tc_fence_after();
+                    for (int mi = 0; mi < p.MT && !*abort_flag; ++mi) {
+                        bool ok = true;
+                        for (int kb = 0; kb < p.kb_h; ++kb) {
+                            if (!wait_or_abort(&ctl->full[stage], ring_phase, abort_flag)) { ok = false; break; }
+                            ptx::tc_fence_after();
+                            const uint64_t a_desc = ptx::smem_desc_k_sw128(ptx::smem_u32(ring + (size_t)stage * A_STAGE_BYTES));
+                            const uint64_t b_desc = ptx::smem_desc_k_sw128(ptx::smem_u32(R_s + (size_t)kb * p.nc_pad * 128));
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                ptx::mma_i8_ss(tmem_base + (uint32_t)(mi * p.nc_pad), a_desc + 2 * k, b_desc + 2 * k, idesc_a,
+                                               (kb | k) != 0);
+                            ptx::mma_commit(&ctl->empty[stage]);
+                            if (++stage == p.stages) { stage = 0; ring_phase ^= 1; }
+                        }
+                        if (!ok) break;
+                        ptx::mma_commit(&ctl->acc_full[mi]);
+                    }
+                }
+                __syncwarp();
+            } else {
+                const int e = warp - 2, quarter = warp & 3, mi = e >> 2;
+                if (mi < p.MT) {
+                    if (__all_sync(0xffffffffu, wait_or_abort(&ctl->acc_full[mi], par, abort_flag))) {
+                        ptx::tc_fence_after();
+                        const int b = mi * 128 + quarter * 32 + lane;
+                        phase_a_row(p, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * p.nc_pad), b, t, n0, n_cnt,
+                                    bh_s, b < p.B);
+                        ptx::tc_fence_before();
+                    }
+                }
+            }
+        }
+        grid_sync(p, epoch, abort_flag);
+        if (*abort_flag) break;
+
+        // ================= phase B: elementwise =================
+        phase_b(p, ctl, t, h_next, row_s);
+        grid_sync(p, epoch, abort_flag);
+        if (*abort_flag) break;
+
+        // ================= phase C: projection =================
+        if (proj) {
+            if (has_ptile) {
+                if (warp == 0) {
+                    if (lane == 0) {
+                        for (int kb = 0; kb < p.kb_c; ++kb) {
+                            if (!wait_or_abort(&ctl->empty[stage], ring_phase ^ 1, abort_flag)) break;
+                            ptx::mbar_arrive_expect_tx(&ctl->full[stage], A_STAGE_BYTES);
+                            ptx::tma_load_2d(ring + (size_t)stage * A_STAGE_BYTES, &map_m, &ctl->full[stage], kb * 128,
+                                             tile_mi * 128);
+                            if (++stage == p.stages) { stage = 0; ring_phase ^= 1; }
+                        }
+                    }
+                    __syncwarp();
+                } else if (warp == 1) {
+                    if (lane == 0) {
+                        ptx::tc_fence_after();
+                        bool ok = true;
+                        for (int kb = 0; kb < p.kb_c; ++kb) {
+                            if (!wait_or_abort(&ctl->full[stage], ring_phase, abort_flag)) { ok = false; break; }
+                            ptx::tc_fence_after();
+                            const uint64_t a_desc = ptx::smem_desc_k_sw128(ptx::smem_u32(ring + (size_t)stage * A_STAGE_BYTES));
+                            const uint64_t b_desc = ptx::smem_desc_k_sw128(ptx::smem_u32(Wp_s + (size_t)kb * p.pn * 128));
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                ptx::mma_i8_ss(tmem_base + acc_cols_a, a_desc + 2 * k, b_desc + 2 * k, idesc_c, (kb | k) != 0);
+                            ptx::mma_commit(&ctl->empty[stage]);
+                            if (++stage == p.stages) { stage = 0; ring_phase ^= 1; }
+                        }
+                        if (ok) ptx::mma_commit(&ctl->acc_full[2]);
+                    }
+                    __syncwarp();
+                } else if (warp - 2 < 4) {
+                    const int quarter = warp & 3;
+                    if (__all_sync(0xffffffffu, wait_or_abort(&ctl->acc_full[2], par, abort_flag))) {
+                        ptx::tc_fence_after();
+                        const int b = tile_mi * 128 + quarter * 32 + lane;
+                        phase_c_row(p, tmem_base + ((uint32_t)(quarter * 32) << 16) + acc_cols_a, b, t, tile_p0, h_next, b < p.B);
+                        ptx::tc_fence_before();
+                    }
+                }
+            }
+            grid_sync(p, epoch, abort_flag);
+            if (*abort_flag) break;
+        }
+    }
+
+    // ---------------- teardown ----------------
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 200; ++i) __nanosleep(500);      // let copies in flight land before the CTA retires
+        if (threadIdx.x == 0) atomicExch(p.status, 2);
+    }
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, tmem_cols);
+    }
+}
+
+size_t rec_smem_bytes(const LayerParams &p, int stages, int nc_pad, int pn, int kb_h, int kb_c)
+{
+    const bool proj = (p.flags & F_PROJECTION) != 0;
+    size_t row_bytes = ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE)) ? ((size_t)p.C * p.G + p.C) * 2 : 0;
+    row_bytes = (row_bytes + 15) & ~(size_t)15;
+    return 1024 + (size_t)stages * A_STAGE_BYTES + (size_t)kb_h * nc_pad * 128 + (proj ? (size_t)kb_c * pn * 128 : 0) +
+           row_bytes + (size_t)nc_pad * 4 + sizeof(RecCtl) + 64;
+}
+
+int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+}  // namespace
+
+int fast_scratch_init(FastScratch &s, int max_B, int maxC, int maxO, int maxN, int sm_count)
+{
+    s.Bpad = round_up(max_B, 128);
+    s.sm_count = sm_count;
+    s.hbuf_bytes = (size_t)2 * s.Bpad * maxO;
+    s.mbuf_bytes = (size_t)s.Bpad * maxC;
+    if (cudaMalloc(&s.hbuf, s.hbuf_bytes) != cudaSuccess) return QLSTM_ERR_NOMEM;
+    if (cudaMalloc(&s.mbuf, s.mbuf_bytes) != cudaSuccess) return QLSTM_ERR_NOMEM;
+    if (cudaMalloc(&s.pre, (size_t)max_B * maxN * sizeof(int32_t)) != cudaSuccess) return QLSTM_ERR_NOMEM;
+    if (cudaMalloc(&s.bar, 64) != cudaSuccess) return QLSTM_ERR_NOMEM;
+    cudaMemset(s.hbuf, 0, s.hbuf_bytes);
+    cudaMemset(s.mbuf, 0, s.mbuf_bytes);
+    cudaMemset(s.bar, 0, 64);
+    return QLSTM_OK;
+}
+
+void fast_scratch_destroy(FastScratch &s)
+{
+    cudaFree(s.hbuf); cudaFree(s.mbuf); cudaFree(s.pre); cudaFree(s.bar);
+    s = FastScratch();
+}
+
+int fast_recurrent_init(FastLayer &f, const LayerParams &p, const FastScratch &s, int max_B)
+{
+    f.rec_ok = false;
+    const bool proj = (p.flags & F_PROJECTION) != 0;
+    if (p.O % 16 != 0 || p.C % 16 != 0 || max_B > 256) return QLSTM_OK;
+    const int grid = s.sm_count;
+    // cells per CTA: the gate-row slice must start on a 16-byte boundary of an int16 row (cpc * G % 8 == 0)
+    const int step = (p.G == 4) ? 2 : 8;
+    int cpc = round_up((p.C + grid - 1) / grid, step);
+    if (cpc * p.G > 256) return QLSTM_OK;
+    f.cpc = cpc;
+    f.n_cta_a = (p.C + cpc - 1) / cpc;
+    f.nc_pad = round_up(cpc * p.G, 16);
+    f.kb_h = (p.O + 127) / 128;
+    f.kb_c = (p.C + 127) / 128;
+    f.grid = grid;
+    const int MT_max = (max_B + 127) / 128;
+    f.pn = 0; f.npn = 0;
+    if (proj) {
+        int pn = 16;
+        while (pn <= 256 && MT_max * ((p.O + pn - 1) / pn) > grid) pn *= 2;
+        if (pn > 256) return QLSTM_OK;
+        f.pn = pn;
+        f.npn = (p.O + pn - 1) / pn;
+    }
+    if (MT_max * f.nc_pad + f.pn > 512) return QLSTM_OK;
+    int dev = 0, max_smem = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    int stages = MAX_STAGES;
+    while (stages >= 2 && rec_smem_bytes(p, stages, f.nc_pad, f.pn, f.kb_h, f.kb_c) > (size_t)max_smem) --stages;
+    if (stages < 2) return QLSTM_OK;
+    f.stages = stages;
+    f.smem = rec_smem_bytes(p, stages, f.nc_pad, f.pn, f.kb_h, f.kb_c);
+    if (!make_tensor_map_i8(&f.map_R, p.R, (uint64_t)p.N, (uint64_t)p.O, (uint32_t)f.nc_pad, 128)) return QLSTM_OK;
+    if (!make_tensor_map_i8(&f.map_h, s.hbuf, (uint64_t)2 * s.Bpad, (uint64_t)p.O, 128, 128)) return QLSTM_OK;
+    if (proj) {
+        if (!make_tensor_map_i8(&f.map_Wp, p.Wproj, (uint64_t)p.O, (uint64_t)p.C, (uint32_t)f.pn, 128)) return QLSTM_OK;
+        if (!make_tensor_map_i8(&f.map_m, s.mbuf, (uint64_t)s.Bpad, (uint64_t)p.C, 128, 128)) return QLSTM_OK;
+    } else {
+        f.map_Wp = f.map_R;
+        f.map_m = f.map_h;
+    }
+    if (cudaFuncSetAttribute(k_recurrent_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
+        return QLSTM_OK;
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_recurrent_sm100, RTHREADS, f.smem) != cudaSuccess || per_sm < 1)
+        return QLSTM_OK;
+    f.rec_ok = true;
+    return QLSTM_OK;
+}
+
+int fast_layer_init(FastLayer &f, const LayerParams &p, const FastScratch &s, int max_T, int max_B)
+{
+    (void)max_T;
+    int rc = fast_projection_init(f, p);
+    if (rc != QLSTM_OK) return rc;
+    return fast_recurrent_init(f, p, s, max_B);
+}
+
+void fast_layer_destroy(FastLayer &) {}
+
+bool fast_recurrent_supported(const FastLayer &f, const LayerParams &, int B) { return f.rec_ok && B <= 256; }
+
+int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastScratch &s, const int16_t *X, int T, int B,
+                          int8_t *h, int16_t *c, int8_t *y, int *status, cudaStream_t st, int *launches)
+{
+    RecParams rp;
+    memset(&rp, 0, sizeof(rp));
+    rp.T = T; rp.B = B; rp.MT = (B + 127) / 128; rp.Bpad = s.Bpad;
+    rp.C = p.C; rp.O = p.O; rp.G = p.G; rp.N = p.N;
+    rp.flags = p.flags; rp.m_bits = p.m_bits; rp.zp_m = p.zp_m; rp.zp_h = p.zp_h;
+    rp.cpc = f.cpc; rp.n_cta_a = f.n_cta_a; rp.nc_pad = f.nc_pad;
+    rp.pn = f.pn; rp.npn = f.npn; rp.n_ptiles = rp.MT * f.npn;
+    rp.kb_h = f.kb_h; rp.kb_c = f.kb_c; rp.stages = f.stages;
+    // elementwise units: (row, chunk of cells).  Layer norm with peephole needs the whole row in one CTA.
+    const bool ln_peep = (p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE);
+    int best_chunks = 1;
+    if (!ln_peep) {
+        double best_eff = -1.0;
+        const int max_chunks = p.C / 16 > 0 ? p.C / 16 : 1;
+        for (int ch = 1; ch <= max_chunks && ch <= 256; ++ch) {
+            long units = (long)B * ch;
+            long per = (units + f.grid - 1) / f.grid;
+            double eff = (double)units / ((double)per * f.grid);
+            if (eff > best_eff + 0.02) { best_eff = eff; best_chunks = ch; }
+        }
+    }
+    rp.chunks = best_chunks;
+    rp.chunk_cells = (p.C + best_chunks - 1) / best_chunks;
+    rp.units_per_cta = (int)(((long)B * best_chunks + f.grid - 1) / f.grid);
+    rp.fast_rescale_ok = 1;
+    for (int g = 0; g < p.G; ++g) {
+        rp.eff_h[g] = p.eff_h[g]; rp.eff_c[g] = p.eff_c[g]; rp.eff_ln[g] = p.eff_ln[g];
+        rp.f_h[g] = make_fast_scale(p.eff_h[g]);
+        if (p.eff_h[g].shift > 0) rp.fast_rescale_ok = 0;
+    }
+    rp.eff_m = p.eff_m; rp.eff_proj = p.eff_proj;
+    rp.f_proj = make_fast_scale(p.eff_proj);
+    if (p.eff_proj.shift > 0) rp.fast_rescale_ok = 0;
+    for (int g = 0; g < 4; ++g) rp.gate_slot[g] = p.slot_of_gate[g];
+    rp.X = X; rp.c = c; rp.y = y;
+    rp.hbuf = s.hbuf; rp.mbuf = s.mbuf; rp.pre = s.pre; rp.bar = s.bar; rp.status = status;
+    rp.bh = p.bh; rp.bp = p.bp; rp.bln = p.bln; rp.P = p.P; rp.L = p.L;
+
+    // h^{-1} into operand buffer 0; barrier words cleared
+    if (cudaMemsetAsync(s.bar, 0, 64, st) != cudaSuccess) return QLSTM_ERR_CUDA;
+    if (cudaMemcpyAsync(s.hbuf, h, (size_t)B * p.O, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return QLSTM_ERR_CUDA;
+
+    void *args[] = {(void *)&f.map_h, (void *)&f.map_R, (void *)&f.map_m, (void *)&f.map_Wp, (void *)&rp};
+    cudaError_t e = cudaLaunchCooperativeKernel((const void *)k_recurrent_sm100, dim3(f.grid), dim3(RTHREADS), args, f.smem, st);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return e == cudaErrorCooperativeLaunchTooLarge ? QLSTM_ERR_LAUNCH : QLSTM_ERR_CUDA;
+    }
+    if (cudaMemcpyAsync(h, s.hbuf + (size_t)(T & 1) * s.Bpad * p.O, (size_t)B * p.O, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+        return QLSTM_ERR_CUDA;
+    if (launches) *launches = 1;
+    return QLSTM_OK;
+}
+
+}  // namespace ql

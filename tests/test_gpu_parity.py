@@ -72,6 +72,23 @@ def test_auto_path_parity_variants(kw):
     check_equal(got, want, str(kw))
 
 
+@pytest.mark.parametrize("kw", VARIANTS, ids=lambda k: "+".join(sorted(k)) or "basic")
+def test_fast_kernels_forced_parity_variants(kw):
+    """Tensor-core projection and persistent recurrent kernel forced on (an unsupported shape would raise)."""
+    w = random_layer_stack(90 + len(kw), 2, 64, 208, 96, T=8, B=37, **kw)
+    want = oracle(w)
+    got = run_gpu(w, impl=(FAST, FAST))
+    check_equal(got, want, str(kw))
+
+
+@pytest.mark.parametrize("B", [1, 2, 31, 128, 129, 200, 256])
+def test_fast_kernels_batch_sizes(B):
+    w = random_layer_stack(7, 1, 32, 64, 48, projection=True, layernorm=True, T=5, B=B)
+    want = oracle(w)
+    got = run_gpu(w, impl=(FAST, FAST))
+    check_equal(got, want, f"B={B}")
+
+
 def test_trace_parity_config3_slice():
     w = make_workload(3, batch=3, T=6)
     want = oracle(w, trace=True)
