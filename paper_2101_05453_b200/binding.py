@@ -44,7 +44,9 @@ class Layer(C.Structure):
 class Profile(C.Structure):
     _fields_ = [("projection_ms", C.c_double), ("projection_launches", C.c_int),
                 ("recurrent_ms", C.c_double), ("recurrent_launches", C.c_int),
-                ("other_ms", C.c_double), ("other_launches", C.c_int)]
+                ("other_ms", C.c_double), ("other_launches", C.c_int),
+                ("phase_a_ms", C.c_double), ("wait_a_ms", C.c_double), ("phase_b_ms", C.c_double),
+                ("wait_b_ms", C.c_double), ("phase_c_ms", C.c_double), ("wait_c_ms", C.c_double)]
 
 
 class QlstmError(RuntimeError):

@@ -38,6 +38,7 @@ struct qlstm {
     SimpleScratch scratch = {};
     FastScratch fscratch = {};
     int *status = nullptr;          // device status word of the persistent kernel
+    unsigned long long *phase_ns = nullptr;   // device phase timers of the persistent kernel (profiling)
     // staging for qlstm_run_host
     int8_t *st_x = nullptr, *st_y = nullptr, *st_h = nullptr;
     int16_t *st_c = nullptr;
@@ -287,7 +288,7 @@ int qlstm_create(const qlstm_layer_t *layers, int n_layers, int max_T, int max_B
     if (ok) {
         ok = dmalloc(&q->X, rows * maxN) && dmalloc(&q->scratch.pre, (size_t)max_B * maxN) &&
              dmalloc(&q->scratch.po, (size_t)max_B * maxC) && dmalloc(&q->scratch.stats, (size_t)max_B * maxG * 2) &&
-             dmalloc(&q->scratch.m, (size_t)max_B * maxC) && dmalloc(&q->status, 4) &&
+             dmalloc(&q->scratch.m, (size_t)max_B * maxC) && dmalloc(&q->status, 4) && dmalloc(&q->phase_ns, 8) &&
              dmalloc(&q->st_x, rows * q->layers[0].p.I) && dmalloc(&q->st_y, rows * q->layers.back().p.O) &&
              dmalloc(&q->st_h, (size_t)max_B * sumO) && dmalloc(&q->st_c, (size_t)max_B * sumC);
         if (ok && n_layers > 1) ok = dmalloc(&q->seq[0], rows * maxO) && dmalloc(&q->seq[1], rows * maxO);
@@ -296,6 +297,7 @@ int qlstm_create(const qlstm_layer_t *layers, int n_layers, int max_T, int max_B
     if (ok && cudaStreamCreateWithFlags(&q->own_stream, cudaStreamNonBlocking) != cudaSuccess) { ok = false; rc = QLSTM_ERR_CUDA; }
     if (ok) {
         cudaMemset(q->status, 0, 4 * sizeof(int));
+        cudaMemset(q->phase_ns, 0, 8 * sizeof(unsigned long long));
         int frc = fast_scratch_init(q->fscratch, max_B, (int)maxC, (int)maxO, (int)maxN, q->sm_count);
         if (frc != QLSTM_OK) { ok = false; rc = frc; }
     }
@@ -321,6 +323,7 @@ void qlstm_destroy(qlstm_t *q)
     cudaFree(q->X); cudaFree(q->seq[0]); cudaFree(q->seq[1]);
     cudaFree(q->scratch.pre); cudaFree(q->scratch.po); cudaFree(q->scratch.stats); cudaFree(q->scratch.m);
     cudaFree(q->status);
+    cudaFree(q->phase_ns);
     cudaFree(q->st_x); cudaFree(q->st_y); cudaFree(q->st_h); cudaFree(q->st_c);
     for (auto &sp : q->spans) { cudaEventDestroy(sp.a); cudaEventDestroy(sp.b); }
     for (auto e : q->event_pool) cudaEventDestroy(e);
@@ -370,7 +373,7 @@ int qlstm_run(qlstm_t *q, const int8_t *x_dev, int T, int B, int8_t *h_dev, int1
             cudaError_t e;
             if (use_fast) {
                 int frc = launch_recurrent_fast(L.fast, p, q->fscratch, q->X, T, B, h_dev + h_off, c_dev + c_off, outp,
-                                                q->status, st, &launches);
+                                                q->status, q->profiling ? q->phase_ns : nullptr, st, &launches);
                 if (frc != QLSTM_OK) return frc;
                 e = cudaSuccess;
             } else {
@@ -453,8 +456,16 @@ int qlstm_get_profile(qlstm_t *q, qlstm_profile_t *out, int reset)
     if (!q || !out) return QLSTM_ERR_ARG;
     if (cudaSetDevice(q->device) != cudaSuccess) return QLSTM_ERR_CUDA;
     collect_spans(q);
+    unsigned long long ns[8] = {0};
+    if (cudaMemcpy(ns, q->phase_ns, sizeof(ns), cudaMemcpyDeviceToHost) != cudaSuccess) return QLSTM_ERR_CUDA;
     *out = q->prof;
-    if (reset) q->prof = qlstm_profile_t{};
+    out->phase_a_ms = ns[0] * 1e-6; out->wait_a_ms = ns[1] * 1e-6;
+    out->phase_b_ms = ns[2] * 1e-6; out->wait_b_ms = ns[3] * 1e-6;
+    out->phase_c_ms = ns[4] * 1e-6; out->wait_c_ms = ns[5] * 1e-6;
+    if (reset) {
+        q->prof = qlstm_profile_t{};
+        cudaMemset(q->phase_ns, 0, sizeof(ns));
+    }
     return QLSTM_OK;
 }
 

@@ -31,7 +31,9 @@ namespace ql {
 
 namespace {
 
-constexpr int RTHREADS = 320;                 // warp 0 TMA producer, warp 1 MMA issuer, warps 2..9 epilogue
+constexpr int RTHREADS = 640;                 // warp 0 TMA producer, warp 1 MMA issuer, warps 2..9 matmul epilogues;
+                                              // all 20 warps share the elementwise phase
+constexpr int MAX_LN_ROWS = 4;                // rows whose layer-norm statistics are held at once
 constexpr int A_STAGE_BYTES = 128 * 128;      // one k-block of the A operand: 128 rows x 128 bytes
 constexpr int MAX_STAGES = 6;
 constexpr unsigned long long SPIN_LIMIT_NS = 2000000000ull;   // 2 s per grid barrier
@@ -44,7 +46,7 @@ struct RecParams {
     int cpc, n_cta_a, nc_pad;
     int pn, npn, n_ptiles;
     int kb_h, kb_c, stages;
-    int chunks, chunk_cells, units_per_cta;
+    int items_per_cta;            // cells of the B x C grid per CTA in the elementwise phase
     int fast_rescale_ok;          // every rescale of this layer has shift <= 0
     const int16_t *X;             // [T][B][N]
     int16_t *c;                   // [B][C]
@@ -56,16 +58,17 @@ struct RecParams {
     const int32_t *bh, *bp, *bln;
     const int16_t *P, *L;
     Scale eff_h[4], eff_c[4], eff_ln[4], eff_m, eff_proj;
-    FastScale f_h[4], f_proj;
+    FastScale f_h[4], f_c[4], f_ln[4], f_m, f_proj;
     int gate_slot[4];             // canonical gate -> slot, -1 if absent
+    unsigned long long *phase_ns; // null, or 6 accumulators: work and barrier wait of phases A, B, C (CTA 0)
 };
 
 struct RecCtl {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[3], w_full;
     uint32_t tmem_base;
     int abort_flag;
-    long long red_sum[10][4], red_sq[10][4];
-    long long stat_mean[4], stat_sigma[4];
+    long long red_sum[RTHREADS / 32][4], red_sq[RTHREADS / 32][4];
+    LnRow ln_rows[MAX_LN_ROWS][4];
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
@@ -124,46 +127,61 @@ __device__ __forceinline__ int32_t rescale_sel(int32_t x, const Scale &s, const 
 {
     return fast_ok ? fast_rescale(x, f) : mbqm(x, s);
 }
+__device__ __forceinline__ int32_t rescale_any(int32_t x, const Scale &s, const FastScale &f)
+{
+    return s.shift <= 0 ? fast_rescale(x, f) : mbqm(x, s);
+}
 
 // ------------------------------------------------------------------------------------------------
-// Phase A epilogue for one thread = one batch row: NC gate sums of this CTA.
+__device__ __forceinline__ int32_t add_sat(int32_t a, int32_t b)
+{
+    int32_t d;
+    asm("add.sat.s32 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ int32_t lo16(uint32_t w) { return (int32_t)(w << 16) >> 16; }
+__device__ __forceinline__ int32_t hi16(uint32_t w) { return (int32_t)w >> 16; }
+__device__ __forceinline__ uint32_t pack16(int32_t lo, int32_t hi) { return ((uint32_t)lo & 0xffffu) | ((uint32_t)hi << 16); }
+
+// Phase A epilogue for one thread = one batch row: the gate sums of this CTA's cells, 8 columns at a time.
 //   out = sat16( X + sat16(rescale(sat32(acc + bh), eff_h)) )            (no peephole: final gate sum, int16)
 //   out = X + sat16(rescale(...))                                        (peephole: int32, finished in phase B)
+template <int G>
 __device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, int b, int t, int n0, int n_cnt,
                                             const int32_t *bh_s, bool row_valid)
 {
     const bool peep = (p.flags & F_PEEPHOLE) != 0;
     const int16_t *xrow = p.X + ((size_t)t * p.B + b) * p.N + n0;
-    for (int col = 0; col < p.nc_pad; col += 16) {
+    for (int col = 0; col < n_cnt; col += 16) {
         uint32_t r[16];
         __syncwarp();                 // the TMEM load is warp-collective: reconverge after the per-row branch
         ptx::tmem_ld_32x16(taddr + (uint32_t)col, r);
         ptx::tmem_ld_wait();
-        if (!row_valid || col >= n_cnt) continue;
-        int32_t out[16];
+        if (!row_valid) continue;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const int n = col + j;
-            if (n < n_cnt) {
-                const int gi = (p.G == 4) ? (j & 3) : (n % 3);
-                int32_t acc = sat32((int64_t)(int32_t)r[j] + bh_s[n]);
-                int32_t H = sat16(rescale_sel(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
-                int32_t X = xrow[n];
-                out[j] = peep ? X + H : sat16(X + H);
-            } else {
-                out[j] = 0;
+        for (int h8 = 0; h8 < 2; ++h8) {
+            const int c8 = col + 8 * h8;
+            if (c8 >= n_cnt) break;                      // n_cnt is a multiple of 8
+            const uint4 xv = __ldg(reinterpret_cast<const uint4 *>(xrow + c8));
+            const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+            const int ph = (G == 4) ? 0 : c8 % 3;
+            int32_t o[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int gi = (G == 4) ? (j & 3) : (ph + j) % 3;
+                const int32_t acc = add_sat((int32_t)r[8 * h8 + j], bh_s[c8 + j]);
+                const int32_t H = sat16(rescale_sel(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
+                const int32_t X = (j & 1) ? hi16(xw[j >> 1]) : lo16(xw[j >> 1]);
+                o[j] = peep ? X + H : sat16(X + H);
             }
-        }
-        if (peep) {
-            int32_t *dst = p.pre + (size_t)b * p.N + n0 + col;
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-                if (col + j < n_cnt) dst[j] = out[j];
-        } else {
-            int16_t *dst = (int16_t *)p.pre + (size_t)b * p.N + n0 + col;
-#pragma unroll
-            for (int j = 0; j < 16; ++j)
-                if (col + j < n_cnt) dst[j] = (int16_t)out[j];
+            if (peep) {
+                int32_t *dst = p.pre + (size_t)b * p.N + n0 + c8;
+                *reinterpret_cast<int4 *>(dst) = make_int4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<int4 *>(dst + 4) = make_int4(o[4], o[5], o[6], o[7]);
+            } else {
+                int16_t *dst = (int16_t *)p.pre + (size_t)b * p.N + n0 + c8;
+                *reinterpret_cast<uint4 *>(dst) = make_uint4(pack16(o[0], o[1]), pack16(o[2], o[3]), pack16(o[4], o[5]), pack16(o[6], o[7]));
+            }
         }
     }
 }
@@ -181,30 +199,27 @@ __device__ __forceinline__ void phase_c_row(const RecParams &p, uint32_t taddr, 
         uint32_t w[4] = {0, 0, 0, 0};
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-            const int o = p0 + col + j;
-            int32_t hq = 0;
-            if (o < p.O) {
-                int32_t acc = sat32((int64_t)(int32_t)r[j] + p.bp[o]);
-                hq = sat8(rescale_sel(acc, p.eff_proj, p.f_proj, p.fast_rescale_ok) + p.zp_h);
-            }
+            // O is a multiple of 16, so a 16-wide group is either fully inside or fully outside
+            const int32_t acc = add_sat((int32_t)r[j], __ldg(p.bp + p0 + col + j));
+            const int32_t hq = sat8(rescale_sel(acc, p.eff_proj, p.f_proj, p.fast_rescale_ok) + p.zp_h);
             w[j >> 2] |= (uint32_t)(hq & 0xff) << (8 * (j & 3));
         }
-        // O is a multiple of 16, so a 16-wide group is either fully inside or fully outside
-        uint4 v = make_uint4(w[0], w[1], w[2], w[3]);
+        const uint4 v = make_uint4(w[0], w[1], w[2], w[3]);
         *reinterpret_cast<uint4 *>(h_next + (size_t)b * p.O + p0 + col) = v;
         *reinterpret_cast<uint4 *>(p.y + ((size_t)t * p.B + b) * p.O + p0 + col) = v;
     }
 }
 
 // ------------------------------------------------------------------------------------------------
-// Phase B helpers
+// Phase B: elementwise work on a contiguous range of the B x C cell grid.
 
-struct GateStats { LnStats s[4]; };
-
-// Block-wide reduction of per-gate sum / sum of squares; result for gate slots in `mask` lands in ctl->stat_*.
-__device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, long long (&sum)[4], long long (&sq)[4], int G, int n)
+// Block-wide reduction of per-gate sum / sum of squares into ctl->ln_rows[slot][*].
+template <int G>
+__device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, const long long (&sum)[4], const long long (&sq)[4], int n,
+                                                   int slot)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+#pragma unroll
     for (int g = 0; g < G; ++g) {
         long long a = sum[g], b = sq[g];
         for (int o = 16; o > 0; o >>= 1) {
@@ -217,141 +232,216 @@ __device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, long long (&sum)
     if (threadIdx.x < G) {
         long long a = 0, b = 0;
         for (int w = 0; w < RTHREADS / 32; ++w) { a += ctl->red_sum[w][threadIdx.x]; b += ctl->red_sq[w][threadIdx.x]; }
-        LnStats st = ln_stats(a, b, n);
-        ctl->stat_mean[threadIdx.x] = st.mean;
-        ctl->stat_sigma[threadIdx.x] = st.sigma;
+        ctl->ln_rows[slot][threadIdx.x] = make_ln_row(ln_stats(a, b, n));
     }
     __syncthreads();
 }
 
-__device__ __forceinline__ int32_t ln_gate(const RecParams &p, const RecCtl *ctl, int32_t pre, int n, int gi)
+// G int16 values of two adjacent cells (cell index even): v[k][gi]
+template <int G>
+__device__ __forceinline__ void load_pair_i16(const int16_t *ptr, bool readonly, int32_t (&v)[2][4])
 {
-    LnStats st;
-    st.mean = ctl->stat_mean[gi];
-    st.sigma = ctl->stat_sigma[gi];
-    return ln_apply(pre, st, p.L[n], p.bln[n], p.eff_ln[gi]);
+    if (G == 4) {
+        const uint4 q = readonly ? __ldg(reinterpret_cast<const uint4 *>(ptr)) : *reinterpret_cast<const uint4 *>(ptr);
+        v[0][0] = lo16(q.x); v[0][1] = hi16(q.x); v[0][2] = lo16(q.y); v[0][3] = hi16(q.y);
+        v[1][0] = lo16(q.z); v[1][1] = hi16(q.z); v[1][2] = lo16(q.w); v[1][3] = hi16(q.w);
+    } else {
+        const uint32_t *w = reinterpret_cast<const uint32_t *>(ptr);
+        const uint32_t a = readonly ? __ldg(w) : w[0], b = readonly ? __ldg(w + 1) : w[1], c = readonly ? __ldg(w + 2) : w[2];
+        v[0][0] = lo16(a); v[0][1] = hi16(a); v[0][2] = lo16(b);
+        v[1][0] = hi16(b); v[1][1] = lo16(c); v[1][2] = hi16(c);
+        v[0][3] = 0; v[1][3] = 0;
+    }
+}
+template <int G>
+__device__ __forceinline__ void load_pair_i32(const int32_t *ptr, bool readonly, int32_t (&v)[2][4])
+{
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+#pragma unroll
+        for (int g = 0; g < 4; ++g) v[k][g] = g < G ? (readonly ? __ldg(ptr + k * G + g) : ptr[k * G + g]) : 0;
 }
 
-__device__ __forceinline__ void store_hidden(const RecParams &p, int b, int u, int t, int32_t m, int8_t *h_next)
+__device__ __forceinline__ void store_hidden_pair(const RecParams &p, int b, int u, int t, int32_t m0, int32_t m1, int8_t *h_next)
 {
+    const uint16_t v = (uint16_t)((m0 & 0xff) | ((m1 & 0xff) << 8));
     if (p.flags & F_PROJECTION) {
-        p.mbuf[(size_t)b * p.C + u] = (int8_t)m;
+        *reinterpret_cast<uint16_t *>(p.mbuf + (size_t)b * p.C + u) = v;
     } else {
-        h_next[(size_t)b * p.O + u] = (int8_t)m;
-        p.y[((size_t)t * p.B + b) * p.O + u] = (int8_t)m;
+        *reinterpret_cast<uint16_t *>(h_next + (size_t)b * p.O + u) = v;
+        *reinterpret_cast<uint16_t *>(p.y + ((size_t)t * p.B + b) * p.O + u) = v;
     }
 }
 
-// Elementwise phase for the units of this CTA.  `row_s` is a shared buffer of C*G int16 plus C int16.
-__device__ void phase_b(const RecParams &p, RecCtl *ctl, int t, int8_t *h_next, int16_t *row_s)
+// Two adjacent cells (u even) of row b, every step after the gate sums (not used for layer norm + peephole).
+template <int G, bool LN, bool PEEP>
+__device__ __forceinline__ void cell_pair(const RecParams &p, const LnRow *lr, int b, int u, int t, int8_t *h_next)
 {
-    const bool ln = (p.flags & F_LAYERNORM) != 0, peep = (p.flags & F_PEEPHOLE) != 0, cifg = (p.flags & F_CIFG) != 0;
-    const int G = p.G;
-    const int si = p.gate_slot[0], sf = p.gate_slot[1], sz = p.gate_slot[2], so = p.gate_slot[3];
-    const int total_units = p.B * p.chunks;
-    int u_begin = blockIdx.x * p.units_per_cta, u_end = u_begin + p.units_per_cta;
-    if (u_end > total_units) u_end = total_units;
-    int stats_row = -1;
-    const int16_t *pre16 = (const int16_t *)p.pre;
+    constexpr int SI = 0, SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
+    const size_t nb = (size_t)b * p.N + (size_t)u * G;
+    const int nu = u * G;
+    int16_t *c_ptr = p.c + (size_t)b * p.C + u;
+    const uint32_t cw = *reinterpret_cast<const uint32_t *>(c_ptr);
+    const int32_t c_old[2] = {lo16(cw), hi16(cw)};
+    int32_t a[2][4], P[2][4];
+    if (PEEP) {
+        load_pair_i32<G>(p.pre + nb, false, a);
+        load_pair_i16<G>(p.P + nu, true, P);
+#pragma unroll
+        for (int k = 0; k < 2; ++k)
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                if (g == SO) continue;
+                int32_t v = a[k][g];
+                if (g != SZ) v += sat16(rescale_any(P[k][g] * c_old[k], p.eff_c[g], p.f_c[g]));
+                a[k][g] = sat16(v);
+            }
+    } else {
+        load_pair_i16<G>((const int16_t *)p.pre + nb, false, a);
+        if (LN) {
+            int32_t L[2][4], bl[2][4];
+            load_pair_i16<G>(p.L + nu, true, L);
+            load_pair_i32<G>(p.bln + nu, true, bl);
+#pragma unroll
+            for (int k = 0; k < 2; ++k)
+#pragma unroll
+                for (int g = 0; g < G; ++g) a[k][g] = ln_apply_fast(a[k][g], lr[g], L[k][g], bl[k][g], p.eff_ln[g], p.f_ln[g]);
+        }
+    }
+    int32_t c_new[2], m[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int32_t f = sigmoid_q_fast(a[k][SF], 3), z = tanh_q_fast(a[k][SZ], 3);
+        int32_t i;
+        if (G == 4) i = sigmoid_q_fast(a[k][SI], 3);
+        else { i = 32768 - f; if (i > 32767) i = 32767; }          // coupled input gate, Section 3.2.9
+        c_new[k] = cell_update_fast(i, z, f, c_old[k], p.m_bits);
+        int32_t ao = a[k][SO];
+        if (PEEP) ao = sat16(ao + sat16(rescale_any(P[k][SO] * c_new[k], p.eff_c[SO], p.f_c[SO])));
+        const int32_t o = sigmoid_q_fast(ao, 3);
+        m[k] = hidden_q_fast(o, c_new[k], p.m_bits, p.eff_m, p.f_m, p.zp_m);
+    }
+    *reinterpret_cast<uint32_t *>(c_ptr) = pack16(c_new[0], c_new[1]);
+    store_hidden_pair(p, b, u, t, m[0], m[1], h_next);
+}
 
-    for (int unit = u_begin; unit < u_end; ++unit) {
-        const int b = unit / p.chunks, ch = unit % p.chunks;
-        const int k0 = ch * p.chunk_cells;
-        const int k1 = (k0 + p.chunk_cells < p.C) ? k0 + p.chunk_cells : p.C;
+template <int G, bool LN, bool PEEP>
+__device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, int t, int8_t *h_next)
+{
+    const int total = p.B * p.C;
+    const int i0 = blockIdx.x * p.items_per_cta;
+    int i1 = i0 + p.items_per_cta;
+    if (i1 > total) i1 = total;
+    if (i0 >= i1) return;
+    const int b_first = i0 / p.C, b_last = (i1 - 1) / p.C;
+    for (int rb = b_first; rb <= b_last; rb += MAX_LN_ROWS) {
+        const int re = (rb + MAX_LN_ROWS - 1 < b_last) ? rb + MAX_LN_ROWS - 1 : b_last;
+        if (LN) {
+            for (int r = rb; r <= re; ++r) {
+                const int16_t *row = (const int16_t *)p.pre + (size_t)r * p.N;
+                long long sum[4] = {0, 0, 0, 0}, sq[4] = {0, 0, 0, 0};
+                for (int u = 2 * threadIdx.x; u < p.C; u += 2 * RTHREADS) {
+                    int32_t v[2][4];
+                    load_pair_i16<G>(row + (size_t)u * G, false, v);
+#pragma unroll
+                    for (int g = 0; g < G; ++g) {
+                        sum[g] += v[0][g] + v[1][g];
+                        sq[g] += (long long)(v[0][g] * v[0][g]) + (long long)(v[1][g] * v[1][g]);
+                    }
+                }
+                block_reduce_stats<G>(ctl, sum, sq, p.C, r - rb);
+            }
+        }
+        const int j0 = i0 > rb * p.C ? i0 : rb * p.C;
+        const int j1 = i1 < (re + 1) * p.C ? i1 : (re + 1) * p.C;
+        for (int i = j0 + 2 * threadIdx.x; i < j1; i += 2 * RTHREADS) {
+            const int b = i / p.C, u = i - b * p.C;
+            cell_pair<G, LN, PEEP>(p, ctl->ln_rows[b - rb], b, u, t, h_next);
+        }
+        if (LN) __syncthreads();      // the statistics slots are reused by the next batch of rows
+    }
+}
+
+// Layer norm with peephole: the gate sums need their peephole term before the statistics, and the output
+// gate's statistics need c^t of the whole row, so a row is processed by one CTA in three passes.
+template <int G>
+__device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl, int t, int8_t *h_next, int16_t *row_s)
+{
+    constexpr int SI = 0, SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
+    const int rows_per_cta = p.items_per_cta / p.C;
+    const int b0 = blockIdx.x * rows_per_cta;
+    const int b1 = (b0 + rows_per_cta < p.B) ? b0 + rows_per_cta : p.B;
+    int16_t *pre_s = row_s, *cnew_s = row_s + (size_t)p.C * G;
+    for (int b = b0; b < b1; ++b) {
         int16_t *c_row = p.c + (size_t)b * p.C;
-
-        if (ln && peep) {
-            // the unit is a whole row: gate sums need the peephole term before their statistics
-            int16_t *pre_s = row_s, *cnew_s = row_s + (size_t)p.C * G;
-            const int32_t *xh = p.pre + (size_t)b * p.N;
-            long long sum[4] = {0, 0, 0, 0}, sq[4] = {0, 0, 0, 0};
-            for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
-                const int32_t c_old = c_row[u];
-                for (int gi = 0; gi < G; ++gi) {
-                    if (gi == so) continue;
-                    const int n = u * G + gi;
-                    int32_t v = xh[n];
-                    if (gi != sz) v += sat16(mbqm((int32_t)p.P[n] * c_old, p.eff_c[gi]));
-                    v = sat16(v);
-                    pre_s[n] = (int16_t)v;
-                    sum[gi] += v;
-                    sq[gi] += (long long)v * v;
-                }
-            }
-            block_reduce_stats(ctl, sum, sq, G, p.C);
-            long long sum_o[4] = {0, 0, 0, 0}, sq_o[4] = {0, 0, 0, 0};
-            for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
-                const int nb = u * G;
-                int32_t f = sigmoid_q(ln_gate(p, ctl, pre_s[nb + sf], nb + sf, sf), 3);
-                int32_t z = tanh_q(ln_gate(p, ctl, pre_s[nb + sz], nb + sz, sz), 3);
-                int32_t i;
-                if (cifg) { i = 32768 - f; if (i > 32767) i = 32767; }
-                else i = sigmoid_q(ln_gate(p, ctl, pre_s[nb + si], nb + si, si), 3);
-                int32_t c_new = cell_update(i, z, f, c_row[u], p.m_bits);
-                c_row[u] = (int16_t)c_new;
-                cnew_s[u] = (int16_t)c_new;
-                int32_t v = sat16(xh[nb + so] + sat16(mbqm((int32_t)p.P[nb + so] * c_new, p.eff_c[so])));
-                pre_s[nb + so] = (int16_t)v;
-                sum_o[so] += v;
-                sq_o[so] += (long long)v * v;
-            }
-            __syncthreads();          // statistics of i, f, z are consumed; the slots are reused for o
-            block_reduce_stats(ctl, sum_o, sq_o, G, p.C);
-            for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
-                const int n = u * G + so;
-                int32_t o = sigmoid_q(ln_gate(p, ctl, pre_s[n], n, so), 3);
-                store_hidden(p, b, u, t, hidden_q(o, cnew_s[u], p.m_bits, p.eff_m, p.zp_m), h_next);
-            }
-            __syncthreads();
-            continue;
-        }
-
-        if (ln && b != stats_row) {
-            const int16_t *row = pre16 + (size_t)b * p.N;
-            long long sum[4] = {0, 0, 0, 0}, sq[4] = {0, 0, 0, 0};
-            for (int u = threadIdx.x; u < p.C; u += RTHREADS)
-                for (int gi = 0; gi < G; ++gi) {
-                    long long v = row[u * G + gi];
-                    sum[gi] += v;
-                    sq[gi] += v * v;
-                }
-            __syncthreads();          // previous unit may still read the statistics
-            block_reduce_stats(ctl, sum, sq, G, p.C);
-            stats_row = b;
-        }
-
-        for (int u = k0 + threadIdx.x; u < k1; u += RTHREADS) {
-            const int nb = u * G;
+        const int32_t *xh = p.pre + (size_t)b * p.N;
+        const LnRow *lr = ctl->ln_rows[0];
+        long long sum[4] = {0, 0, 0, 0}, sq[4] = {0, 0, 0, 0};
+        for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
             const int32_t c_old = c_row[u];
-            int32_t af, az, ai = 0, ao_part;
-            if (peep) {
-                const int32_t *xh = p.pre + (size_t)b * p.N + nb;
-                af = sat16(xh[sf] + sat16(mbqm((int32_t)p.P[nb + sf] * c_old, p.eff_c[sf])));
-                az = sat16(xh[sz]);
-                if (!cifg) ai = sat16(xh[si] + sat16(mbqm((int32_t)p.P[nb + si] * c_old, p.eff_c[si])));
-                ao_part = xh[so];
-            } else {
-                const int16_t *pr = pre16 + (size_t)b * p.N + nb;
-                af = pr[sf]; az = pr[sz];
-                if (!cifg) ai = pr[si];
-                ao_part = pr[so];
-                if (ln) {
-                    af = ln_gate(p, ctl, af, nb + sf, sf);
-                    az = ln_gate(p, ctl, az, nb + sz, sz);
-                    if (!cifg) ai = ln_gate(p, ctl, ai, nb + si, si);
-                    ao_part = ln_gate(p, ctl, ao_part, nb + so, so);
-                }
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                if (g == SO) continue;
+                const int n = u * G + g;
+                int32_t v = xh[n];
+                if (g != SZ) v += sat16(rescale_any((int32_t)__ldg(p.P + n) * c_old, p.eff_c[g], p.f_c[g]));
+                v = sat16(v);
+                pre_s[n] = (int16_t)v;
+                sum[g] += v;
+                sq[g] += (long long)(v * v);
             }
-            int32_t f = sigmoid_q(af, 3), z = tanh_q(az, 3), i;
-            if (cifg) { i = 32768 - f; if (i > 32767) i = 32767; }
-            else i = sigmoid_q(ai, 3);
-            int32_t c_new = cell_update(i, z, f, c_old, p.m_bits);
-            c_row[u] = (int16_t)c_new;
-            int32_t ao = ao_part;
-            if (peep) ao = sat16(ao_part + sat16(mbqm((int32_t)p.P[nb + so] * c_new, p.eff_c[so])));
-            int32_t o = sigmoid_q(ao, 3);
-            store_hidden(p, b, u, t, hidden_q(o, c_new, p.m_bits, p.eff_m, p.zp_m), h_next);
         }
+        block_reduce_stats<G>(ctl, sum, sq, p.C, 0);
+        long long sum_o[4] = {0, 0, 0, 0}, sq_o[4] = {0, 0, 0, 0};
+        for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
+            const int nb = u * G;
+            int32_t a[4];
+#pragma unroll
+            for (int g = 0; g < G; ++g)
+                if (g != SO) a[g] = ln_apply_fast(pre_s[nb + g], lr[g], __ldg(p.L + nb + g), __ldg(p.bln + nb + g), p.eff_ln[g], p.f_ln[g]);
+            const int32_t f = sigmoid_q_fast(a[SF], 3), z = tanh_q_fast(a[SZ], 3);
+            int32_t i;
+            if (G == 4) i = sigmoid_q_fast(a[SI], 3);
+            else { i = 32768 - f; if (i > 32767) i = 32767; }
+            const int32_t c_new = cell_update_fast(i, z, f, c_row[u], p.m_bits);
+            c_row[u] = (int16_t)c_new;
+            cnew_s[u] = (int16_t)c_new;
+            const int32_t v = sat16(xh[nb + SO] + sat16(rescale_any((int32_t)__ldg(p.P + nb + SO) * c_new, p.eff_c[SO], p.f_c[SO])));
+            pre_s[nb + SO] = (int16_t)v;
+            sum_o[SO] += v;
+            sq_o[SO] += (long long)(v * v);
+        }
+        __syncthreads();              // statistics of i, f, z are consumed; their slots are reused for o
+        block_reduce_stats<G>(ctl, sum_o, sq_o, p.C, 0);
+        for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
+            const int n = u * G + SO;
+            const int32_t ao = ln_apply_fast(pre_s[n], lr[SO], __ldg(p.L + n), __ldg(p.bln + n), p.eff_ln[SO], p.f_ln[SO]);
+            const int32_t o = sigmoid_q_fast(ao, 3);
+            const int32_t m = hidden_q_fast(o, cnew_s[u], p.m_bits, p.eff_m, p.f_m, p.zp_m);
+            if (p.flags & F_PROJECTION) {
+                p.mbuf[(size_t)b * p.C + u] = (int8_t)m;
+            } else {
+                h_next[(size_t)b * p.O + u] = (int8_t)m;
+                p.y[((size_t)t * p.B + b) * p.O + u] = (int8_t)m;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+__device__ __forceinline__ void phase_b(const RecParams &p, RecCtl *ctl, int t, int8_t *h_next, int16_t *row_s)
+{
+    const bool ln = (p.flags & F_LAYERNORM) != 0, peep = (p.flags & F_PEEPHOLE) != 0;
+    if (p.G == 4) {
+        if (ln && peep) phase_b_ln_peep<4>(p, ctl, t, h_next, row_s);
+        else if (ln) phase_b_flat<4, true, false>(p, ctl, t, h_next);
+        else if (peep) phase_b_flat<4, false, true>(p, ctl, t, h_next);
+        else phase_b_flat<4, false, false>(p, ctl, t, h_next);
+    } else {
+        if (ln && peep) phase_b_ln_peep<3>(p, ctl, t, h_next, row_s);
+        else if (ln) phase_b_flat<3, true, false>(p, ctl, t, h_next);
+        else if (peep) phase_b_flat<3, false, true>(p, ctl, t, h_next);
+        else phase_b_flat<3, false, false>(p, ctl, t, h_next);
     }
 }
 
@@ -431,6 +521,16 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
     int stage = 0; uint32_t ring_phase = 0;      // advanced identically by producer and MMA issuer
     const uint32_t idesc_a = ptx::idesc_i8(128, p.nc_pad), idesc_c = ptx::idesc_i8(128, p.pn);
 
+    const bool timing = p.phase_ns != nullptr && cta == 0 && threadIdx.x == 0;
+    unsigned long long t_mark = timing ? globaltimer() : 0ull;
+    auto lap = [&](int slot) {
+        if (timing) {
+            unsigned long long now = globaltimer();
+            p.phase_ns[slot] += now - t_mark;
+            t_mark = now;
+        }
+    };
+
     for (int t = 0; t < p.T; ++t) {
         const int cur = t & 1;
         int8_t *h_next = p.hbuf + (size_t)(cur ^ 1) * p.Bpad * p.O;
@@ -472,25 +572,32 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
                     }
                 }
                 __syncwarp();
-            } else {
+            } else if (warp < 10) {
                 const int e = warp - 2, quarter = warp & 3, mi = e >> 2;
                 if (mi < p.MT) {
                     if (__all_sync(0xffffffffu, wait_or_abort(&ctl->acc_full[mi], par, abort_flag))) {
                         ptx::tc_fence_after();
                         const int b = mi * 128 + quarter * 32 + lane;
-                        phase_a_row(p, tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * p.nc_pad), b, t, n0, n_cnt,
-                                    bh_s, b < p.B);
+                        const uint32_t ta = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * p.nc_pad);
+                        if (p.G == 4) phase_a_row<4>(p, ta, b, t, n0, n_cnt, bh_s, b < p.B);
+                        else phase_a_row<3>(p, ta, b, t, n0, n_cnt, bh_s, b < p.B);
                         ptx::tc_fence_before();
                     }
                 }
             }
         }
+        __syncthreads();
+        lap(0);
         grid_sync(p, epoch, abort_flag);
+        lap(1);
         if (*abort_flag) break;
 
         // ================= phase B: elementwise =================
         phase_b(p, ctl, t, h_next, row_s);
+        __syncthreads();
+        lap(2);
         grid_sync(p, epoch, abort_flag);
+        lap(3);
         if (*abort_flag) break;
 
         // ================= phase C: projection =================
@@ -535,7 +642,10 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
                     }
                 }
             }
+            __syncthreads();
+            lap(4);
             grid_sync(p, epoch, abort_flag);
+            lap(5);
             if (*abort_flag) break;
         }
     }
@@ -653,7 +763,8 @@ void fast_layer_destroy(FastLayer &) {}
 bool fast_recurrent_supported(const FastLayer &f, const LayerParams &, int B) { return f.rec_ok && B <= 256; }
 
 int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastScratch &s, const int16_t *X, int T, int B,
-                          int8_t *h, int16_t *c, int8_t *y, int *status, cudaStream_t st, int *launches)
+                          int8_t *h, int16_t *c, int8_t *y, int *status, unsigned long long *phase_ns, cudaStream_t st,
+                          int *launches)
 {
     RecParams rp;
     memset(&rp, 0, sizeof(rp));
@@ -663,30 +774,23 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     rp.cpc = f.cpc; rp.n_cta_a = f.n_cta_a; rp.nc_pad = f.nc_pad;
     rp.pn = f.pn; rp.npn = f.npn; rp.n_ptiles = rp.MT * f.npn;
     rp.kb_h = f.kb_h; rp.kb_c = f.kb_c; rp.stages = f.stages;
-    // elementwise units: (row, chunk of cells).  Layer norm with peephole needs the whole row in one CTA.
-    const bool ln_peep = (p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE);
-    int best_chunks = 1;
-    if (!ln_peep) {
-        double best_eff = -1.0;
-        const int max_chunks = p.C / 16 > 0 ? p.C / 16 : 1;
-        for (int ch = 1; ch <= max_chunks && ch <= 256; ++ch) {
-            long units = (long)B * ch;
-            long per = (units + f.grid - 1) / f.grid;
-            double eff = (double)units / ((double)per * f.grid);
-            if (eff > best_eff + 0.02) { best_eff = eff; best_chunks = ch; }
-        }
-    }
-    rp.chunks = best_chunks;
-    rp.chunk_cells = (p.C + best_chunks - 1) / best_chunks;
-    rp.units_per_cta = (int)(((long)B * best_chunks + f.grid - 1) / f.grid);
+    // elementwise phase: contiguous ranges of the B x C cell grid (whole rows with layer norm + peephole)
+    if ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE))
+        rp.items_per_cta = ((B + f.grid - 1) / f.grid) * p.C;
+    else
+        rp.items_per_cta = round_up((int)(((long)B * p.C + f.grid - 1) / f.grid), 8);
     rp.fast_rescale_ok = 1;
     for (int g = 0; g < p.G; ++g) {
         rp.eff_h[g] = p.eff_h[g]; rp.eff_c[g] = p.eff_c[g]; rp.eff_ln[g] = p.eff_ln[g];
         rp.f_h[g] = make_fast_scale(p.eff_h[g]);
+        rp.f_c[g] = make_fast_scale(p.eff_c[g]);
+        rp.f_ln[g] = make_fast_scale(p.eff_ln[g]);
         if (p.eff_h[g].shift > 0) rp.fast_rescale_ok = 0;
     }
     rp.eff_m = p.eff_m; rp.eff_proj = p.eff_proj;
     rp.f_proj = make_fast_scale(p.eff_proj);
+    rp.f_m = make_fast_scale(p.eff_m);
+    rp.phase_ns = phase_ns;
     if (p.eff_proj.shift > 0) rp.fast_rescale_ok = 0;
     for (int g = 0; g < 4; ++g) rp.gate_slot[g] = p.slot_of_gate[g];
     rp.X = X; rp.c = c; rp.y = y;

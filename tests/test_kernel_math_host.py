@@ -109,3 +109,68 @@ def test_cell_update_and_hidden(H):
         zp = int(rng.integers(-128, 128))
         want_m = max(-128, min(127, R.mbqm(o * R.tanh(want_c, m), eff) + zp))
         assert H.qmh_hidden(o, want_c, m, eff[0], eff[1], zp) == want_m
+
+
+# ---------------------------------------------------------------- the 32-bit / fp32-assisted forms the kernels run
+
+@pytest.mark.parametrize("m", [0, 1, 2, 3, 4, 5, 6, 9, 12, 15])
+def test_fast_activations_exhaustive(H, m):
+    out = np.empty(65536, np.int32)
+    H.qmh_sigmoid_fast_all(m, out.ctypes.data_as(C.c_void_p))
+    assert np.array_equal(out, R.sigmoid_all(m))
+    H.qmh_tanh_fast_all(m, out.ctypes.data_as(C.c_void_p))
+    assert np.array_equal(out, R.tanh_all(m))
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_fast_layernorm_rows(H, seed):
+    rng = np.random.default_rng(500 + seed)
+    n = int(rng.integers(1, 2100))
+    q = (rng.integers(-32768, 32768, n) // int(rng.integers(1, 60))).astype(np.int16)
+    if seed == 0:
+        q[:] = -5
+    if seed == 1:                                   # one outlier: the largest z-score
+        q[:] = 0
+        q[3] = 32767
+    if seed == 2:
+        q = np.where(np.arange(n) % 2 == 0, 32767, -32768).astype(np.int16)
+    L = rng.integers(-32767, 32768, n).astype(np.int16)
+    b = (rng.integers(-2 ** 31 + 1, 2 ** 31, n) // int(rng.integers(1, 3000))).astype(np.int32)
+    eff = (int(rng.integers(1 << 30, 1 << 31)), int(rng.integers(-14, 2)))
+    out = np.empty(n, np.int16)
+    H.qmh_layernorm_row_fast(q.ctypes.data_as(C.c_void_p), n, L.ctypes.data_as(C.c_void_p), b.ctypes.data_as(C.c_void_p),
+                             eff[0], eff[1], out.ctypes.data_as(C.c_void_p))
+    assert np.array_equal(out, R.layernorm_row(q, L, b, eff))
+
+
+def test_fast_ln_quotient_with_adversarial_statistics(H):
+    """Statistics that cannot come from a real row still must divide exactly (tiny sigma, huge deviation)."""
+    H.qmh_ln_quotient_fast.restype = C.c_int64
+    H.qmh_ln_quotient_fast.argtypes = [C.c_int32, C.c_int64, C.c_int64]
+    rng = np.random.default_rng(9)
+    cases = [(32767, -(1 << 25), 1), (-32768, (1 << 25), 1), (5000, 0, 3), (123, 125000, 7), (0, 0, 0), (77, 5, (1 << 26) - 1)]
+    cases += [(int(rng.integers(-32768, 32768)), int(rng.integers(-(1 << 25), 1 << 25)), int(rng.integers(1, 1 << int(rng.integers(1, 27)))))
+              for _ in range(20000)]
+    for q, mean, sigma in cases:
+        want = 0 if sigma == 0 else R.rdiv(1024 * (1024 * q - mean), sigma)
+        assert H.qmh_ln_quotient_fast(q, mean, sigma) == want, (q, mean, sigma)
+
+
+def test_fast_cell_update_and_hidden(H):
+    H.qmh_cell_update_fast.restype = C.c_int32
+    H.qmh_cell_update_fast.argtypes = [C.c_int32] * 5
+    H.qmh_hidden_fast.restype = C.c_int32
+    H.qmh_hidden_fast.argtypes = [C.c_int32] * 6
+    rng = np.random.default_rng(12)
+    edge = [(32767, 32767, 32767, 32767), (32767, -32768, 32767, -32768), (1, -1, 1, -1), (0, 0, 0, 0), (16384, 1, 16384, -1)]
+    rand = [tuple(int(v) for v in (rng.integers(0, 32768), rng.integers(-32768, 32768), rng.integers(0, 32768),
+                                   rng.integers(-32768, 32768))) for _ in range(5000)]
+    for i, z, f, c in edge + rand:
+        for m in (0, 3, 5):
+            want = max(-32768, min(32767, R.rdivpot(i * z, 15 + m) + R.rdivpot(f * c, 15)))
+            assert H.qmh_cell_update_fast(i, z, f, c, m) == want
+    for _ in range(3000):
+        o = int(rng.integers(0, 32768)); c = int(rng.integers(-32768, 32768)); m = int(rng.integers(0, 7))
+        eff = (int(rng.integers(1 << 30, 1 << 31)), int(rng.integers(-24, -18))); zp = int(rng.integers(-128, 128))
+        want = max(-128, min(127, R.mbqm(o * R.tanh(c, m), eff) + zp))
+        assert H.qmh_hidden_fast(o, c, m, eff[0], eff[1], zp) == want
