@@ -150,6 +150,20 @@ typedef struct {
 int qlstm_set_profiling(qlstm_t *q, int enabled);
 int qlstm_get_profile(qlstm_t *q, qlstm_profile_t *out, int reset);
 
+/*
+ * Evaluators of two building blocks on their own, on the current device, with the same device code the
+ * recurrent kernel runs.  They exist so that the integer nonlinearities can be checked over their whole
+ * domain (Section 3.2.1: int16 Q_{m.15-m} in, Q0.15 out) and the integer layer norm (Section 3.2.6) on
+ * hand-picked rows.
+ *   qlstm_eval_activations: sigmoid_dev / tanh_dev DEVICE int16 [65536], entry x + 32768 holds f(x) for the
+ *     input format Q_{m.15-m} with m = cell_int_bits (gates use m = 3).
+ *   qlstm_eval_layernorm_row: q_dev int16 [n], L_dev int16 [n], b_dev int32 [n], out_dev int16 [n] (Q3.12);
+ *     n <= 8191.
+ */
+int qlstm_eval_activations(int cell_int_bits, int16_t *sigmoid_dev, int16_t *tanh_dev, void *cuda_stream);
+int qlstm_eval_layernorm_row(const int16_t *q_dev, int n, const int16_t *L_dev, const int32_t *b_dev,
+                             qlstm_scale_t eff_ln, int16_t *out_dev, void *cuda_stream);
+
 /* Device properties the library sees: SM count, and resident blocks of the persistent kernel. */
 int qlstm_device_info(qlstm_t *q, int *sm_count, int *persistent_blocks);
 

@@ -21,7 +21,7 @@ IMPL_AUTO, IMPL_SIMPLE, IMPL_FAST = 0, 1, 2
 
 EXPORTS = ["qlstm_create", "qlstm_run", "qlstm_run_host", "qlstm_input_projection", "qlstm_last_status",
            "qlstm_destroy", "qlstm_strerror", "qlstm_trace_bytes", "qlstm_set_impl", "qlstm_set_profiling",
-           "qlstm_get_profile", "qlstm_device_info"]
+           "qlstm_get_profile", "qlstm_device_info", "qlstm_eval_activations", "qlstm_eval_layernorm_row"]
 
 
 class Scale(C.Structure):
@@ -93,6 +93,10 @@ def lib():
         L.qlstm_get_profile.argtypes = [C.c_void_p, C.POINTER(Profile), C.c_int]
         L.qlstm_device_info.restype = C.c_int
         L.qlstm_device_info.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
+        L.qlstm_eval_activations.restype = C.c_int
+        L.qlstm_eval_activations.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.qlstm_eval_layernorm_row.restype = C.c_int
+        L.qlstm_eval_layernorm_row.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -224,6 +228,17 @@ class QLSTM:
         a, b = C.c_int(), C.c_int()
         _check(lib().qlstm_device_info(self._h, C.byref(a), C.byref(b)), "qlstm_device_info")
         return a.value, b.value
+
+
+def eval_activations(cell_int_bits: int, sigmoid_out, tanh_out, stream: int = 0):
+    """qlstm_eval_activations on two device int16 [65536] tensors."""
+    _check(lib().qlstm_eval_activations(cell_int_bits, _dev_ptr(sigmoid_out), _dev_ptr(tanh_out), stream),
+           "qlstm_eval_activations")
+
+
+def eval_layernorm_row(q, n: int, L, b, eff_ln, out, stream: int = 0):
+    _check(lib().qlstm_eval_layernorm_row(_dev_ptr(q), n, _dev_ptr(L), _dev_ptr(b), Scale(int(eff_ln[0]), int(eff_ln[1])),
+                                          _dev_ptr(out), stream), "qlstm_eval_layernorm_row")
 
 
 def parse_trace(buf: np.ndarray, dims: Sequence, T: int, B: int):

@@ -133,18 +133,23 @@ QL_HD int32_t tanh_q(int32_t x, int m)
 }
 
 // ---- the same two functions in 32-bit registers ------------------------------------------------
-// Bit-identical to sigmoid_q / tanh_q above (swept exhaustively on the host), but written for the
-// GPU's integer pipes: 32x32->64 multiply-adds, funnel shifts, and one fp32 reciprocal whose result
-// is only an estimate of the final quotient - an exact 64-bit remainder test then fixes it.
-//
-// Rounding x / 2^26 half away from zero on a signed product p: (p + 2^25 - [p < 0]) >> 26.  In the
-// Horner chain the sign of the accumulator alternates deterministically (|c_k| dominates the term
-// it is added to), so [p < 0] depends on the sign of g alone and costs nothing per step.
+// Bit-identical to sigmoid_q / tanh_q above (swept exhaustively on the host and on the GPU), but
+// written for the GPU's integer pipes:
+//  * the polynomial variable is pre-shifted by 6 bits so that "/ 2^26" is "take the high word" of one
+//    32x32+64 multiply-add, whose 64-bit addend carries the next coefficient (high word) and the
+//    rounding term (low word).  Rounding half away from zero on a signed product p is
+//    (p + 2^25 - [p < 0]) >> 26, and the sign of the accumulator alternates deterministically down the
+//    Horner chain (|c_k| dominates the term added to it), so [p < 0] depends on the sign of g alone;
+//  * the final division is estimated in fp32 (biased low so that the estimate is q or q - 1) and fixed
+//    by one exact remainder test, evaluated modulo 2^32 because the remainder is known to be small.
+// sigmoid and tanh are one routine: tanh uses k = 2 and the numerator 2^30 - E instead of 2^30.
 
-QL_HD float rcp_rn(float x)
+QL_HD float rcp_est(float x)            // reciprocal estimate, relative error <= 2^-22
 {
 #if defined(__CUDA_ARCH__)
-    return __frcp_rn(x);
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
 #else
     return 1.0f / x;
 #endif
@@ -167,61 +172,47 @@ QL_HD float mul_rn(float a, float b)
 #endif
 }
 
-// 2^30 * exp(-k |x|), k folded into ck = k * round(2^30 log2 e); sh = 19 - m.
-QL_HD uint32_t exp_neg_q30_fast(uint32_t a, int sh, uint32_t ck)
+template <bool TANH>
+QL_HD int32_t act_q_fast(int32_t x, int m)
 {
     const int32_t c0 = 759250125, c1 = -526272083, c2 = 182392005, c3 = -42141501,
                   c4 = 7302566, c5 = -1012351, c6 = 116951;
-    uint64_t t = ((uint64_t)a * ck + ((uint64_t)1 << (sh - 1))) >> sh;
-    uint32_t n = (uint32_t)(t >> 26);
-    int32_t g = (int32_t)((uint32_t)t & 0x3FFFFFFu) - (1 << 25);
-    int32_t sg = g >> 31;
-    const int64_t add_pos = (int64_t)((1 << 25) + sg);      // accumulator > 0: product negative iff g < 0
-    const int64_t add_neg = (int64_t)((1 << 25) + ~sg);     // accumulator < 0: product negative iff g > 0
+    const uint32_t ck = TANH ? 3098164010u : 1549082005u;         // k * round(2^30 log2 e)
+    const uint32_t a = (uint32_t)(x < 0 ? -x : x);
+    const int sh = 19 - m;
+    const uint64_t t = ((uint64_t)a * ck + ((uint64_t)1 << (sh - 1))) >> sh;
+    const uint32_t n = (uint32_t)(t >> 26);
+    const int32_t g6 = (int32_t)((((uint32_t)t & 0x3FFFFFFu) - (1u << 25)) << 6);     // 64 * g
+    const uint32_t s = (uint32_t)(g6 >> 31);                       // all ones iff g < 0
+    const uint32_t lo_pos = 0x80000000u + (s & 0xFFFFFFC0u);       // 64 * (2^25 - [g < 0]): accumulator > 0
+    const uint32_t lo_neg = 0x7FFFFFC0u - (s & 0xFFFFFFC0u);       // 64 * (2^25 - [g >= 0]): accumulator < 0
+#define QL_HORNER(acc, ck_, lo_) (int32_t)(((int64_t)(acc) * g6 + (int64_t)(((uint64_t)(uint32_t)(ck_) << 32) | (lo_))) >> 32)
     int32_t acc = c6;
-    acc = (int32_t)(((int64_t)acc * g + add_pos) >> 26) + c5;
-    acc = (int32_t)(((int64_t)acc * g + add_neg) >> 26) + c4;
-    acc = (int32_t)(((int64_t)acc * g + add_pos) >> 26) + c3;
-    acc = (int32_t)(((int64_t)acc * g + add_neg) >> 26) + c2;
-    acc = (int32_t)(((int64_t)acc * g + add_pos) >> 26) + c1;
-    acc = (int32_t)(((int64_t)acc * g + add_neg) >> 26) + c0;
-    uint32_t p = (uint32_t)acc;                              // in (2^29, 2^30 + small]
-    if (n == 0) return p;
-    if (n > 31) return 0;
-    return (p + (1u << (n - 1))) >> n;
+    acc = QL_HORNER(acc, c5, lo_pos);
+    acc = QL_HORNER(acc, c4, lo_neg);
+    acc = QL_HORNER(acc, c3, lo_pos);
+    acc = QL_HORNER(acc, c2, lo_neg);
+    acc = QL_HORNER(acc, c1, lo_pos);
+    acc = QL_HORNER(acc, c0, lo_neg);
+#undef QL_HORNER
+    const uint32_t nn = n > 31 ? 31 : n;
+    uint32_t E = ((uint32_t)acc + ((1u << nn) >> 1)) >> nn;
+    E = n > 31 ? 0u : E;
+    E = E > (1u << 30) ? (1u << 30) : E;          // only x = 0 can exceed 2^30, by a few units; same quotient
+    const uint32_t D = (1u << 30) + E;
+    const uint32_t N = TANH ? (1u << 30) - E : (1u << 30);
+    // q = floor(2^15 N / D + 1/2); the estimate is biased low by more than its error: it is q or q - 1
+    const float est = fma_rn(mul_rn((float)N, 32768.0f), rcp_est((float)D), 0.47f);
+    uint32_t q = (uint32_t)est;
+    // q + 1 is admissible iff D q + ceil(D / 2) <= 2^15 N; the difference lies in [-D, D), so mod 2^32 suffices
+    const int32_t rem = (int32_t)((N << 15) - D * q - ((D + 1u) >> 1));
+    q += rem >= 0 ? 1u : 0u;
+    const int32_t pos = q > 32767u ? 32767 : (int32_t)q;
+    return x >= 0 ? pos : (TANH ? -(int32_t)q : 32768 - (int32_t)q);
 }
 
-// largest q with d * (2q - 1) <= rhs, given an estimate within +-1
-QL_HD uint32_t fix_quotient(uint32_t q, uint32_t d, uint64_t rhs)
-{
-    if (q > 0 && (uint64_t)d * (2 * q - 1) > rhs) return q - 1;
-    if ((uint64_t)d * (2 * q + 1) <= rhs) return q + 1;
-    return q;
-}
-
-QL_HD int32_t sigmoid_q_fast(int32_t x, int m)
-{
-    uint32_t a = (uint32_t)(x < 0 ? -x : x);
-    uint32_t E = exp_neg_q30_fast(a, 19 - m, 1549082005u);
-    uint32_t D = (1u << 30) + E;
-    float r = rcp_rn((float)D);
-    uint32_t q = (uint32_t)fma_rn(35184372088832.0f, r, 0.5f);          // 2^45 / D + 1/2
-    int32_t S = (int32_t)fix_quotient(q, D, (uint64_t)1 << 46);
-    return x >= 0 ? (S > 32767 ? 32767 : S) : 32768 - S;
-}
-
-QL_HD int32_t tanh_q_fast(int32_t x, int m)
-{
-    uint32_t a = (uint32_t)(x < 0 ? -x : x);
-    uint32_t E = exp_neg_q30_fast(a, 19 - m, 3098164010u);
-    uint32_t D = (1u << 30) + E;
-    int32_t N = (1 << 30) - (int32_t)E;             // E can exceed 2^30 by a few units at x = 0: the quotient is 0 there
-    if (N <= 0) return 0;
-    float r = rcp_rn((float)D);
-    uint32_t q = (uint32_t)fma_rn(mul_rn((float)N, 32768.0f), r, 0.5f);  // 2^15 N / D + 1/2
-    int32_t T = (int32_t)fix_quotient(q, D, (uint64_t)(uint32_t)N << 16);
-    return x >= 0 ? (T > 32767 ? 32767 : T) : -T;
-}
+QL_HD int32_t sigmoid_q_fast(int32_t x, int m) { return act_q_fast<false>(x, m); }
+QL_HD int32_t tanh_q_fast(int32_t x, int m) { return act_q_fast<true>(x, m); }
 
 // ---- integer layer normalisation (Section 3.2.6) --------------------------------------------
 
@@ -251,43 +242,44 @@ QL_HD LnRow make_ln_row(LnStats s)
     LnRow r;
     r.mean = (int32_t)s.mean;                      // |mean| <= 2^25
     r.sigma = (uint32_t)s.sigma;                   // < 2^26
-    r.inv_sigma = s.sigma > 0 ? rcp_rn((float)r.sigma) : 0.0f;
+    r.inv_sigma = s.sigma > 0 ? 1.0f / (float)r.sigma : 0.0f;
     return r;
 }
 
-// q' = round(2^10 (2^10 q - mean) / sigma), exact: fp32 estimate, 64-bit remainder check, and the plain
-// division as a fallback where the estimate could be more than one off (tiny sigma against large deviations).
-QL_HD int64_t ln_quotient_fast(int32_t q, const LnRow &r)
+// q' = round(2^10 (2^10 q - mean) / sigma), exact.  Quotients below 2^16 (|z-score| < 64) take the fp32
+// estimate (biased low: q' or q' - 1) and one remainder test modulo 2^32; anything larger - a tiny sigma
+// against a large deviation - takes the plain 64-bit division.
+QL_HD int32_t ln_quotient_fast(int32_t q, const LnRow &r, int64_t *wide)
 {
-    if (r.sigma == 0) return 0;
-    int32_t d = 1024 * q - r.mean;
-    uint32_t ad = (uint32_t)(d < 0 ? -d : d);
-    uint64_t num = (uint64_t)ad * 1024u + (r.sigma >> 1);
-    float est = mul_rn(fma_rn((float)ad, 1024.0f, (float)(r.sigma >> 1)), r.inv_sigma);
-    uint64_t quo;
-    if (est < 2.0e9f) {
-        uint32_t qe = (uint32_t)est;
-        int64_t rem = (int64_t)num - (int64_t)((uint64_t)qe * r.sigma);
-        if (rem < 0) { --qe; rem += r.sigma; }
-        else if (rem >= (int64_t)r.sigma) { ++qe; rem -= r.sigma; }
-        quo = (rem < 0 || rem >= (int64_t)r.sigma) ? num / r.sigma : (uint64_t)qe;
-    } else {
-        quo = num / r.sigma;
+    const int32_t d = 1024 * q - r.mean;
+    const uint32_t ad = (uint32_t)(d < 0 ? -d : d);
+    const uint32_t half = r.sigma >> 1;
+    const float est = fma_rn(fma_rn((float)ad, 1024.0f, (float)half), r.inv_sigma, -0.05f);
+    *wide = 0;
+    if (est < 65536.0f) {
+        uint32_t qe = est > 0.0f ? (uint32_t)est : 0u;
+        const uint32_t rem = (ad << 10) + half - qe * r.sigma;     // in [0, 2 sigma), exact modulo 2^32
+        qe += (rem >= r.sigma && r.sigma != 0u) ? 1u : 0u;
+        return d < 0 ? -(int32_t)qe : (int32_t)qe;
     }
-    return d < 0 ? -(int64_t)quo : (int64_t)quo;
+    const uint64_t quo = r.sigma ? ((uint64_t)ad * 1024u + half) / r.sigma : 0u;
+    *wide = d < 0 ? -(int64_t)quo : (int64_t)quo;
+    return 0;
 }
 
 QL_HD int32_t ln_apply_fast(int32_t q, const LnRow &r, int32_t L, int32_t b, Scale eff_ln, const FastScale &f_ln)
 {
-    int64_t v = ln_quotient_fast(q, r) * (int64_t)L + (int64_t)b;
-    int32_t v32 = sat32(v);
+    int64_t wide;
+    const int32_t qp = ln_quotient_fast(q, r, &wide);
+    const int64_t v = ((int64_t)qp + wide) * (int64_t)L + (int64_t)b;
+    const int32_t v32 = sat32(v);
     return sat16(eff_ln.shift <= 0 ? fast_rescale(v32, f_ln) : mbqm(v32, eff_ln));
 }
 
 // ---- cell update and hidden state (Section 3.2.7) -------------------------------------------
 
-// x / 2^e on a 32-bit product, ties away from zero, 1 <= e <= 31
-QL_HD int32_t rdivpot32(int32_t x, int e) { return (int32_t)(((int64_t)x + ((int64_t)1 << (e - 1)) + (x >> 31)) >> e); }
+// x / 2^e for |x| <= 2^30 and 1 <= e <= 30, ties away from zero, in 32 bits
+QL_HD int32_t rdivpot32(int32_t x, int e) { return (x + (1 << (e - 1)) + (x >> 31)) >> e; }
 
 QL_HD int32_t cell_update_fast(int32_t i, int32_t z, int32_t f, int32_t c_old, int m)
 {

@@ -244,3 +244,42 @@ def test_saturating_extremes_match_oracle():
     assert_trace_equal(got[3], want[3], "extremes")
     got2 = run_gpu(w)
     check_equal(got2, want, "extremes auto")
+
+
+# ------------------------------------------------------------------ building blocks over their whole domain
+
+@pytest.mark.parametrize("m", [0, 1, 2, 3, 4, 5, 6, 9, 15])
+def test_device_activations_exhaustive(m):
+    """Every int16 input of the kernels' integer sigmoid / tanh, on the device, against the oracle."""
+    import torch
+    from paper_2101_05453_b200 import binding
+    sig = torch.zeros(65536, dtype=torch.int16, device="cuda")
+    tnh = torch.zeros(65536, dtype=torch.int16, device="cuda")
+    binding.eval_activations(m, sig, tnh, stream=torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert np.array_equal(sig.cpu().numpy().astype(np.int32), R.sigmoid_all(m))
+    assert np.array_equal(tnh.cpu().numpy().astype(np.int32), R.tanh_all(m))
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_device_layernorm_rows(seed):
+    import torch
+    from paper_2101_05453_b200 import binding
+    rng = np.random.default_rng(700 + seed)
+    n = int(rng.integers(1, 8191)) if seed else 8191
+    q = (rng.integers(-32768, 32768, n) // int(rng.integers(1, 60))).astype(np.int16)
+    if seed == 1:
+        q[:] = 123                                   # sigma = 0
+    if seed == 2:
+        q[:] = 0
+        q[n // 2] = 32767                            # one outlier: the largest z-score
+    if seed == 3:
+        q = np.where(np.arange(n) % 2 == 0, 32767, -32768).astype(np.int16)
+    L = rng.integers(-32767, 32768, n).astype(np.int16)
+    b = (rng.integers(-2 ** 31 + 1, 2 ** 31, n) // int(rng.integers(1, 3000))).astype(np.int32)
+    eff = (int(rng.integers(1 << 30, 1 << 31)), int(rng.integers(-14, 2)))
+    qd, Ld, bd = (torch.from_numpy(a).cuda() for a in (q, L, b))
+    out = torch.zeros(n, dtype=torch.int16, device="cuda")
+    binding.eval_layernorm_row(qd, n, Ld, bd, eff, out, stream=torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy(), R.layernorm_row(q, L, b, eff))
