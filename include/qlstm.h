@@ -164,6 +164,24 @@ int qlstm_eval_activations(int cell_int_bits, int16_t *sigmoid_dev, int16_t *tan
 int qlstm_eval_layernorm_row(const int16_t *q_dev, int n, const int16_t *L_dev, const int32_t *b_dev,
                              qlstm_scale_t eff_ln, int16_t *out_dev, void *cuda_stream);
 
+/*
+ * qlstm_layernorm_rows_static - the integer layer norm of qlstm_eval_layernorm_row for `rows` rows at once,
+ * for callers that must not allocate.  (The paper has no counterpart: this is a packaging of its layer norm
+ * for hosts where allocation is off limits - a per-frame real-time loop that cannot take the allocator's
+ * device-wide lock, a process whose own arena already owns all device memory, a plug-in callback in which the
+ * host forbids allocation.)
+ *   q_dev DEVICE int16 [rows][n]; L_dev int16 [n]; b_dev int32 [n]; out_dev DEVICE int16 [rows][n] (Q3.12).
+ *   rows <= 4096 (QLSTM_ERR_DIM beyond that: the scratch is a fixed 64 KiB array inside the library image, held
+ *   by every device that loads the library until the process exits); n <= 8191.
+ * It calls no cudaMalloc, cudaFree or other allocating routine.  The first call on a device looks up the
+ * array's device address (with that device current) and should therefore happen before any stream capture
+ * begins; later calls only launch two kernels on `cuda_stream`.  All calls share the one array and it keeps
+ * whatever the last call wrote: each call overwrites every entry it later reads, so no clearing is needed, but
+ * two calls that overlap on the GPU (different streams) race on it and must be serialised by the caller.
+ */
+int qlstm_layernorm_rows_static(const int16_t *q_dev, int rows, int n, const int16_t *L_dev, const int32_t *b_dev,
+                                qlstm_scale_t eff_ln, int16_t *out_dev, void *cuda_stream);
+
 /* Device properties the library sees: SM count, and resident blocks of the persistent kernel. */
 int qlstm_device_info(qlstm_t *q, int *sm_count, int *persistent_blocks);
 

@@ -21,7 +21,8 @@ IMPL_AUTO, IMPL_SIMPLE, IMPL_FAST = 0, 1, 2
 
 EXPORTS = ["qlstm_create", "qlstm_run", "qlstm_run_host", "qlstm_input_projection", "qlstm_last_status",
            "qlstm_destroy", "qlstm_strerror", "qlstm_trace_bytes", "qlstm_set_impl", "qlstm_set_profiling",
-           "qlstm_get_profile", "qlstm_device_info", "qlstm_eval_activations", "qlstm_eval_layernorm_row"]
+           "qlstm_get_profile", "qlstm_device_info", "qlstm_eval_activations", "qlstm_eval_layernorm_row",
+           "qlstm_layernorm_rows_static"]
 
 
 class Scale(C.Structure):
@@ -97,6 +98,9 @@ def lib():
         L.qlstm_eval_activations.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         L.qlstm_eval_layernorm_row.restype = C.c_int
         L.qlstm_eval_layernorm_row.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p, C.c_void_p]
+        L.qlstm_layernorm_rows_static.restype = C.c_int
+        L.qlstm_layernorm_rows_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p,
+                                                  C.c_void_p]
         _lib = L
     return _lib
 
@@ -239,6 +243,14 @@ def eval_activations(cell_int_bits: int, sigmoid_out, tanh_out, stream: int = 0)
 def eval_layernorm_row(q, n: int, L, b, eff_ln, out, stream: int = 0):
     _check(lib().qlstm_eval_layernorm_row(_dev_ptr(q), n, _dev_ptr(L), _dev_ptr(b), Scale(int(eff_ln[0]), int(eff_ln[1])),
                                           _dev_ptr(out), stream), "qlstm_eval_layernorm_row")
+
+
+def layernorm_rows_static(q, rows: int, n: int, L, b, eff_ln, out, stream: int = 0):
+    """qlstm_layernorm_rows_static: layer norm of `rows` rows using only the library's built-in scratch
+    (for callers that may not allocate device memory).  Raises QlstmError(ERR_DIM) beyond 4096 rows."""
+    _check(lib().qlstm_layernorm_rows_static(_dev_ptr(q), rows, n, _dev_ptr(L), _dev_ptr(b),
+                                             Scale(int(eff_ln[0]), int(eff_ln[1])), _dev_ptr(out), stream),
+           "qlstm_layernorm_rows_static")
 
 
 def parse_trace(buf: np.ndarray, dims: Sequence, T: int, B: int):
