@@ -22,7 +22,9 @@ struct FastScratch {
 
 struct FastLayer {
     bool proj_ok = false;        // tensor-core projection usable for this layer
-    CUtensorMap map_W;           // W [N][I] int8, K-major, 128B swizzle
+    CUtensorMap map_W;           // W [N][I] int8, K-major, 128B swizzle, box = one k-block of the resident panel
+    int proj_bn = 0;             // panel width (rows of W resident in shared memory)
+    int proj_stages = 0;         // depth of the x ring
     // persistent recurrent kernel plan
     bool rec_ok = false;
     int grid = 0;                // CTAs of the cooperative launch (one per SM)

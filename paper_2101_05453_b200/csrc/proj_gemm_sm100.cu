@@ -7,12 +7,18 @@
 // accumulators would double the HBM traffic of a kernel whose output already costs as much time
 // as its math (K is only 512-1024).
 //
+// With K this small a 128 x 256 output tile needs 240 KB of operands for 42 MOP: streaming both
+// operands per tile is bound by L2 -> SM bandwidth, not by the tensor cores.  So the weight panel
+// (BN rows of W, all of K) stays resident in shared memory while the CTA walks down the M tiles of
+// that panel; only the x tile (128 x K bytes) is streamed per output tile.
+//
 // One persistent CTA per SM, warp specialised:
-//   warp 0      TMA producer: x tile [128 x 128 B] and W tile [256 x 128 B] per k-block, 4-stage ring
-//   warp 1      MMA issuer:   4 x (M128 N256 K32) per k-block into one of two 256-column TMEM buffers
-//   warps 2..9  epilogue:     tcgen05.ld -> + folded bias -> fixed-point rescale -> sat16 -> 16-byte stores,
-//                             overlapping the next tile's MMAs through the second TMEM buffer
-// No cluster launch and no multicast.
+//   warp 0       TMA producer: W panel [BN x K] once per panel; x k-blocks [128 x 128 B] through a ring
+//   warp 1       MMA issuer:   4 x (M128 N=BN K32) per k-block into one of two TMEM accumulators
+//   warps 2..17  epilogue:     tcgen05.ld -> + folded bias -> fixed-point rescale -> sat16 -> stores,
+//                              overlapping the next tile's MMAs through the second TMEM accumulator
+// Tiles are numbered panel-major and split into equal contiguous ranges, so a CTA touches at most two
+// panels.  No cluster launch and no multicast.
 #include "fast_kernels.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
@@ -21,24 +27,26 @@ namespace ql {
 
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 128, STAGES = 4, EPI_WARPS = 8;
-constexpr int A_BYTES = BM * BK, B_BYTES = BN * BK, STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int BM = 128, BK = 128, MAX_STAGES = 6, EPI_WARPS = 16;
+constexpr int A_BYTES = BM * BK;
 constexpr int THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
-constexpr size_t SMEM_BYTES = 1024 /*align slack*/ + (size_t)STAGES * STAGE_BYTES + EPI_WARPS * 128 * sizeof(int32_t) + 256;
+constexpr int W_BYTES_MAX = 160 * 1024;           // resident weight panel
+constexpr int BIAS_PER_WARP = 64;                 // two 32-column chunks per epilogue warp
 
 struct ProjParams {
     int M, N, K, G;
+    int bn, kb, stages;          // panel width (multiple of 32), 128-byte k-blocks, ring depth
     const int32_t *bx;
     int16_t *out;
     FastScale fs[4];
     Scale sc[4];
-    int generic;        // some gate has a positive shift: use the generic rescale
+    int generic;                 // some gate has a positive shift: use the generic rescale
     int *status;
 };
 
 struct SharedCtl {
-    uint64_t full[STAGES], empty[STAGES], tmem_full[2], tmem_empty[2];
+    uint64_t a_full[MAX_STAGES], a_empty[MAX_STAGES], w_full, w_free, tmem_full[2], tmem_empty[2];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -61,26 +69,23 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], const in
     uint32_t packed[16];
     const int phase = n_first % G;
 #pragma unroll
-    for (int j = 0; j < 32; j += 2) {
-        int32_t v0 = (int32_t)r[j] + bias[j], v1 = (int32_t)r[j + 1] + bias[j + 1];
-        int g0, g1;
-        if (G == 4) { g0 = j & 3; g1 = (j + 1) & 3; }
-        else { g0 = (phase + j) % 3; g1 = (phase + j + 1) % 3; }
-        int32_t y0, y1;
-        if (p.generic) { y0 = mbqm(v0, p.sc[g0]); y1 = mbqm(v1, p.sc[g1]); }
-        else { y0 = fast_rescale(v0, p.fs[g0]); y1 = fast_rescale(v1, p.fs[g1]); }
-        packed[j >> 1] = ptx::pack_sat_s16(y0, y1);
-    }
-    if (n_valid >= 32) {
+    for (int j = 0; j < 32; j += 4) {
+        const int4 b4 = *reinterpret_cast<const int4 *>(bias + j);
+        const int32_t bb[4] = {b4.x, b4.y, b4.z, b4.w};
+        int32_t y[4];
 #pragma unroll
-        for (int v = 0; v < 4; ++v)
+        for (int i = 0; i < 4; ++i) {
+            const int32_t v = (int32_t)r[j + i] + bb[i];          // |acc| + |bias| < 2^30: no overflow
+            const int g = (G == 4) ? i : (phase + j + i) % 3;
+            y[i] = p.generic ? mbqm(v, p.sc[g]) : fast_rescale(v, p.fs[g]);
+        }
+        packed[j >> 1] = ptx::pack_sat_s16(y[0], y[1]);
+        packed[(j >> 1) + 1] = ptx::pack_sat_s16(y[2], y[3]);
+    }
+#pragma unroll
+    for (int v = 0; v < 4; ++v)
+        if (8 * v + 8 <= n_valid)
             *reinterpret_cast<uint4 *>(dst + 8 * v) = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-    } else {
-#pragma unroll
-        for (int v = 0; v < 4; ++v)
-            if (8 * v + 8 <= n_valid)
-                *reinterpret_cast<uint4 *>(dst + 8 * v) = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
-    }
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
@@ -88,17 +93,24 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint8_t *tiles = smem;
-    int32_t *bias_s = (int32_t *)(smem + (size_t)STAGES * STAGE_BYTES);
-    SharedCtl *ctl = (SharedCtl *)(bias_s + EPI_WARPS * 128);
+    const int w_block = p.bn * BK;                                   // bytes of one k-block of the panel
+    uint8_t *W_s = smem;
+    uint8_t *ring = W_s + (size_t)p.kb * w_block;
+    int32_t *bias_s = (int32_t *)(ring + (size_t)p.stages * A_BYTES);
+    SharedCtl *ctl = (SharedCtl *)(bias_s + EPI_WARPS * BIAS_PER_WARP);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + BN - 1) / BN;
-    const int n_tiles = tiles_m * tiles_n, k_blocks = (p.K + BK - 1) / BK;
+    const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + p.bn - 1) / p.bn;
+    const int n_tiles = tiles_m * tiles_n;
+    const int per_cta = (n_tiles + gridDim.x - 1) / gridDim.x;
+    const int t_begin = blockIdx.x * per_cta;
+    const int t_end = (t_begin + per_cta < n_tiles) ? t_begin + per_cta : n_tiles;
     volatile int *abort_flag = &ctl->abort_flag;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(&ctl->full[s], 1); ptx::mbar_init(&ctl->empty[s], 1); }
+        for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&ctl->a_full[s], 1); ptx::mbar_init(&ctl->a_empty[s], 1); }
+        ptx::mbar_init(&ctl->w_full, 1);
+        ptx::mbar_init(&ctl->w_free, 1);
         for (int b = 0; b < 2; ++b) { ptx::mbar_init(&ctl->tmem_full[b], 1); ptx::mbar_init(&ctl->tmem_empty[b], EPI_WARPS); }
         ctl->abort_flag = 0;
         ptx::fence_barrier_init();
@@ -117,16 +129,25 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
-            int stage = 0; uint32_t phase = 0;
-            for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x) {
-                const int m0 = (t / tiles_n) * BM, n0 = (t % tiles_n) * BN;
-                for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!wait_or_abort(&ctl->empty[stage], phase ^ 1, abort_flag)) break;
-                    uint8_t *a = tiles + (size_t)stage * STAGE_BYTES, *b = a + A_BYTES;
-                    ptx::mbar_arrive_expect_tx(&ctl->full[stage], STAGE_BYTES);
-                    ptx::tma_load_2d(a, &map_x, &ctl->full[stage], kb * BK, m0);
-                    ptx::tma_load_2d(b, &map_w, &ctl->full[stage], kb * BK, n0);
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+            int stage = 0; uint32_t phase = 0, wfree_par = 0;
+            int cur_n = -1;
+            for (int t = t_begin; t < t_end && !*abort_flag; ++t) {
+                const int n_tile = t / tiles_m, m0 = (t % tiles_m) * BM;
+                if (n_tile != cur_n) {
+                    if (cur_n >= 0) {                                  // all MMAs that read the old panel are done
+                        if (!wait_or_abort(&ctl->w_free, wfree_par, abort_flag)) break;
+                        wfree_par ^= 1;
+                    }
+                    ptx::mbar_arrive_expect_tx(&ctl->w_full, (uint32_t)(p.kb * w_block));
+                    for (int kb = 0; kb < p.kb; ++kb)
+                        ptx::tma_load_2d(W_s + (size_t)kb * w_block, &map_w, &ctl->w_full, kb * BK, n_tile * p.bn);
+                    cur_n = n_tile;
+                }
+                for (int kb = 0; kb < p.kb; ++kb) {
+                    if (!wait_or_abort(&ctl->a_empty[stage], phase ^ 1, abort_flag)) break;
+                    ptx::mbar_arrive_expect_tx(&ctl->a_full[stage], A_BYTES);
+                    ptx::tma_load_2d(ring + (size_t)stage * A_BYTES, &map_x, &ctl->a_full[stage], kb * BK, m0);
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
             }
         }
@@ -134,29 +155,36 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            constexpr uint32_t IDESC = ptx::idesc_i8(BM, BN);
-            int stage = 0; uint32_t phase = 0;
-            int it = 0;
-            for (int t = blockIdx.x; t < n_tiles && !*abort_flag; t += gridDim.x, ++it) {
+            const uint32_t idesc = ptx::idesc_i8(BM, p.bn);
+            int stage = 0; uint32_t phase = 0, wfull_par = 0;
+            int cur_n = -1, it = 0;
+            for (int t = t_begin; t < t_end && !*abort_flag; ++t, ++it) {
+                const int n_tile = t / tiles_m;
+                if (n_tile != cur_n) {
+                    if (!wait_or_abort(&ctl->w_full, wfull_par, abort_flag)) break;
+                    wfull_par ^= 1;
+                    cur_n = n_tile;
+                }
                 const int buf = it & 1;
                 const uint32_t acc_phase = (uint32_t)(it >> 1) & 1;
                 if (!wait_or_abort(&ctl->tmem_empty[buf], acc_phase ^ 1, abort_flag)) break;
                 ptx::tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)buf * BN;
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * p.bn);
                 bool ok = true;
-                for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!wait_or_abort(&ctl->full[stage], phase, abort_flag)) { ok = false; break; }
+                for (int kb = 0; kb < p.kb; ++kb) {
+                    if (!wait_or_abort(&ctl->a_full[stage], phase, abort_flag)) { ok = false; break; }
                     ptx::tc_fence_after();
-                    const uint32_t a_addr = ptx::smem_u32(tiles + (size_t)stage * STAGE_BYTES), b_addr = a_addr + A_BYTES;
-                    const uint64_t a_desc = ptx::smem_desc_k_sw128(a_addr), b_desc = ptx::smem_desc_k_sw128(b_addr);
+                    const uint64_t a_desc = ptx::smem_desc_k_sw128(ptx::smem_u32(ring + (size_t)stage * A_BYTES));
+                    const uint64_t b_desc = ptx::smem_desc_k_sw128(ptx::smem_u32(W_s + (size_t)kb * w_block));
 #pragma unroll
                     for (int k = 0; k < BK / 32; ++k)     // 32 int8 = 32 bytes = 2 descriptor units along K
-                        ptx::mma_i8_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, IDESC, (kb | k) != 0);
-                    ptx::mma_commit(&ctl->empty[stage]);  // frees the smem stage once these MMAs are done
-                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                        ptx::mma_i8_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+                    ptx::mma_commit(&ctl->a_empty[stage]);  // frees the ring stage once these MMAs are done
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
                 if (!ok) break;
                 ptx::mma_commit(&ctl->tmem_full[buf]);
+                if (t + 1 < t_end && (t + 1) / tiles_m != cur_n) ptx::mma_commit(&ctl->w_free);
             }
         }
         __syncwarp();
@@ -164,36 +192,48 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
         // ---------------- epilogue ----------------
         const int e = warp - 2;
         const int quarter = warp & 3;                    // TMEM lanes this warp may read: 32 * (warp % 4)
-        const int half = e >> 2;                         // which 128 of the 256 columns
-        int32_t *bias = bias_s + e * 128;                // this warp's 128 folded biases of the current tile
+        const int cgrp = e >> 2;                         // this warp takes 32-column chunks cgrp and cgrp + 4
+        int32_t *bias = bias_s + e * BIAS_PER_WARP;
+        const int n_chunks = p.bn >> 5;
+        const int c0 = cgrp, c1 = cgrp + 4;
+        const bool has0 = c0 < n_chunks, has1 = c1 < n_chunks;
         int it = 0;
-        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++it) {
+        for (int t = t_begin; t < t_end; ++t, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1;
-            const int m0 = (t / tiles_n) * BM, n0 = (t % tiles_n) * BN;
+            const int n0 = (t / tiles_m) * p.bn, m0 = (t % tiles_m) * BM;
             __syncwarp();
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int n = n0 + half * 128 + i * 32 + lane;
-                bias[i * 32 + lane] = n < p.N ? p.bx[n] : 0;
+            {
+                const int na = n0 + c0 * 32 + lane, nb = n0 + c1 * 32 + lane;
+                bias[lane] = (has0 && na < p.N) ? p.bx[na] : 0;
+                bias[32 + lane] = (has1 && nb < p.N) ? p.bx[nb] : 0;
             }
             __syncwarp();
             if (!__all_sync(0xffffffffu, wait_or_abort(&ctl->tmem_full[buf], acc_phase, abort_flag))) break;
             ptx::tc_fence_after();
             const int row = m0 + quarter * 32 + lane;
-#pragma unroll 1
-            for (int ch = 0; ch < 4; ++ch) {
-                const int col = half * 128 + ch * 32, cw = ch * 32;
-                uint32_t r[32];
-                __syncwarp();             // the TMEM load is warp-collective: reconverge after the per-row branch
-                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * BN + col), r);
-                ptx::tmem_ld_wait();
-                const int n_first = n0 + col;
-                int n_valid = p.N - n_first;
+            const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.bn);
+            // the second chunk's TMEM load is in flight while the first chunk is processed
+            uint32_t r0[32], r1[32];
+            if (has0) ptx::tmem_ld_32x32(tbase + (uint32_t)(c0 * 32), r0);
+            ptx::tmem_ld_wait();
+            if (has1) ptx::tmem_ld_32x32(tbase + (uint32_t)(c1 * 32), r1);
+            if (has0) {
+                const int n_first = n0 + c0 * 32, n_valid = p.N - n_first;
                 if (row < p.M && n_valid > 0) {
                     int16_t *dst = p.out + (size_t)row * p.N + n_first;
-                    if (p.G == 4) epilogue_chunk<4>(r, bias + cw, p, n_first, dst, n_valid);
-                    else epilogue_chunk<3>(r, bias + cw, p, n_first, dst, n_valid);
+                    if (p.G == 4) epilogue_chunk<4>(r0, bias, p, n_first, dst, n_valid);
+                    else epilogue_chunk<3>(r0, bias, p, n_first, dst, n_valid);
+                }
+            }
+            __syncwarp();
+            ptx::tmem_ld_wait();
+            if (has1) {
+                const int n_first = n0 + c1 * 32, n_valid = p.N - n_first;
+                if (row < p.M && n_valid > 0) {
+                    int16_t *dst = p.out + (size_t)row * p.N + n_first;
+                    if (p.G == 4) epilogue_chunk<4>(r1, bias + 32, p, n_first, dst, n_valid);
+                    else epilogue_chunk<3>(r1, bias + 32, p, n_first, dst, n_valid);
                 }
             }
             ptx::tc_fence_before();
@@ -216,6 +256,19 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
     }
 }
 
+int panel_width(int K)
+{
+    const int kb = (K + BK - 1) / BK;
+    int bn = (W_BYTES_MAX / (kb * BK)) / 32 * 32;
+    return bn > 256 ? 256 : bn;
+}
+
+size_t smem_bytes(int bn, int kb, int stages)
+{
+    return 1024 + (size_t)kb * bn * BK + (size_t)stages * A_BYTES + EPI_WARPS * BIAS_PER_WARP * sizeof(int32_t) +
+           sizeof(SharedCtl) + 64;
+}
+
 }  // namespace
 
 bool fast_projection_supported(const FastLayer &f, const LayerParams &p)
@@ -227,13 +280,19 @@ int fast_projection_init(FastLayer &f, const LayerParams &p)
 {
     f.proj_ok = false;
     if (p.I % 16 != 0 || p.N % 8 != 0) return 0;
-    if (!make_tensor_map_i8(&f.map_W, p.W, (uint64_t)p.N, (uint64_t)p.I, BN, BK)) return 0;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(k_projection_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess)
-            return 0;
-        attr_set = true;
-    }
+    const int bn = panel_width(p.I);
+    if (bn < 32) return 0;                                   // K too large for a resident panel
+    const int kb = (p.I + BK - 1) / BK;
+    int dev = 0, max_smem = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    int stages = MAX_STAGES;
+    while (stages >= 2 && smem_bytes(bn, kb, stages) > (size_t)max_smem) --stages;
+    if (stages < 2) return 0;
+    f.proj_bn = bn;
+    f.proj_stages = stages;
+    if (!make_tensor_map_i8(&f.map_W, p.W, (uint64_t)p.N, (uint64_t)p.I, (uint32_t)bn, BK)) return 0;
+    if (cudaFuncSetAttribute(k_projection_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess) return 0;
     f.proj_ok = true;
     return 0;
 }
@@ -245,18 +304,17 @@ cudaError_t launch_projection_fast(const FastLayer &f, const LayerParams &p, con
     if (!make_tensor_map_i8(&map_x, x, (uint64_t)rows, (uint64_t)p.I, BM, BK)) return cudaErrorInvalidValue;
     ProjParams pp;
     pp.M = rows; pp.N = p.N; pp.K = p.I; pp.G = p.G;
+    pp.bn = f.proj_bn; pp.kb = (p.I + BK - 1) / BK; pp.stages = f.proj_stages;
     pp.bx = p.bx; pp.out = X; pp.status = status; pp.generic = 0;
     for (int g = 0; g < 4; ++g) {
         Scale s = g < p.G ? p.eff_x[g] : Scale{0, 0};
         pp.sc[g] = s;
         if (s.shift > 0) pp.generic = 1;
-        int R = s.shift < 0 ? -s.shift : 0;
         pp.fs[g] = make_fast_scale(s);
-        (void)R;
     }
-    const int tiles = ((rows + BM - 1) / BM) * ((p.N + BN - 1) / BN);
+    const int tiles = ((rows + BM - 1) / BM) * ((p.N + pp.bn - 1) / pp.bn);
     const int grid = tiles < sm_count ? tiles : sm_count;
-    k_projection_sm100<<<grid, THREADS, SMEM_BYTES, st>>>(map_x, f.map_W, pp);
+    k_projection_sm100<<<grid, THREADS, smem_bytes(pp.bn, pp.kb, pp.stages), st>>>(map_x, f.map_W, pp);
     return cudaGetLastError();
 }
 
