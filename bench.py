@@ -279,7 +279,7 @@ def main():
                 "peak_source": f"2 x bf16 sustained, {peaks['source']}", "ms_per_launch": rec_ms / n_l,
                 "us_per_layer_step": 1e3 * rec_ms / (n_l * T),
                 "phase_us_per_layer_step": {k: 1e3 * prof[k] / (max(args.steps, 1) * n_l * T) for k in
-                                            ("phase_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms", "phase_c_ms", "wait_c_ms")}}
+                                            ("phase_a_ms", "matmul_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms", "phase_c_ms", "wait_c_ms")}}
     dominant = roof_rec if rec_ms >= proj_ms else roof_proj
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

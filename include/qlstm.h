@@ -146,6 +146,7 @@ typedef struct {
     /* inside the persistent recurrent kernel, as seen by its first block (device timer): time spent working in
      * the matmul (a), elementwise (b) and projection (c) phases, and waiting at the grid barrier after each */
     double phase_a_ms, wait_a_ms, phase_b_ms, wait_b_ms, phase_c_ms, wait_c_ms;
+    double matmul_a_ms;   /* part of phase_a_ms before the first accumulator is ready (operand load + MMA) */
 } qlstm_profile_t;
 int qlstm_set_profiling(qlstm_t *q, int enabled);
 int qlstm_get_profile(qlstm_t *q, qlstm_profile_t *out, int reset);

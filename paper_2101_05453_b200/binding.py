@@ -47,7 +47,8 @@ class Profile(C.Structure):
                 ("recurrent_ms", C.c_double), ("recurrent_launches", C.c_int),
                 ("other_ms", C.c_double), ("other_launches", C.c_int),
                 ("phase_a_ms", C.c_double), ("wait_a_ms", C.c_double), ("phase_b_ms", C.c_double),
-                ("wait_b_ms", C.c_double), ("phase_c_ms", C.c_double), ("wait_c_ms", C.c_double)]
+                ("wait_b_ms", C.c_double), ("phase_c_ms", C.c_double), ("wait_c_ms", C.c_double),
+                ("matmul_a_ms", C.c_double)]
 
 
 class QlstmError(RuntimeError):

@@ -63,7 +63,7 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
 
 template <int G>
 __device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], const int32_t *bias, const ProjParams &p,
-                                               int n_first, int16_t *dst, int n_valid)
+                                               int n_first, int16_t *dst, int n_valid, bool wide_ok)
 {
     // column j of this chunk is global column n_first + j; its gate slot is (n_first + j) % G
     uint32_t packed[16];
@@ -81,6 +81,16 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], const in
         }
         packed[j >> 1] = ptx::pack_sat_s16(y[0], y[1]);
         packed[(j >> 1) + 1] = ptx::pack_sat_s16(y[2], y[3]);
+    }
+    if (n_valid >= 32 && wide_ok) {
+        // 32-byte stores: every store fills whole 32-byte sectors
+#pragma unroll
+        for (int v = 0; v < 2; ++v)
+            asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 16 * v),
+                         "r"(packed[8 * v]), "r"(packed[8 * v + 1]), "r"(packed[8 * v + 2]), "r"(packed[8 * v + 3]),
+                         "r"(packed[8 * v + 4]), "r"(packed[8 * v + 5]), "r"(packed[8 * v + 6]), "r"(packed[8 * v + 7])
+                         : "memory");
+        return;
     }
 #pragma unroll
     for (int v = 0; v < 4; ++v)
@@ -192,11 +202,13 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
         // ---------------- epilogue ----------------
         const int e = warp - 2;
         const int quarter = warp & 3;                    // TMEM lanes this warp may read: 32 * (warp % 4)
-        const int cgrp = e >> 2;                         // this warp takes 32-column chunks cgrp and cgrp + 4
+        const int cgrp = e >> 2;                         // this warp takes the adjacent 32-column chunks 2 cgrp, 2 cgrp + 1:
+                                                         // each thread then writes whole 128-byte lines of its row
         int32_t *bias = bias_s + e * BIAS_PER_WARP;
         const int n_chunks = p.bn >> 5;
-        const int c0 = cgrp, c1 = cgrp + 4;
+        const int c0 = 2 * cgrp, c1 = 2 * cgrp + 1;
         const bool has0 = c0 < n_chunks, has1 = c1 < n_chunks;
+        const bool wide_ok = (p.N % 16) == 0;            // every row starts on a 32-byte boundary
         int it = 0;
         for (int t = t_begin; t < t_end; ++t, ++it) {
             const int buf = it & 1;
@@ -222,8 +234,8 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
                 const int n_first = n0 + c0 * 32, n_valid = p.N - n_first;
                 if (row < p.M && n_valid > 0) {
                     int16_t *dst = p.out + (size_t)row * p.N + n_first;
-                    if (p.G == 4) epilogue_chunk<4>(r0, bias, p, n_first, dst, n_valid);
-                    else epilogue_chunk<3>(r0, bias, p, n_first, dst, n_valid);
+                    if (p.G == 4) epilogue_chunk<4>(r0, bias, p, n_first, dst, n_valid, wide_ok);
+                    else epilogue_chunk<3>(r0, bias, p, n_first, dst, n_valid, wide_ok);
                 }
             }
             __syncwarp();
@@ -232,8 +244,8 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
                 const int n_first = n0 + c1 * 32, n_valid = p.N - n_first;
                 if (row < p.M && n_valid > 0) {
                     int16_t *dst = p.out + (size_t)row * p.N + n_first;
-                    if (p.G == 4) epilogue_chunk<4>(r1, bias + 32, p, n_first, dst, n_valid);
-                    else epilogue_chunk<3>(r1, bias + 32, p, n_first, dst, n_valid);
+                    if (p.G == 4) epilogue_chunk<4>(r1, bias + 32, p, n_first, dst, n_valid, wide_ok);
+                    else epilogue_chunk<3>(r1, bias + 32, p, n_first, dst, n_valid, wide_ok);
                 }
             }
             ptx::tc_fence_before();

@@ -462,6 +462,7 @@ int qlstm_get_profile(qlstm_t *q, qlstm_profile_t *out, int reset)
     out->phase_a_ms = ns[0] * 1e-6; out->wait_a_ms = ns[1] * 1e-6;
     out->phase_b_ms = ns[2] * 1e-6; out->wait_b_ms = ns[3] * 1e-6;
     out->phase_c_ms = ns[4] * 1e-6; out->wait_c_ms = ns[5] * 1e-6;
+    out->matmul_a_ms = ns[6] * 1e-6;
     if (reset) {
         q->prof = qlstm_profile_t{};
         cudaMemset(q->phase_ns, 0, sizeof(ns));

@@ -143,33 +143,48 @@ __device__ __forceinline__ int32_t lo16(uint32_t w) { return (int32_t)(w << 16) 
 __device__ __forceinline__ int32_t hi16(uint32_t w) { return (int32_t)w >> 16; }
 __device__ __forceinline__ uint32_t pack16(int32_t lo, int32_t hi) { return ((uint32_t)lo & 0xffffu) | ((uint32_t)hi << 16); }
 
-// Phase A epilogue for one thread = one batch row: the gate sums of this CTA's cells, 8 columns at a time.
+// Phase A epilogue for one thread = one batch row and a range of 8-column groups of this CTA's gate sums.
 //   out = sat16( X + sat16(rescale(sat32(acc + bh), eff_h)) )            (no peephole: final gate sum, int16)
 //   out = X + sat16(rescale(...))                                        (peephole: int32, finished in phase B)
+// The X values do not depend on the recurrence: the first groups are fetched before the accumulator is awaited.
+constexpr int XPRE = 4;
+
+__device__ __forceinline__ void phase_a_prefetch(const RecParams &p, int b, int t, int n0, int g_begin, int g_end,
+                                                 bool row_valid, uint4 (&xv)[XPRE])
+{
+    const int16_t *xrow = p.X + ((size_t)t * p.B + b) * p.N + n0;
+#pragma unroll
+    for (int i = 0; i < XPRE; ++i)
+        xv[i] = (row_valid && g_begin + i < g_end) ? __ldg(reinterpret_cast<const uint4 *>(xrow + 8 * (g_begin + i)))
+                                                    : make_uint4(0, 0, 0, 0);
+}
+
 template <int G>
-__device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, int b, int t, int n0, int n_cnt,
-                                            const int32_t *bh_s, bool row_valid)
+__device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, int b, int t, int n0, int g_begin,
+                                            int g_end, const int32_t *bh_s, bool row_valid, const uint4 (&xv)[XPRE])
 {
     const bool peep = (p.flags & F_PEEPHOLE) != 0;
     const int16_t *xrow = p.X + ((size_t)t * p.B + b) * p.N + n0;
-    for (int col = 0; col < n_cnt; col += 16) {
-        uint32_t r[16];
-        __syncwarp();                 // the TMEM load is warp-collective: reconverge after the per-row branch
-        ptx::tmem_ld_32x16(taddr + (uint32_t)col, r);
-        ptx::tmem_ld_wait();
-        if (!row_valid) continue;
+#pragma unroll 1
+    for (int gbase = g_begin; gbase < g_end; gbase += XPRE) {
 #pragma unroll
-        for (int h8 = 0; h8 < 2; ++h8) {
-            const int c8 = col + 8 * h8;
-            if (c8 >= n_cnt) break;                      // n_cnt is a multiple of 8
-            const uint4 xv = __ldg(reinterpret_cast<const uint4 *>(xrow + c8));
-            const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+        for (int i = 0; i < XPRE; ++i) {
+            const int grp = gbase + i;
+            if (grp >= g_end) break;                         // warp-uniform
+            const int c8 = grp * 8;
+            uint32_t r[8];
+            __syncwarp();                                    // the TMEM load is warp-collective
+            ptx::tmem_ld_32x8(taddr + (uint32_t)c8, r);
+            ptx::tmem_ld_wait();
+            if (!row_valid) continue;
+            const uint4 x4 = (gbase == g_begin) ? xv[i] : __ldg(reinterpret_cast<const uint4 *>(xrow + c8));
+            const uint32_t xw[4] = {x4.x, x4.y, x4.z, x4.w};
             const int ph = (G == 4) ? 0 : c8 % 3;
             int32_t o[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int gi = (G == 4) ? (j & 3) : (ph + j) % 3;
-                const int32_t acc = add_sat((int32_t)r[8 * h8 + j], bh_s[c8 + j]);
+                const int32_t acc = add_sat((int32_t)r[j], bh_s[c8 + j]);
                 const int32_t H = sat16(rescale_sel(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
                 const int32_t X = (j & 1) ? hi16(xw[j >> 1]) : lo16(xw[j >> 1]);
                 o[j] = peep ? X + H : sat16(X + H);
@@ -572,17 +587,24 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
                     }
                 }
                 __syncwarp();
-            } else if (warp < 10) {
-                const int e = warp - 2, quarter = warp & 3, mi = e >> 2;
-                if (mi < p.MT) {
-                    if (__all_sync(0xffffffffu, wait_or_abort(&ctl->acc_full[mi], par, abort_flag))) {
-                        ptx::tc_fence_after();
-                        const int b = mi * 128 + quarter * 32 + lane;
-                        const uint32_t ta = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * p.nc_pad);
-                        if (p.G == 4) phase_a_row<4>(p, ta, b, t, n0, n_cnt, bh_s, b < p.B);
-                        else phase_a_row<3>(p, ta, b, t, n0, n_cnt, bh_s, b < p.B);
-                        ptx::tc_fence_before();
-                    }
+            } else if (warp < 18) {
+                // 16 epilogue warps: 4 TMEM lane quarters x (batch tile, column part)
+                const int e = warp - 2, quarter = warp & 3, slot = e >> 2;
+                const int mi = slot % p.MT, part = slot / p.MT, nparts = 4 / p.MT;
+                const int ngroups = n_cnt >> 3;
+                const int g_begin = part * ngroups / nparts, g_end = (part + 1) * ngroups / nparts;
+                const int b = mi * 128 + quarter * 32 + lane;
+                uint4 xv[XPRE];
+                const bool probe = p.phase_ns != nullptr && cta == 0 && warp == 2 && lane == 0;
+                const unsigned long long t_in = probe ? globaltimer() : 0ull;
+                phase_a_prefetch(p, b, t, n0, g_begin, g_end, b < p.B, xv);
+                if (__all_sync(0xffffffffu, wait_or_abort(&ctl->acc_full[mi], par, abort_flag))) {
+                    if (probe) p.phase_ns[6] += globaltimer() - t_in;      // operand load + matmul latency
+                    ptx::tc_fence_after();
+                    const uint32_t ta = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * p.nc_pad);
+                    if (p.G == 4) phase_a_row<4>(p, ta, b, t, n0, g_begin, g_end, bh_s, b < p.B, xv);
+                    else phase_a_row<3>(p, ta, b, t, n0, g_begin, g_end, bh_s, b < p.B, xv);
+                    ptx::tc_fence_before();
                 }
             }
         }
