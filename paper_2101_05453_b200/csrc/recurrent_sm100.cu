@@ -95,8 +95,10 @@ __device__ __forceinline__ unsigned long long globaltimer()
 }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// Grid-wide barrier on a monotonic counter.  Global writes made before it by any thread of any CTA are
-// visible after it to every thread and to TMA loads (async proxy) of every CTA.
+// Grid-wide barrier on a monotonic counter: every thread's earlier global writes are ordered before the
+// CTA barrier, thread 0 then publishes them with a release-add and polls with acquire loads.  The proxy
+// fence before it makes those generic-proxy writes visible to other CTAs' TMA loads (async proxy); the
+// thread that issues TMA loads fences again on its side after the barrier.
 __device__ __forceinline__ void grid_sync(const RecParams &p, unsigned &epoch, volatile int *abort_flag)
 {
     fence_proxy_async_all();
@@ -104,23 +106,22 @@ __device__ __forceinline__ void grid_sync(const RecParams &p, unsigned &epoch, v
     if (threadIdx.x == 0) {
         ++epoch;
         const unsigned target = epoch * gridDim.x;
-        __threadfence();
-        atomicAdd(p.bar, 1u);
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.bar) : "memory");
         const unsigned long long t0 = globaltimer();
         unsigned spins = 0;
         while (ld_acquire(p.bar) < target) {
-            if (ld_acquire(p.bar + 1) != 0u) { *abort_flag = 1; break; }
-            if ((++spins & 1023u) == 0u && globaltimer() - t0 > SPIN_LIMIT_NS) {
-                atomicExch(p.bar + 1, 1u);
-                *abort_flag = 1;
-                break;
+            if ((++spins & 63u) == 0u) {
+                if (ld_acquire(p.bar + 1) != 0u) { *abort_flag = 1; break; }
+                if (globaltimer() - t0 > SPIN_LIMIT_NS) {
+                    atomicExch(p.bar + 1, 1u);
+                    *abort_flag = 1;
+                    break;
+                }
             }
         }
         if (*abort_flag) atomicExch(p.bar + 1, 1u);
-        __threadfence();
     }
     __syncthreads();
-    fence_proxy_async_all();
 }
 
 __device__ __forceinline__ int32_t rescale_sel(int32_t x, const Scale &s, const FastScale &f, int fast_ok)
@@ -147,7 +148,7 @@ __device__ __forceinline__ uint32_t pack16(int32_t lo, int32_t hi) { return ((ui
 //   out = sat16( X + sat16(rescale(sat32(acc + bh), eff_h)) )            (no peephole: final gate sum, int16)
 //   out = X + sat16(rescale(...))                                        (peephole: int32, finished in phase B)
 // The X values do not depend on the recurrence: the first groups are fetched before the accumulator is awaited.
-constexpr int XPRE = 4;
+constexpr int XPRE = 2;
 
 __device__ __forceinline__ void phase_a_prefetch(const RecParams &p, int b, int t, int n0, int g_begin, int g_end,
                                                  bool row_valid, uint4 (&xv)[XPRE])
@@ -165,26 +166,41 @@ __device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, 
 {
     const bool peep = (p.flags & F_PEEPHOLE) != 0;
     const int16_t *xrow = p.X + ((size_t)t * p.B + b) * p.N + n0;
+    uint4 xn[XPRE];
+#pragma unroll
+    for (int i = 0; i < XPRE; ++i) xn[i] = xv[i];
 #pragma unroll 1
     for (int gbase = g_begin; gbase < g_end; gbase += XPRE) {
+        // X of the next batch of groups is requested before this batch is processed
+        uint4 xc[XPRE];
+#pragma unroll
+        for (int i = 0; i < XPRE; ++i) {
+            xc[i] = xn[i];
+            if (row_valid && gbase + XPRE + i < g_end) xn[i] = __ldg(reinterpret_cast<const uint4 *>(xrow + 8 * (gbase + XPRE + i)));
+        }
+        // all TMEM loads of this batch first, one wait, then the arithmetic
+        uint32_t r[XPRE][8];
+        __syncwarp();                                        // the TMEM loads are warp-collective
+#pragma unroll
+        for (int i = 0; i < XPRE; ++i)
+            if (gbase + i < g_end) ptx::tmem_ld_32x8(taddr + (uint32_t)((gbase + i) * 8), r[i]);   // warp-uniform
+        ptx::tmem_ld_wait();
+        if (!row_valid) continue;
 #pragma unroll
         for (int i = 0; i < XPRE; ++i) {
             const int grp = gbase + i;
-            if (grp >= g_end) break;                         // warp-uniform
+            if (grp >= g_end) break;
             const int c8 = grp * 8;
-            uint32_t r[8];
-            __syncwarp();                                    // the TMEM load is warp-collective
-            ptx::tmem_ld_32x8(taddr + (uint32_t)c8, r);
-            ptx::tmem_ld_wait();
-            if (!row_valid) continue;
-            const uint4 x4 = (gbase == g_begin) ? xv[i] : __ldg(reinterpret_cast<const uint4 *>(xrow + c8));
+            const uint4 x4 = xc[i];
             const uint32_t xw[4] = {x4.x, x4.y, x4.z, x4.w};
+            const int4 b0 = *reinterpret_cast<const int4 *>(bh_s + c8), b1 = *reinterpret_cast<const int4 *>(bh_s + c8 + 4);
+            const int32_t bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
             const int ph = (G == 4) ? 0 : c8 % 3;
             int32_t o[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const int gi = (G == 4) ? (j & 3) : (ph + j) % 3;
-                const int32_t acc = add_sat((int32_t)r[j], bh_s[c8 + j]);
+                const int32_t acc = add_sat((int32_t)r[i][j], bb[j]);
                 const int32_t H = sat16(rescale_sel(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
                 const int32_t X = (j & 1) ? hi16(xw[j >> 1]) : lo16(xw[j >> 1]);
                 o[j] = peep ? X + H : sat16(X + H);
@@ -228,10 +244,9 @@ __device__ __forceinline__ void phase_c_row(const RecParams &p, uint32_t taddr, 
 // ------------------------------------------------------------------------------------------------
 // Phase B: elementwise work on a contiguous range of the B x C cell grid.
 
-// Block-wide reduction of per-gate sum / sum of squares into ctl->ln_rows[slot][*].
+// Warp-level part of the statistics reduction: per-gate sum / sum of squares of this warp into shared memory.
 template <int G>
-__device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, const long long (&sum)[4], const long long (&sq)[4], int n,
-                                                   int slot)
+__device__ __forceinline__ void warp_reduce_stats(RecCtl *ctl, const long long (&sum)[4], const long long (&sq)[4])
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 #pragma unroll
@@ -243,6 +258,14 @@ __device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, const long long 
         }
         if (lane == 0) { ctl->red_sum[warp][g] = a; ctl->red_sq[warp][g] = b; }
     }
+}
+
+// Block-wide reduction (all warps contribute to one row) into ctl->ln_rows[slot][*].
+template <int G>
+__device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, const long long (&sum)[4], const long long (&sq)[4], int n,
+                                                   int slot)
+{
+    warp_reduce_stats<G>(ctl, sum, sq);
     __syncthreads();
     if (threadIdx.x < G) {
         long long a = 0, b = 0;
@@ -352,10 +375,16 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, in
     for (int rb = b_first; rb <= b_last; rb += MAX_LN_ROWS) {
         const int re = (rb + MAX_LN_ROWS - 1 < b_last) ? rb + MAX_LN_ROWS - 1 : b_last;
         if (LN) {
-            for (int r = rb; r <= re; ++r) {
-                const int16_t *row = (const int16_t *)p.pre + (size_t)r * p.N;
-                long long sum[4] = {0, 0, 0, 0}, sq[4] = {0, 0, 0, 0};
-                for (int u = 2 * threadIdx.x; u < p.C; u += 2 * RTHREADS) {
+            // statistics of all rows of this batch at once: the warps are split evenly over the rows
+            const int nrows = re - rb + 1;
+            const int wpr = (RTHREADS / 32) / nrows;                       // warps per row
+            const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+            const int r = warp / wpr;
+            long long sum[4] = {0, 0, 0, 0}, sq[4] = {0, 0, 0, 0};
+            if (r < nrows) {
+                const int16_t *row = (const int16_t *)p.pre + (size_t)(rb + r) * p.N;
+                const int tig = (warp - r * wpr) * 32 + lane, gs = wpr * 32;
+                for (int u = 2 * tig; u < p.C; u += 2 * gs) {
                     int32_t v[2][4];
                     load_pair_i16<G>(row + (size_t)u * G, false, v);
 #pragma unroll
@@ -364,8 +393,16 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, in
                         sq[g] += (long long)(v[0][g] * v[0][g]) + (long long)(v[1][g] * v[1][g]);
                     }
                 }
-                block_reduce_stats<G>(ctl, sum, sq, p.C, r - rb);
             }
+            warp_reduce_stats<G>(ctl, sum, sq);
+            __syncthreads();
+            if (threadIdx.x < nrows * 4 && (threadIdx.x & 3) < G) {
+                const int rr = threadIdx.x >> 2, g = threadIdx.x & 3;
+                long long a = 0, b = 0;
+                for (int w = rr * wpr; w < (rr + 1) * wpr; ++w) { a += ctl->red_sum[w][g]; b += ctl->red_sq[w][g]; }
+                ctl->ln_rows[rr][g] = make_ln_row(ln_stats(a, b, p.C));
+            }
+            __syncthreads();
         }
         const int j0 = i0 > rb * p.C ? i0 : rb * p.C;
         const int j1 = i1 < (re + 1) * p.C ? i1 : (re + 1) * p.C;
@@ -555,6 +592,7 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
         if (has_cells) {
             if (warp == 0) {
                 if (lane == 0) {
+                    fence_proxy_async_all();
                     for (int mi = 0; mi < p.MT && !*abort_flag; ++mi)
                         for (int kb = 0; kb < p.kb_h; ++kb) {
                             if (!wait_or_abort(&ctl->empty[stage], ring_phase ^ 1, abort_flag)) break;
@@ -627,6 +665,7 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
             if (has_ptile) {
                 if (warp == 0) {
                     if (lane == 0) {
+                        fence_proxy_async_all();
                         for (int kb = 0; kb < p.kb_c; ++kb) {
                             if (!wait_or_abort(&ctl->empty[stage], ring_phase ^ 1, abort_flag)) break;
                             ptx::mbar_arrive_expect_tx(&ctl->full[stage], A_STAGE_BYTES);
