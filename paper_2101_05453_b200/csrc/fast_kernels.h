@@ -53,7 +53,7 @@ cudaError_t launch_projection_fast(const FastLayer &f, const LayerParams &p, con
 bool fast_recurrent_supported(const FastLayer &f, const LayerParams &p, int B);
 // h / c are the caller's state (B rows); y is [T][B][O].  Returns a qlstm_error.
 int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastScratch &s, const int16_t *X, int T, int B,
-                          int8_t *h, int16_t *c, int8_t *y, int *status, unsigned long long *phase_ns, cudaStream_t st,
-                          int *launches);
+                          int8_t *h, int16_t *c, int8_t *y, int *status, unsigned long long *phase_ns, bool allow_small,
+                          cudaStream_t st, int *launches);
 
 }  // namespace ql

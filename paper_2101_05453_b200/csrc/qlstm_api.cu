@@ -367,13 +367,13 @@ int qlstm_run(qlstm_t *q, const int8_t *x_dev, int T, int B, int8_t *h_dev, int1
             size_t rec = trace_record_bytes(B, p.C, p.O);
             bool fast_ok = !trace && fast_recurrent_supported(L.fast, p, B);
             int impl = q->impl_rec;
-            if (impl == 2 && !fast_ok) return trace ? QLSTM_ERR_ARG : QLSTM_ERR_DIM;
-            bool use_fast = (impl == 2) || (impl == 0 && fast_ok);
+            if (impl >= 2 && !fast_ok) return trace ? QLSTM_ERR_ARG : QLSTM_ERR_DIM;
+            bool use_fast = (impl >= 2) || (impl == 0 && fast_ok);
             int launches = 0;
             cudaError_t e;
             if (use_fast) {
                 int frc = launch_recurrent_fast(L.fast, p, q->fscratch, q->X, T, B, h_dev + h_off, c_dev + c_off, outp,
-                                                q->status, q->profiling ? q->phase_ns : nullptr, st, &launches);
+                                                q->status, q->profiling ? q->phase_ns : nullptr, impl != 3, st, &launches);
                 if (frc != QLSTM_OK) return frc;
                 e = cudaSuccess;
             } else {
@@ -438,7 +438,7 @@ int qlstm_last_status(qlstm_t *q)
 
 int qlstm_set_impl(qlstm_t *q, int projection_impl, int recurrent_impl)
 {
-    if (!q || projection_impl < 0 || projection_impl > 2 || recurrent_impl < 0 || recurrent_impl > 2) return QLSTM_ERR_ARG;
+    if (!q || projection_impl < 0 || projection_impl > 2 || recurrent_impl < 0 || recurrent_impl > 3) return QLSTM_ERR_ARG;
     q->impl_proj = projection_impl;
     q->impl_rec = recurrent_impl;
     return QLSTM_OK;

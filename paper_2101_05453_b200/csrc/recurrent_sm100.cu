@@ -47,6 +47,9 @@ struct RecParams {
     int pn, npn, n_ptiles;
     int kb_h, kb_c, stages;
     int items_per_cta;            // cells of the B x C grid per CTA in the elementwise phase
+    int small;                    // small batch: dp4a mat-vec with warp reductions instead of TMA + tcgen05
+    int rpc;                      // small batch: projection rows per CTA
+    const int8_t *R, *Wproj;      // packed weights (small-batch prologue copies its slices with plain loads)
     int fast_rescale_ok;          // every rescale of this layer has shift <= 0
     const int16_t *X;             // [T][B][N]
     int16_t *c;                   // [B][C]
@@ -280,12 +283,12 @@ template <int G>
 __device__ __forceinline__ void load_pair_i16(const int16_t *ptr, bool readonly, int32_t (&v)[2][4])
 {
     if (G == 4) {
-        const uint4 q = readonly ? __ldg(reinterpret_cast<const uint4 *>(ptr)) : *reinterpret_cast<const uint4 *>(ptr);
+        const uint4 q = readonly ? __ldg(reinterpret_cast<const uint4 *>(ptr)) : __ldcg(reinterpret_cast<const uint4 *>(ptr));
         v[0][0] = lo16(q.x); v[0][1] = hi16(q.x); v[0][2] = lo16(q.y); v[0][3] = hi16(q.y);
         v[1][0] = lo16(q.z); v[1][1] = hi16(q.z); v[1][2] = lo16(q.w); v[1][3] = hi16(q.w);
     } else {
         const uint32_t *w = reinterpret_cast<const uint32_t *>(ptr);
-        const uint32_t a = readonly ? __ldg(w) : w[0], b = readonly ? __ldg(w + 1) : w[1], c = readonly ? __ldg(w + 2) : w[2];
+        const uint32_t a = readonly ? __ldg(w) : __ldcg(w), b = readonly ? __ldg(w + 1) : __ldcg(w + 1), c = readonly ? __ldg(w + 2) : __ldcg(w + 2);
         v[0][0] = lo16(a); v[0][1] = hi16(a); v[0][2] = lo16(b);
         v[1][0] = hi16(b); v[1][1] = lo16(c); v[1][2] = hi16(c);
         v[0][3] = 0; v[1][3] = 0;
@@ -297,7 +300,7 @@ __device__ __forceinline__ void load_pair_i32(const int32_t *ptr, bool readonly,
 #pragma unroll
     for (int k = 0; k < 2; ++k)
 #pragma unroll
-        for (int g = 0; g < 4; ++g) v[k][g] = g < G ? (readonly ? __ldg(ptr + k * G + g) : ptr[k * G + g]) : 0;
+        for (int g = 0; g < 4; ++g) v[k][g] = g < G ? (readonly ? __ldg(ptr + k * G + g) : __ldcg(ptr + k * G + g)) : 0;
 }
 
 __device__ __forceinline__ void store_hidden_pair(const RecParams &p, int b, int u, int t, int32_t m0, int32_t m1, int8_t *h_next)
@@ -498,6 +501,79 @@ __device__ __forceinline__ void phase_b(const RecParams &p, RecCtl *ctl, int t, 
 }
 
 // ------------------------------------------------------------------------------------------------
+// Small batch (B <= 16): the matmuls are mat-vec products, far too small for a 128-row tensor-core tile
+// and dominated by TMA / TMEM round-trip latency.  Each warp takes whole weight rows from shared memory,
+// lanes split K in 128-byte strides (conflict-free), dp4a accumulates, one warp reduction per (row, batch).
+
+__device__ __forceinline__ void stage_rows(int8_t *dst_s, const int8_t *src, int bytes)
+{
+    const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
+    uint4 *d4 = reinterpret_cast<uint4 *>(dst_s);
+    for (int i = threadIdx.x; i < (bytes >> 4); i += RTHREADS) d4[i] = __ldcg(s4 + i);   // L2 loads: written by other CTAs this step
+    __syncthreads();
+}
+
+template <int BMAX>
+__device__ __forceinline__ int32_t warp_dots(const int8_t *w_row, const int8_t *v_s, int K, int lane)
+{
+    const int32_t *rw = reinterpret_cast<const int32_t *>(w_row);
+    int32_t part[BMAX];
+#pragma unroll
+    for (int b = 0; b < BMAX; ++b) part[b] = 0;
+    for (int w = lane; w < (K >> 2); w += 32) {
+        const int32_t r = rw[w];
+#pragma unroll
+        for (int b = 0; b < BMAX; ++b)
+            part[b] = __dp4a(r, reinterpret_cast<const int32_t *>(v_s + (size_t)b * K)[w], part[b]);
+    }
+    int32_t mine = 0;
+#pragma unroll
+    for (int b = 0; b < BMAX; ++b) {
+        const int32_t sum = __reduce_add_sync(0xffffffffu, part[b]);
+        if (lane == b) mine = sum;
+    }
+    return mine;                                   // lane b holds the dot product with batch row b
+}
+
+template <int BMAX>
+__device__ __forceinline__ void phase_a_small(const RecParams &p, int t, int cur, int n0, int n_cnt, const int8_t *R_s,
+                                              int8_t *stage_s, const int32_t *bh_s)
+{
+    stage_rows(stage_s, p.hbuf + (size_t)cur * p.Bpad * p.O, p.B * p.O);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const bool peep = (p.flags & F_PEEPHOLE) != 0;
+    for (int n = warp; n < n_cnt; n += RTHREADS / 32) {
+        const int32_t mine = warp_dots<BMAX>(R_s + (size_t)n * p.O, stage_s, p.O, lane);
+        if (lane < p.B) {
+            const int b = lane, gi = n % p.G;
+            const int32_t acc = add_sat(mine, bh_s[n]);
+            const int32_t H = sat16(rescale_sel(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
+            const int32_t X = __ldg(p.X + ((size_t)t * p.B + b) * p.N + n0 + n);
+            if (peep) p.pre[(size_t)b * p.N + n0 + n] = X + H;
+            else ((int16_t *)p.pre)[(size_t)b * p.N + n0 + n] = (int16_t)sat16(X + H);
+        }
+    }
+}
+
+template <int BMAX>
+__device__ __forceinline__ void phase_c_small(const RecParams &p, int t, int p_lo, int cnt, const int8_t *Wp_s,
+                                              int8_t *stage_s, int8_t *h_next)
+{
+    stage_rows(stage_s, p.mbuf, p.B * p.C);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int r = warp; r < cnt; r += RTHREADS / 32) {
+        const int32_t mine = warp_dots<BMAX>(Wp_s + (size_t)r * p.C, stage_s, p.C, lane);
+        if (lane < p.B) {
+            const int b = lane, o = p_lo + r;
+            const int32_t acc = add_sat(mine, __ldg(p.bp + o));
+            const int32_t hq = sat8(rescale_sel(acc, p.eff_proj, p.f_proj, p.fast_rescale_ok) + p.zp_h);
+            h_next[(size_t)b * p.O + o] = (int8_t)hq;
+            p.y[((size_t)t * p.B + b) * p.O + o] = (int8_t)hq;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 
 __global__ void __launch_bounds__(RTHREADS, 1)
 k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_R,
@@ -549,11 +625,25 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    // resident weights: one TMA box per k-block
+    // small batch: this CTA's rows of R and W_proj as plain row-major copies
+    const int sp_lo = cta * p.rpc;
+    int sp_cnt = (proj && p.small) ? p.rpc : 0;
+    if (sp_lo + sp_cnt > p.O) sp_cnt = p.O - sp_lo > 0 ? p.O - sp_lo : 0;
+    if (p.small) {
+        if (has_cells) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(p.R + (size_t)n0 * p.O);
+            for (int i = threadIdx.x; i < (n_cnt * p.O) >> 4; i += RTHREADS) reinterpret_cast<uint4 *>(R_s)[i] = __ldg(src + i);
+        }
+        if (sp_cnt > 0) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(p.Wproj + (size_t)sp_lo * p.C);
+            for (int i = threadIdx.x; i < (sp_cnt * p.C) >> 4; i += RTHREADS) reinterpret_cast<uint4 *>(Wp_s)[i] = __ldg(src + i);
+        }
+    }
+    // resident weights of the tensor-core path: one TMA box per k-block
     if (threadIdx.x == 0) {
         uint32_t bytes = 0;
-        if (has_cells) bytes += (uint32_t)(p.kb_h * p.nc_pad * 128);
-        if (has_ptile) bytes += (uint32_t)(p.kb_c * p.pn * 128);
+        if (has_cells && !p.small) bytes += (uint32_t)(p.kb_h * p.nc_pad * 128);
+        if (has_ptile && !p.small) bytes += (uint32_t)(p.kb_c * p.pn * 128);
         if (bytes) {
             ptx::mbar_arrive_expect_tx(&ctl->w_full, bytes);
             if (has_cells)
@@ -589,7 +679,15 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
         const uint32_t par = (uint32_t)t & 1u;
 
         // ================= phase A: gate sums =================
-        if (has_cells) {
+        if (p.small) {
+            if (has_cells) {
+                if (p.B == 1) phase_a_small<1>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
+                else if (p.B <= 2) phase_a_small<2>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
+                else if (p.B <= 4) phase_a_small<4>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
+                else if (p.B <= 8) phase_a_small<8>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
+                else phase_a_small<16>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
+            }
+        } else if (has_cells) {
             if (warp == 0) {
                 if (lane == 0) {
                     fence_proxy_async_all();
@@ -662,7 +760,15 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
 
         // ================= phase C: projection =================
         if (proj) {
-            if (has_ptile) {
+            if (p.small) {
+                if (sp_cnt > 0) {
+                    if (p.B == 1) phase_c_small<1>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
+                    else if (p.B <= 2) phase_c_small<2>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
+                    else if (p.B <= 4) phase_c_small<4>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
+                    else if (p.B <= 8) phase_c_small<8>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
+                    else phase_c_small<16>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
+                }
+            } else if (has_ptile) {
                 if (warp == 0) {
                     if (lane == 0) {
                         fence_proxy_async_all();
@@ -824,8 +930,8 @@ void fast_layer_destroy(FastLayer &) {}
 bool fast_recurrent_supported(const FastLayer &f, const LayerParams &, int B) { return f.rec_ok && B <= 256; }
 
 int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastScratch &s, const int16_t *X, int T, int B,
-                          int8_t *h, int16_t *c, int8_t *y, int *status, unsigned long long *phase_ns, cudaStream_t st,
-                          int *launches)
+                          int8_t *h, int16_t *c, int8_t *y, int *status, unsigned long long *phase_ns, bool allow_small,
+                          cudaStream_t st, int *launches)
 {
     RecParams rp;
     memset(&rp, 0, sizeof(rp));
@@ -840,6 +946,13 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
         rp.items_per_cta = ((B + f.grid - 1) / f.grid) * p.C;
     else
         rp.items_per_cta = round_up((int)(((long)B * p.C + f.grid - 1) / f.grid), 8);
+    rp.R = p.R; rp.Wproj = p.Wproj;
+    rp.rpc = (p.O + f.grid - 1) / f.grid;
+    {
+        const int maxk = p.O > p.C ? p.O : p.C;
+        const bool fits = (size_t)16 * maxk <= (size_t)f.stages * A_STAGE_BYTES && (!(p.flags & F_PROJECTION) || rp.rpc <= f.pn);
+        rp.small = (allow_small && B <= 16 && fits) ? 1 : 0;
+    }
     rp.fast_rescale_ok = 1;
     for (int g = 0; g < p.G; ++g) {
         rp.eff_h[g] = p.eff_h[g]; rp.eff_c[g] = p.eff_c[g]; rp.eff_ln[g] = p.eff_ln[g];
