@@ -303,18 +303,26 @@ def main():
             h1, c1 = torch.from_numpy(hi).to(dev), torch.from_numpy(ci).to(dev)
             y1 = torch.zeros((T, 1, O), dtype=torch.int8, device=dev)
             ts = []
-            for i in range(5):
+            for i in range(6):
+                if i == 3:
+                    q1.set_profiling(True)
+                    q1.get_profile(reset=True)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record()
                 q1.run(x1, T, 1, h1, c1, y1, stream=stream)
                 b.record()
                 torch.cuda.synchronize()
-                if i >= 2:
+                if i >= 3:
                     ts.append(a.elapsed_time(b))
             q1.last_status()
+            p1 = q1.get_profile(reset=True)
             ms = statistics.median(ts)
             line["latency_batch1"] = {"us_per_timestep_whole_stack": 1e3 * ms / T,
-                                      "us_per_layer_step": 1e3 * ms / (T * n_l), "ms_per_pass": ms}
+                                      "us_per_layer_step": 1e3 * ms / (T * n_l), "ms_per_pass": ms,
+                                      "projection_us_per_layer": 1e3 * p1["projection_ms"] / (len(ts) * n_l),
+                                      "phase_us_per_layer_step": {k: 1e3 * p1[k] / (len(ts) * n_l * T) for k in
+                                                                  ("phase_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms",
+                                                                   "phase_c_ms", "wait_c_ms")}}
             q1.close()
         if not args.no_cpu_baseline:
             from oracle import qlstm_ref
