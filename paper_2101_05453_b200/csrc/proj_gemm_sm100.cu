@@ -53,8 +53,9 @@ struct SharedCtl {
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
-    for (uint32_t i = 0; i < (1u << 20); ++i) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
+    // each attempt parks the thread for up to 20 us; 100 000 attempts bound the wait to about 2 s
+    for (uint32_t i = 0; i < 100000u; ++i) {
+        if (ptx::mbar_try_wait_parked(bar, parity, 20000u)) return true;
         if (*abort_flag) return false;
     }
     *abort_flag = 1;
