@@ -32,9 +32,7 @@ void qmh_layernorm_row_fast(const int16_t *q, int n, const int16_t *L, const int
 int64_t qmh_ln_quotient_fast(int32_t q, int64_t mean, int64_t sigma)
 {
     ql::LnStats st{mean, sigma};
-    int64_t wide;
-    int32_t v = ql::ln_quotient_fast(q, ql::make_ln_row(st), &wide);
-    return (int64_t)v + wide;
+    return ql::ln_quotient_fast(q, ql::make_ln_row(st));
 }
 int32_t qmh_cell_update_fast(int32_t i, int32_t z, int32_t f, int32_t c, int m) { return ql::cell_update_fast(i, z, f, c, m); }
 int32_t qmh_hidden_fast(int32_t o, int32_t c, int m, int32_t mult, int32_t shift, int32_t zp)

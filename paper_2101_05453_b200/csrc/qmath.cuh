@@ -172,6 +172,17 @@ QL_HD float mul_rn(float a, float b)
 #endif
 }
 
+QL_HD uint32_t shr_clamp(uint32_t v, uint32_t s)     // v >> s, 0 for s >= 32
+{
+#if defined(__CUDA_ARCH__)
+    uint32_t r;
+    asm("shr.b32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(s));
+    return r;
+#else
+    return s >= 32 ? 0u : v >> s;
+#endif
+}
+
 template <bool TANH>
 QL_HD int32_t act_q_fast(int32_t x, int m)
 {
@@ -182,10 +193,11 @@ QL_HD int32_t act_q_fast(int32_t x, int m)
     const int sh = 19 - m;
     const uint64_t t = ((uint64_t)a * ck + ((uint64_t)1 << (sh - 1))) >> sh;
     const uint32_t n = (uint32_t)(t >> 26);
-    const int32_t g6 = (int32_t)((((uint32_t)t & 0x3FFFFFFu) - (1u << 25)) << 6);     // 64 * g
+    // 64 * g with g = frac(t) - 2^25: the shift drops the integer part, subtracting 2^31 flips the top bit
+    const int32_t g6 = (int32_t)(((uint32_t)t << 6) ^ 0x80000000u);
     const uint32_t s = (uint32_t)(g6 >> 31);                       // all ones iff g < 0
     const uint32_t lo_pos = 0x80000000u + (s & 0xFFFFFFC0u);       // 64 * (2^25 - [g < 0]): accumulator > 0
-    const uint32_t lo_neg = 0x7FFFFFC0u - (s & 0xFFFFFFC0u);       // 64 * (2^25 - [g >= 0]): accumulator < 0
+    const uint32_t lo_neg = lo_pos ^ 0xFFFFFFC0u;                  // 64 * (2^25 - [g >= 0]): accumulator < 0
 #define QL_HORNER(acc, ck_, lo_) (int32_t)(((int64_t)(acc) * g6 + (int64_t)(((uint64_t)(uint32_t)(ck_) << 32) | (lo_))) >> 32)
     int32_t acc = c6;
     acc = QL_HORNER(acc, c5, lo_pos);
@@ -195,10 +207,11 @@ QL_HD int32_t act_q_fast(int32_t x, int m)
     acc = QL_HORNER(acc, c1, lo_pos);
     acc = QL_HORNER(acc, c0, lo_neg);
 #undef QL_HORNER
-    const uint32_t nn = n > 31 ? 31 : n;
-    uint32_t E = ((uint32_t)acc + ((1u << nn) >> 1)) >> nn;
-    E = n > 31 ? 0u : E;
-    E = E > (1u << 30) ? (1u << 30) : E;          // only x = 0 can exceed 2^30, by a few units; same quotient
+    // E = round(acc / 2^n): for n >= 1 the high word of acc * 2^(32-n) + 2^31 (0 once n > 32); for n = 0 acc itself,
+    // clamped to 2^30 (only x = 0 exceeds it, by a few units, and the quotient is the same)
+    const uint32_t p = (uint32_t)acc;
+    const uint32_t scaled = (uint32_t)(((uint64_t)p * shr_clamp(0x80000000u, n - 1u) + 0x80000000ull) >> 32);
+    const uint32_t E = n == 0 ? (p > (1u << 30) ? (1u << 30) : p) : scaled;
     const uint32_t D = (1u << 30) + E;
     const uint32_t N = TANH ? (1u << 30) - E : (1u << 30);
     // q = floor(2^15 N / D + 1/2); the estimate is biased low by more than its error: it is q or q - 1
@@ -249,30 +262,34 @@ QL_HD LnRow make_ln_row(LnStats s)
 // q' = round(2^10 (2^10 q - mean) / sigma), exact.  Quotients below 2^16 (|z-score| < 64) take the fp32
 // estimate (biased low: q' or q' - 1) and one remainder test modulo 2^32; anything larger - a tiny sigma
 // against a large deviation - takes the plain 64-bit division.
-QL_HD int32_t ln_quotient_fast(int32_t q, const LnRow &r, int64_t *wide)
+QL_HD int64_t ln_scaled_fast(int32_t q, const LnRow &r, int32_t L, int32_t b)   // q' * L + b
 {
     const int32_t d = 1024 * q - r.mean;
     const uint32_t ad = (uint32_t)(d < 0 ? -d : d);
     const uint32_t half = r.sigma >> 1;
     const float est = fma_rn(fma_rn((float)ad, 1024.0f, (float)half), r.inv_sigma, -0.05f);
-    *wide = 0;
     if (est < 65536.0f) {
         uint32_t qe = est > 0.0f ? (uint32_t)est : 0u;
         const uint32_t rem = (ad << 10) + half - qe * r.sigma;     // in [0, 2 sigma), exact modulo 2^32
         qe += (rem >= r.sigma && r.sigma != 0u) ? 1u : 0u;
-        return d < 0 ? -(int32_t)qe : (int32_t)qe;
+        const int32_t qp = d < 0 ? -(int32_t)qe : (int32_t)qe;
+        return (int64_t)qp * L + b;                                // one 32 x 32 + 64 multiply-add
     }
     const uint64_t quo = r.sigma ? ((uint64_t)ad * 1024u + half) / r.sigma : 0u;
-    *wide = d < 0 ? -(int64_t)quo : (int64_t)quo;
-    return 0;
+    return (d < 0 ? -(int64_t)quo : (int64_t)quo) * (int64_t)L + (int64_t)b;
+}
+
+QL_HD int64_t ln_quotient_fast(int32_t q, const LnRow &r) { return ln_scaled_fast(q, r, 1, 0); }
+
+QL_HD int32_t sat32_halves(int64_t v)              // saturate through the two 32-bit halves
+{
+    const int32_t lo = (int32_t)v, hi = (int32_t)(v >> 32);
+    return hi == (lo >> 31) ? lo : (int32_t)(0x7fffffff ^ (hi >> 31));
 }
 
 QL_HD int32_t ln_apply_fast(int32_t q, const LnRow &r, int32_t L, int32_t b, Scale eff_ln, const FastScale &f_ln)
 {
-    int64_t wide;
-    const int32_t qp = ln_quotient_fast(q, r, &wide);
-    const int64_t v = ((int64_t)qp + wide) * (int64_t)L + (int64_t)b;
-    const int32_t v32 = sat32(v);
+    const int32_t v32 = sat32_halves(ln_scaled_fast(q, r, L, b));
     return sat16(eff_ln.shift <= 0 ? fast_rescale(v32, f_ln) : mbqm(v32, eff_ln));
 }
 
