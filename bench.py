@@ -94,6 +94,22 @@ class ClockSampler:
         return out
 
 
+# DRAM traffic of the recurrent kernel from one ncu capture (profiles/k_recurrent_sm100_config5_b256_T40.md):
+# dram__bytes_read.sum + dram__bytes_write.sum = 188.0 MB for 40 steps of config 5 at batch 256; per-step traffic is
+# steady, so a launch of T steps moves T / 40 of that.  Valid only for the kernel sources the counters were taken
+# from: if they changed since, the figure is reported as null.
+NCU_RECURRENT = {"bytes": 188.04e6, "steps": 40, "config": 5, "batch": 256, "source_sha": "8fc728514bc393f5"}
+
+
+def recurrent_source_sha():
+    import hashlib
+    m = hashlib.sha256()
+    for f in ("recurrent_sm100.cu", "qmath.cuh", "sm100_ptx.cuh"):
+        with open(os.path.join(ROOT, "paper_2101_05453_b200", "csrc", f), "rb") as fh:
+            m.update(fh.read())
+    return m.hexdigest()[:16]
+
+
 def algorithmic_ops(layers, B, T):
     """int8 multiply-accumulates counted as 2 ops, per pass: (projection GEMMs, recurrent + projection matmuls)."""
     gemm = rec = 0
@@ -280,6 +296,13 @@ def main():
                 "us_per_layer_step": 1e3 * rec_ms / (n_l * T),
                 "phase_us_per_layer_step": {k: 1e3 * prof[k] / (max(args.steps, 1) * n_l * T) for k in
                                             ("phase_a_ms", "matmul_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms", "phase_c_ms", "wait_c_ms")}}
+    if (args.config == NCU_RECURRENT["config"] and B == NCU_RECURRENT["batch"]
+            and recurrent_source_sha() == NCU_RECURRENT["source_sha"]):
+        roof_rec["traffic"] = NCU_RECURRENT["bytes"] * T / NCU_RECURRENT["steps"]      # bytes per launch (one layer)
+    # algorithmic HBM bytes of the recurrent kernel per launch: X read once, y written once, state in and out
+    q0 = w.layers[0]
+    G0 = 3 if (q0.flags & 8) else 4
+    roof_rec["algorithmic_hbm_bytes"] = T * B * (q0.n_cell * G0 * 2 + q0.n_output) + 2 * B * (q0.n_output + 2 * q0.n_cell)
     dominant = roof_rec if rec_ms >= proj_ms else roof_proj
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
