@@ -138,6 +138,12 @@ size_t qlstm_trace_bytes(const qlstm_t *q, int T, int B);
  * recurrent_impl 3 = like 2 but with the tensor-core matmuls even at batch <= 16, where 0 and 2 use dp4a mat-vecs. */
 int qlstm_set_impl(qlstm_t *q, int projection_impl, int recurrent_impl);
 
+/* Failure-path check: with missing_arrivals > 0 every grid barrier of the persistent recurrent kernel waits for
+ * that many arrivals that never come, for at most limit_ns (<= 1 s); the wait then runs out, the kernel sets its
+ * status word, every block leaves the time loop, frees its tensor memory and returns, and qlstm_last_status
+ * reports QLSTM_ERR_TIMEOUT.  Nothing faults or hangs and the handle stays usable; 0 restores normal operation. */
+int qlstm_debug_barrier_timeout(qlstm_t *q, int missing_arrivals, unsigned long long limit_ns);
+
 /* Per-kernel device times of the runs since the last reset, measured with CUDA events on the
  * run's stream when profiling is on (it adds two event records per launch). */
 typedef struct {

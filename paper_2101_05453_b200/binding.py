@@ -22,7 +22,7 @@ IMPL_AUTO, IMPL_SIMPLE, IMPL_FAST = 0, 1, 2
 EXPORTS = ["qlstm_create", "qlstm_run", "qlstm_run_host", "qlstm_input_projection", "qlstm_last_status",
            "qlstm_destroy", "qlstm_strerror", "qlstm_trace_bytes", "qlstm_set_impl", "qlstm_set_profiling",
            "qlstm_get_profile", "qlstm_device_info", "qlstm_eval_activations", "qlstm_eval_layernorm_row",
-           "qlstm_layernorm_rows_static"]
+           "qlstm_layernorm_rows_static", "qlstm_debug_barrier_timeout"]
 
 
 class Scale(C.Structure):
@@ -68,7 +68,8 @@ def lib():
     """Loads libqlstm.so, building it first if the sources are newer.  Raises if that fails."""
     global _lib
     if _lib is None:
-        path = _build.build() if os.environ.get("QLSTM_NO_BUILD") != "1" else _build.LIB
+        # QLSTM_LIB names a prebuilt library to load instead of the in-tree one
+        path = os.environ.get("QLSTM_LIB") or (_build.build() if os.environ.get("QLSTM_NO_BUILD") != "1" else _build.LIB)
         L = C.CDLL(path)
         L.qlstm_create.restype = C.c_int
         L.qlstm_create.argtypes = [C.POINTER(Layer), C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_void_p)]
@@ -99,6 +100,8 @@ def lib():
         L.qlstm_eval_activations.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         L.qlstm_eval_layernorm_row.restype = C.c_int
         L.qlstm_eval_layernorm_row.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p, C.c_void_p]
+        L.qlstm_debug_barrier_timeout.restype = C.c_int
+        L.qlstm_debug_barrier_timeout.argtypes = [C.c_void_p, C.c_int, C.c_ulonglong]
         L.qlstm_layernorm_rows_static.restype = C.c_int
         L.qlstm_layernorm_rows_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p,
                                                   C.c_void_p]
@@ -228,6 +231,9 @@ class QLSTM:
         p = Profile()
         _check(lib().qlstm_get_profile(self._h, C.byref(p), int(reset)), "qlstm_get_profile")
         return {k: getattr(p, k) for k, _ in Profile._fields_}
+
+    def debug_barrier_timeout(self, missing_arrivals: int, limit_ns: int = 0):
+        _check(lib().qlstm_debug_barrier_timeout(self._h, missing_arrivals, limit_ns), "qlstm_debug_barrier_timeout")
 
     def device_info(self):
         a, b = C.c_int(), C.c_int()

@@ -36,6 +36,9 @@ struct FastLayer {
     int stages = 0;
     size_t smem = 0;
     CUtensorMap map_R, map_Wp, map_h, map_m;
+    // test hook: make every grid barrier expect `dbg_barrier_extra` arrivals that never come, with a short wait limit
+    unsigned dbg_barrier_extra = 0;
+    unsigned long long dbg_spin_limit_ns = 0;
 };
 
 int fast_scratch_init(FastScratch &s, int max_B, int maxC, int maxO, int maxN, int sm_count);

@@ -444,6 +444,17 @@ int qlstm_set_impl(qlstm_t *q, int projection_impl, int recurrent_impl)
     return QLSTM_OK;
 }
 
+int qlstm_debug_barrier_timeout(qlstm_t *q, int missing_arrivals, unsigned long long limit_ns)
+{
+    if (!q || missing_arrivals < 0 || missing_arrivals > 1024) return QLSTM_ERR_ARG;
+    if (missing_arrivals > 0 && (limit_ns == 0 || limit_ns > 1000000000ull)) return QLSTM_ERR_ARG;   // at most 1 s
+    for (auto &L : q->layers) {
+        L.fast.dbg_barrier_extra = (unsigned)missing_arrivals;
+        L.fast.dbg_spin_limit_ns = missing_arrivals > 0 ? limit_ns : 0;
+    }
+    return QLSTM_OK;
+}
+
 int qlstm_set_profiling(qlstm_t *q, int enabled)
 {
     if (!q) return QLSTM_ERR_ARG;

@@ -63,6 +63,8 @@ struct RecParams {
     Scale eff_h[4], eff_c[4], eff_ln[4], eff_m, eff_proj;
     FastScale f_h[4], f_c[4], f_ln[4], f_m, f_proj;
     int gate_slot[4];             // canonical gate -> slot, -1 if absent
+    unsigned long long spin_limit_ns;   // bound of one grid-barrier wait
+    unsigned barrier_extra;             // 0; a test sets it to make the barrier wait for an arrival that never comes
     unsigned long long *phase_ns; // null, or 6 accumulators: work and barrier wait of phases A, B, C (CTA 0)
 };
 
@@ -109,14 +111,14 @@ __device__ __forceinline__ void grid_sync(const RecParams &p, unsigned &epoch, v
     __syncthreads();
     if (threadIdx.x == 0) {
         ++epoch;
-        const unsigned target = epoch * gridDim.x;
+        const unsigned target = epoch * gridDim.x + p.barrier_extra;
         asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.bar) : "memory");
         const unsigned long long t0 = globaltimer();
         unsigned spins = 0;
         while (ld_acquire(p.bar) < target) {
             if ((++spins & 63u) == 0u) {
                 if (ld_acquire(p.bar + 1) != 0u) { *abort_flag = 1; break; }
-                if (globaltimer() - t0 > SPIN_LIMIT_NS) {
+                if (globaltimer() - t0 > p.spin_limit_ns) {
                     atomicExch(p.bar + 1, 1u);
                     *abort_flag = 1;
                     break;
@@ -966,6 +968,8 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     rp.f_proj = make_fast_scale(p.eff_proj);
     rp.f_m = make_fast_scale(p.eff_m);
     rp.phase_ns = phase_ns;
+    rp.spin_limit_ns = f.dbg_spin_limit_ns ? f.dbg_spin_limit_ns : SPIN_LIMIT_NS;
+    rp.barrier_extra = f.dbg_barrier_extra;
     if (p.eff_proj.shift > 0) rp.fast_rescale_ok = 0;
     for (int g = 0; g < 4; ++g) rp.gate_slot[g] = p.slot_of_gate[g];
     rp.X = X; rp.c = c; rp.y = y;

@@ -216,6 +216,27 @@ def test_empty_inputs_and_limits():
         assert e.value.code == qlstm.ERR_ARG
 
 
+def test_bounded_wait_reports_timeout_and_handle_stays_usable():
+    """A grid barrier that waits for an arrival nobody makes runs into its (here 3 ms) limit: the kernel returns
+    by itself, the status is QLSTM_ERR_TIMEOUT, and the next run on the same handle is correct again."""
+    import paper_2101_05453_b200 as qlstm
+    w = random_layer_stack(55, 1, 32, 64, 48, projection=True, layernorm=True, T=4, B=20)
+    want = oracle(w)
+    with qlstm.QLSTM(w.layers, w.T, w.B) as hnd:
+        hnd.set_impl(FAST, FAST)
+        hnd.debug_barrier_timeout(1, 3_000_000)
+        with pytest.raises(qlstm.QlstmError) as e:
+            run_gpu(w, handle=hnd, impl=(FAST, FAST))
+        assert e.value.code == qlstm.ERR_TIMEOUT
+        hnd.debug_barrier_timeout(0)
+        check_equal(run_gpu(w, handle=hnd, impl=(FAST, FAST)), want, "after timeout")
+
+
+def test_batch_beyond_the_persistent_kernel_limit_uses_the_simple_path():
+    w = random_layer_stack(56, 1, 16, 32, 32, T=3, B=300)
+    check_equal(run_gpu(w), oracle(w), "B=300")
+
+
 def test_folded_bias_out_of_range_is_rejected():
     import paper_2101_05453_b200 as qlstm
     w = make_workload(1)
