@@ -94,7 +94,7 @@ class ClockSampler:
         return out
 
 
-# DRAM traffic of the recurrent kernel from one ncu capture (profiles/k_recurrent_sm100_config5_b256_T40.md):
+# DRAM traffic of the recurrent kernel from one ncu capture (its summary is kept with the other profile summaries):
 # dram__bytes_read.sum + dram__bytes_write.sum = 188.0 MB for 40 steps of config 5 at batch 256; per-step traffic is
 # steady, so a launch of T steps moves T / 40 of that.  Valid only for the kernel sources the counters were taken
 # from: if they changed since, the figure is reported as null.
@@ -227,7 +227,7 @@ def main():
         one_step()
     q.last_status()
     torch.cuda.synchronize()
-    q.set_profiling(True)
+    q.set_profiling(1)                    # per-kernel event times only: the device phase timers slow the kernel
     q.get_profile(reset=True)
 
     sampler = ClockSampler(local)
@@ -244,7 +244,12 @@ def main():
     step_ms = [a.elapsed_time(b) for a, b in events]
     total_ms = sum(step_ms)
     prof = q.get_profile(reset=True)
-    q.set_profiling(False)
+    # phase breakdown of the recurrent kernel: a separate untimed pass with the device phase timers on
+    q.set_profiling(2)
+    one_step()
+    torch.cuda.synchronize()
+    prof_phase = q.get_profile(reset=True)
+    q.set_profiling(0)
     if dist is not None:
         t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -294,8 +299,10 @@ def main():
                 "frac": rec_tops / int8_peak, "traffic": None,
                 "peak_source": f"2 x bf16 sustained, {peaks['source']}", "ms_per_launch": rec_ms / n_l,
                 "us_per_layer_step": 1e3 * rec_ms / (n_l * T),
-                "phase_us_per_layer_step": {k: 1e3 * prof[k] / (max(args.steps, 1) * n_l * T) for k in
-                                            ("phase_a_ms", "matmul_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms", "phase_c_ms", "wait_c_ms")}}
+                "phase_us_per_layer_step": {k: 1e3 * prof_phase[k] / (n_l * T) for k in
+                                            ("phase_a_ms", "matmul_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms", "phase_c_ms", "wait_c_ms")},
+                "phase_note": "separate pass with the device phase timers on (they slow the kernel: "
+                              f"{1e3 * prof_phase['recurrent_ms'] / (n_l * T):.2f} us per layer-step in that pass)"}
     if (args.config == NCU_RECURRENT["config"] and B == NCU_RECURRENT["batch"]
             and recurrent_source_sha() == NCU_RECURRENT["source_sha"]):
         roof_rec["traffic"] = NCU_RECURRENT["bytes"] * T / NCU_RECURRENT["steps"]      # bytes per launch (one layer)
@@ -326,24 +333,27 @@ def main():
             h1, c1 = torch.from_numpy(hi).to(dev), torch.from_numpy(ci).to(dev)
             y1 = torch.zeros((T, 1, O), dtype=torch.int8, device=dev)
             ts = []
-            for i in range(6):
+            q1.set_profiling(1)
+            for i in range(7):
                 if i == 3:
-                    q1.set_profiling(True)
                     q1.get_profile(reset=True)
+                if i == 6:                        # one extra pass with the device phase timers, not part of the latency
+                    p1 = q1.get_profile(reset=True)
+                    q1.set_profiling(2)
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record()
                 q1.run(x1, T, 1, h1, c1, y1, stream=stream)
                 b.record()
                 torch.cuda.synchronize()
-                if i >= 3:
+                if 3 <= i < 6:
                     ts.append(a.elapsed_time(b))
             q1.last_status()
-            p1 = q1.get_profile(reset=True)
+            p1_phase = q1.get_profile(reset=True)
             ms = statistics.median(ts)
             line["latency_batch1"] = {"us_per_timestep_whole_stack": 1e3 * ms / T,
                                       "us_per_layer_step": 1e3 * ms / (T * n_l), "ms_per_pass": ms,
                                       "projection_us_per_layer": 1e3 * p1["projection_ms"] / (len(ts) * n_l),
-                                      "phase_us_per_layer_step": {k: 1e3 * p1[k] / (len(ts) * n_l * T) for k in
+                                      "phase_us_per_layer_step": {k: 1e3 * p1_phase[k] / (n_l * T) for k in
                                                                   ("phase_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms",
                                                                    "phase_c_ms", "wait_c_ms")}}
             q1.close()

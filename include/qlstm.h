@@ -145,7 +145,11 @@ int qlstm_set_impl(qlstm_t *q, int projection_impl, int recurrent_impl);
 int qlstm_debug_barrier_timeout(qlstm_t *q, int missing_arrivals, unsigned long long limit_ns);
 
 /* Per-kernel device times of the runs since the last reset, measured with CUDA events on the
- * run's stream when profiling is on (it adds two event records per launch). */
+ * run's stream when profiling is on (it adds two event records per launch).
+ * qlstm_set_profiling levels: 0 off; 1 the per-kernel event times; 2 also the device phase timers inside the
+ * persistent recurrent kernel.  Level 2 perturbs what it measures (the first block updates its timers in
+ * global memory before every grid barrier and so arrives late at each), so take throughput numbers at
+ * level 0 or 1 and the phase breakdown in a separate pass. */
 typedef struct {
     double projection_ms; int projection_launches;
     double recurrent_ms;  int recurrent_launches;
@@ -155,7 +159,7 @@ typedef struct {
     double phase_a_ms, wait_a_ms, phase_b_ms, wait_b_ms, phase_c_ms, wait_c_ms;
     double matmul_a_ms;   /* part of phase_a_ms before the first accumulator is ready (operand load + MMA) */
 } qlstm_profile_t;
-int qlstm_set_profiling(qlstm_t *q, int enabled);
+int qlstm_set_profiling(qlstm_t *q, int level);
 int qlstm_get_profile(qlstm_t *q, qlstm_profile_t *out, int reset);
 
 /*

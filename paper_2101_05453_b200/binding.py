@@ -224,8 +224,9 @@ class QLSTM:
     def set_impl(self, projection: int = IMPL_AUTO, recurrent: int = IMPL_AUTO):
         _check(lib().qlstm_set_impl(self._h, projection, recurrent), "qlstm_set_impl")
 
-    def set_profiling(self, on: bool):
-        _check(lib().qlstm_set_profiling(self._h, int(on)), "qlstm_set_profiling")
+    def set_profiling(self, level: int):
+        """0 off, 1 per-kernel event times, 2 also the device phase timers (which slow the kernel they time)."""
+        _check(lib().qlstm_set_profiling(self._h, int(level)), "qlstm_set_profiling")
 
     def get_profile(self, reset: bool = True) -> dict:
         p = Profile()

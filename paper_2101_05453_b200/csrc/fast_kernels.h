@@ -12,8 +12,9 @@ namespace ql {
 struct FastScratch {
     int Bpad = 0;                // max batch rounded up to 128: rows of the MMA operands
     int sm_count = 0;
-    int8_t *hbuf = nullptr;      // [2][Bpad][max O]  h^{t-1} / h^t, the recurrent matmul's A operand
-    int8_t *mbuf = nullptr;      // [Bpad][max C]     hidden state m, the projection's A operand
+    int8_t *hbuf = nullptr;      // [2][Bpad x max O]  h^{t-1} / h^t, the recurrent matmul's A operand (tiled k-block image,
+                                 //                    plain rows at small batch)
+    int8_t *mbuf = nullptr;      // [Bpad x max C]     hidden state m, the projection's A operand (same layouts)
     int32_t *pre = nullptr;      // [max B][max N]    gate sums between the matmul and elementwise phases
                                  //                   (int16 values, or int32 X+H when a peephole follows)
     unsigned *bar = nullptr;     // [0] grid-barrier counter, [1] abort word
@@ -33,9 +34,10 @@ struct FastLayer {
     int nc_pad = 0;              // UMMA N of the recurrent matmul (multiple of 16)
     int pn = 0, npn = 0;         // projection: N-slice width and number of N slices
     int kb_h = 0, kb_c = 0;      // 128-byte k-blocks of the recurrent / projection matmul
-    int stages = 0;
+    int stages = 0;              // ring stages (power of two)
+    int n_issue_c = 1;           // projection MMA issuers, each with its own partial accumulator
     size_t smem = 0;
-    CUtensorMap map_R, map_Wp, map_h, map_m;
+    CUtensorMap map_R, map_Wp;   // resident weight slices; the streamed operands h, m use plain bulk copies
     // test hook: make every grid barrier expect `dbg_barrier_extra` arrivals that never come, with a short wait limit
     unsigned dbg_barrier_extra = 0;
     unsigned long long dbg_spin_limit_ns = 0;

@@ -133,7 +133,7 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before();
-    __syncthreads();
+    ptx::cta_sync();
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
@@ -256,13 +256,13 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
     }
 
     // ---------------- teardown ----------------
-    __syncthreads();
+    ptx::cta_sync();
     if (*abort_flag) {
         // a wait ran out: give copies in flight time to land, then report
         for (int i = 0; i < 200; ++i) __nanosleep(500);
         if (threadIdx.x == 0) atomicExch(p.status, 1);
     }
-    __syncthreads();
+    ptx::cta_sync();
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, TMEM_COLS);

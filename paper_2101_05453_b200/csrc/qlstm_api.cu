@@ -46,7 +46,8 @@ struct qlstm {
     cudaStream_t last_stream = nullptr;
     int impl_proj = 0, impl_rec = 0;
     // profiling
-    bool profiling = false;
+    bool profiling = false;      // level >= 1: event pairs around every launch
+    bool phase_timers = false;   // level 2: device timers inside the persistent kernel
     struct Span { cudaEvent_t a, b; int kind; int launches; };
     std::vector<Span> spans;
     std::vector<cudaEvent_t> event_pool;
@@ -373,7 +374,7 @@ int qlstm_run(qlstm_t *q, const int8_t *x_dev, int T, int B, int8_t *h_dev, int1
             cudaError_t e;
             if (use_fast) {
                 int frc = launch_recurrent_fast(L.fast, p, q->fscratch, q->X, T, B, h_dev + h_off, c_dev + c_off, outp,
-                                                q->status, q->profiling ? q->phase_ns : nullptr, impl != 3, st, &launches);
+                                                q->status, q->phase_timers ? q->phase_ns : nullptr, impl != 3, st, &launches);
                 if (frc != QLSTM_OK) return frc;
                 e = cudaSuccess;
             } else {
@@ -455,10 +456,11 @@ int qlstm_debug_barrier_timeout(qlstm_t *q, int missing_arrivals, unsigned long 
     return QLSTM_OK;
 }
 
-int qlstm_set_profiling(qlstm_t *q, int enabled)
+int qlstm_set_profiling(qlstm_t *q, int level)
 {
     if (!q) return QLSTM_ERR_ARG;
-    q->profiling = enabled != 0;
+    q->profiling = level >= 1;
+    q->phase_timers = level >= 2;
     return QLSTM_OK;
 }
 

@@ -34,18 +34,22 @@ namespace {
 constexpr int RTHREADS = 640;                 // warp 0 TMA producer, warp 1 MMA issuer, warps 2..9 matmul epilogues;
                                               // all 20 warps share the elementwise phase
 constexpr int MAX_LN_ROWS = 4;                // rows whose layer-norm statistics are held at once
-constexpr int A_STAGE_BYTES = 128 * 128;      // one k-block of the A operand: 128 rows x 128 bytes
-constexpr int MAX_STAGES = 6;
+constexpr int KB_BYTES = 128 * 128;           // one k-block of the A operand: 128 rows x 128 bytes
+constexpr int STAGE_KB = 2;                   // k-blocks per ring stage: one bulk copy brings up to 32 KB
+constexpr int STAGE_BYTES = STAGE_KB * KB_BYTES;
+constexpr int MAX_STAGES = 4;
 constexpr unsigned long long SPIN_LIMIT_NS = 2000000000ull;   // 2 s per grid barrier
 
 struct RecParams {
     int T, B, MT, Bpad;
+    size_t h_stride;              // bytes between the two h operand buffers
     int C, O, G, N;
     uint32_t flags;
     int m_bits, zp_m, zp_h;
     int cpc, n_cta_a, nc_pad;
     int pn, npn, n_ptiles;
     int kb_h, kb_c, stages;
+    int n_issue_c;                // projection: MMA issuers (= partial accumulators) sharing the K range
     int items_per_cta;            // cells of the B x C grid per CTA in the elementwise phase
     int small;                    // small batch: dp4a mat-vec with warp reductions instead of TMA + tcgen05
     int rpc;                      // small batch: projection rows per CTA
@@ -96,19 +100,21 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned *p)
 __device__ __forceinline__ unsigned long long globaltimer()
 {
     unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)::"memory");      // not to be moved across barriers
     return t;
 }
-__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// orders this thread's generic-proxy accesses to global memory with async-proxy (bulk copy) accesses to it
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 
 // Grid-wide barrier on a monotonic counter: every thread's earlier global writes are ordered before the
-// CTA barrier, thread 0 then publishes them with a release-add and polls with acquire loads.  The proxy
-// fence before it makes those generic-proxy writes visible to other CTAs' TMA loads (async proxy); the
-// thread that issues TMA loads fences again on its side after the barrier.
-__device__ __forceinline__ void grid_sync(const RecParams &p, unsigned &epoch, volatile int *abort_flag)
+// CTA barrier, one thread then publishes them with a release-add and polls with acquire loads.  Where the
+// phase before it wrote data that other CTAs fetch with bulk copies (async proxy: the operands h and m),
+// each writer first orders its generic-proxy writes against that proxy; the thread that issues the copies
+// fences again on its side after the barrier.  Gate sums are read with ordinary loads and need neither.
+__device__ __forceinline__ void grid_sync(const RecParams &p, unsigned &epoch, volatile int *abort_flag, bool wrote_operands)
 {
-    fence_proxy_async_all();
-    __syncthreads();
+    if (wrote_operands) fence_proxy_async_global();
+    ptx::cta_sync();
     if (threadIdx.x == 0) {
         ++epoch;
         const unsigned target = epoch * gridDim.x + p.barrier_extra;
@@ -127,7 +133,7 @@ __device__ __forceinline__ void grid_sync(const RecParams &p, unsigned &epoch, v
         }
         if (*abort_flag) atomicExch(p.bar + 1, 1u);
     }
-    __syncthreads();
+    ptx::cta_sync();
 }
 
 __device__ __forceinline__ int32_t rescale_sel(int32_t x, const Scale &s, const FastScale &f, int fast_ok)
@@ -149,6 +155,21 @@ __device__ __forceinline__ int32_t add_sat(int32_t a, int32_t b)
 __device__ __forceinline__ int32_t lo16(uint32_t w) { return (int32_t)(w << 16) >> 16; }
 __device__ __forceinline__ int32_t hi16(uint32_t w) { return (int32_t)w >> 16; }
 __device__ __forceinline__ uint32_t pack16(int32_t lo, int32_t hi) { return ((uint32_t)lo & 0xffffu) | ((uint32_t)hi << 16); }
+
+// Streamed matmul operands (h, m) live in global memory already in the shared-memory image the MMA reads:
+// 128-row x 128-byte k-blocks, [row tile][k-block][row][128 B], 16-byte chunks swizzled by (row mod 8) as
+// the 128-byte swizzle mode does.  A k-block (or a run of them) is then one contiguous bulk copy, which
+// streams about twice as fast per SM as a tiled tensor-map box of 128 separate 128-byte rows.
+__host__ __device__ __forceinline__ size_t tile_off(int row, int k, int nkb)
+{
+    return ((size_t)(row >> 7) * nkb + (k >> 7)) * KB_BYTES + (size_t)((row & 127) << 7) +
+           (size_t)(((((k >> 4) & 7) ^ (row & 7)) << 4) | (k & 15));
+}
+// byte offset of element (row, k) of a [rows][K] operand: plain rows at small batch, tiled otherwise
+__device__ __forceinline__ size_t operand_off(const RecParams &p, int row, int k, int K, int nkb)
+{
+    return p.small ? (size_t)row * K + k : tile_off(row, k, nkb);
+}
 
 // Phase A epilogue for one thread = one batch row and a range of 8-column groups of this CTA's gate sums.
 //   out = sat16( X + sat16(rescale(sat32(acc + bh), eff_h)) )            (no peephole: final gate sum, int16)
@@ -223,27 +244,34 @@ __device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, 
     }
 }
 
-// Phase C epilogue for one thread = one batch row: PN outputs of the projection tile.
-__device__ __forceinline__ void phase_c_row(const RecParams &p, uint32_t taddr, int b, int t, int p0, int8_t *h_next,
-                                            bool row_valid)
+// Phase C epilogue for one thread = one batch row and the columns [c_begin, c_end) of the projection tile, four at
+// a time: sum of the issuers' partial accumulators + folded bias (saturating) -> rescale -> + zp_h -> int8.
+__device__ __forceinline__ void phase_c_row(const RecParams &p, uint32_t taddr, int n_acc, int b, int t, int p0, int c_begin,
+                                            int c_end, int8_t *h_next, bool row_valid)
 {
-    for (int col = 0; col < p.pn; col += 16) {
-        uint32_t r[16];
-        __syncwarp();
-        ptx::tmem_ld_32x16(taddr + (uint32_t)col, r);
-        ptx::tmem_ld_wait();
-        if (!row_valid || p0 + col >= p.O) continue;
-        uint32_t w[4] = {0, 0, 0, 0};
+    for (int col = c_begin; col < c_end; col += 4) {
+        uint32_t r[4][4];
+        __syncwarp();                                        // the TMEM loads are warp-collective
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            // O is a multiple of 16, so a 16-wide group is either fully inside or fully outside
-            const int32_t acc = add_sat((int32_t)r[j], __ldg(p.bp + p0 + col + j));
+        for (int a = 0; a < 4; ++a)
+            if (a < n_acc) ptx::tmem_ld_32x4(taddr + (uint32_t)(a * p.pn + col), r[a]);   // warp-uniform
+        ptx::tmem_ld_wait();
+        if (!row_valid || p0 + col >= p.O) continue;         // O is a multiple of 16: a group of 4 is inside or outside
+        const int4 bias = __ldg(reinterpret_cast<const int4 *>(p.bp + p0 + col));
+        const int32_t bb[4] = {bias.x, bias.y, bias.z, bias.w};
+        uint32_t w = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            int32_t sum = (int32_t)r[0][j];
+#pragma unroll
+            for (int a = 1; a < 4; ++a)
+                if (a < n_acc) sum += (int32_t)r[a][j];      // partial sums of the other issuers (exact in int32)
+            const int32_t acc = add_sat(sum, bb[j]);
             const int32_t hq = sat8(rescale_sel(acc, p.eff_proj, p.f_proj, p.fast_rescale_ok) + p.zp_h);
-            w[j >> 2] |= (uint32_t)(hq & 0xff) << (8 * (j & 3));
+            w |= (uint32_t)(hq & 0xff) << (8 * j);
         }
-        const uint4 v = make_uint4(w[0], w[1], w[2], w[3]);
-        *reinterpret_cast<uint4 *>(h_next + (size_t)b * p.O + p0 + col) = v;
-        *reinterpret_cast<uint4 *>(p.y + ((size_t)t * p.B + b) * p.O + p0 + col) = v;
+        *reinterpret_cast<uint32_t *>(h_next + tile_off(b, p0 + col, p.kb_h)) = w;
+        *reinterpret_cast<uint32_t *>(p.y + ((size_t)t * p.B + b) * p.O + p0 + col) = w;
     }
 }
 
@@ -272,13 +300,13 @@ __device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, const long long 
                                                    int slot)
 {
     warp_reduce_stats<G>(ctl, sum, sq);
-    __syncthreads();
+    ptx::cta_sync();
     if (threadIdx.x < G) {
         long long a = 0, b = 0;
         for (int w = 0; w < RTHREADS / 32; ++w) { a += ctl->red_sum[w][threadIdx.x]; b += ctl->red_sq[w][threadIdx.x]; }
         ctl->ln_rows[slot][threadIdx.x] = make_ln_row(ln_stats(a, b, n));
     }
-    __syncthreads();
+    ptx::cta_sync();
 }
 
 // G int16 values of two adjacent cells (cell index even): v[k][gi]
@@ -310,9 +338,9 @@ __device__ __forceinline__ void store_hidden_pair(const RecParams &p, int b, int
 {
     const uint16_t v = (uint16_t)((m0 & 0xff) | ((m1 & 0xff) << 8));
     if (p.flags & F_PROJECTION) {
-        *reinterpret_cast<uint16_t *>(p.mbuf + (size_t)b * p.C + u) = v;
+        *reinterpret_cast<uint16_t *>(p.mbuf + operand_off(p, b, u, p.C, p.kb_c)) = v;
     } else {
-        *reinterpret_cast<uint16_t *>(h_next + (size_t)b * p.O + u) = v;
+        *reinterpret_cast<uint16_t *>(h_next + operand_off(p, b, u, p.O, p.kb_h)) = v;
         *reinterpret_cast<uint16_t *>(p.y + ((size_t)t * p.B + b) * p.O + u) = v;
     }
 }
@@ -401,14 +429,14 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, in
                 }
             }
             warp_reduce_stats<G>(ctl, sum, sq);
-            __syncthreads();
+            ptx::cta_sync();
             if (threadIdx.x < nrows * 4 && (threadIdx.x & 3) < G) {
                 const int rr = threadIdx.x >> 2, g = threadIdx.x & 3;
                 long long a = 0, b = 0;
                 for (int w = rr * wpr; w < (rr + 1) * wpr; ++w) { a += ctl->red_sum[w][g]; b += ctl->red_sq[w][g]; }
                 ctl->ln_rows[rr][g] = make_ln_row(ln_stats(a, b, p.C));
             }
-            __syncthreads();
+            ptx::cta_sync();
         }
         const int j0 = i0 > rb * p.C ? i0 : rb * p.C;
         const int j1 = i1 < (re + 1) * p.C ? i1 : (re + 1) * p.C;
@@ -416,7 +444,7 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, in
             const int b = i / p.C, u = i - b * p.C;
             cell_pair<G, LN, PEEP>(p, ctl->ln_rows[b - rb], b, u, t, h_next);
         }
-        if (LN) __syncthreads();      // the statistics slots are reused by the next batch of rows
+        if (LN) ptx::cta_sync();      // the statistics slots are reused by the next batch of rows
     }
 }
 
@@ -469,7 +497,7 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
             sum_o[SO] += v;
             sq_o[SO] += (long long)(v * v);
         }
-        __syncthreads();              // statistics of i, f, z are consumed; their slots are reused for o
+        ptx::cta_sync();              // statistics of i, f, z are consumed; their slots are reused for o
         block_reduce_stats<G>(ctl, sum_o, sq_o, p.C, 0);
         for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
             const int n = u * G + SO;
@@ -477,13 +505,13 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
             const int32_t o = sigmoid_q_fast(ao, 3);
             const int32_t m = hidden_q_fast(o, cnew_s[u], p.m_bits, p.eff_m, p.f_m, p.zp_m);
             if (p.flags & F_PROJECTION) {
-                p.mbuf[(size_t)b * p.C + u] = (int8_t)m;
+                p.mbuf[operand_off(p, b, u, p.C, p.kb_c)] = (int8_t)m;
             } else {
-                h_next[(size_t)b * p.O + u] = (int8_t)m;
+                h_next[operand_off(p, b, u, p.O, p.kb_h)] = (int8_t)m;
                 p.y[((size_t)t * p.B + b) * p.O + u] = (int8_t)m;
             }
         }
-        __syncthreads();
+        ptx::cta_sync();
     }
 }
 
@@ -513,7 +541,7 @@ __device__ __forceinline__ void stage_rows(int8_t *dst_s, const int8_t *src, int
     const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
     uint4 *d4 = reinterpret_cast<uint4 *>(dst_s);
     for (int i = threadIdx.x; i < (bytes >> 4); i += RTHREADS) d4[i] = __ldcg(s4 + i);   // L2 loads: written by other CTAs this step
-    __syncthreads();
+    ptx::cta_sync();
 }
 
 template <int BMAX>
@@ -542,7 +570,7 @@ template <int BMAX>
 __device__ __forceinline__ void phase_a_small(const RecParams &p, int t, int cur, int n0, int n_cnt, const int8_t *R_s,
                                               int8_t *stage_s, const int32_t *bh_s)
 {
-    stage_rows(stage_s, p.hbuf + (size_t)cur * p.Bpad * p.O, p.B * p.O);
+    stage_rows(stage_s, p.hbuf + (size_t)cur * p.h_stride, p.B * p.O);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const bool peep = (p.flags & F_PEEPHOLE) != 0;
     for (int n = warp; n < n_cnt; n += RTHREADS / 32) {
@@ -577,17 +605,76 @@ __device__ __forceinline__ void phase_c_small(const RecParams &p, int t, int p_l
 }
 
 // ------------------------------------------------------------------------------------------------
+// Operand ring of the tensor-core phases.  Chunks (up to STAGE_KB k-blocks, contiguous in the tiled global
+// image) are numbered by a per-CTA sequence number that runs over both matmul phases of all steps:
+// stage = seq mod stages, mbarrier parity = (seq / stages) mod 2; stages is a power of two.
+// One producer thread issues the bulk copies; several issuer threads (one per accumulator) consume the
+// chunks: a single thread's issue latency (wait, descriptors, 4 MMAs per k-block, commit), not the copy
+// rate, is what bounds a one-issuer loop.
+
+struct Ring {
+    uint8_t *base;
+    uint32_t mask, log2;
+};
+
+// producer: chunk i of the phase (i < n) is `bytes_of(i)` bytes at src_of(i)
+__device__ __forceinline__ void ring_produce(RecCtl *ctl, const Ring &r, uint32_t seq0, int n, int kb_total, int chunks_per_tile,
+                                             const int8_t *src, volatile int *abort_flag)
+{
+    // tile j of the operand starts at src + j * kb_total * KB_BYTES; its chunks are consecutive
+    int tile = 0, ci = 0;
+    for (int i = 0; i < n; ++i) {
+        const uint32_t seq = seq0 + (uint32_t)i, stage = seq & r.mask, par = (seq >> r.log2) & 1u;
+        const int kb = ci * STAGE_KB;
+        const uint32_t bytes = (uint32_t)((kb_total - kb < STAGE_KB ? kb_total - kb : STAGE_KB) * KB_BYTES);
+        if (!wait_or_abort(&ctl->empty[stage], par ^ 1u, abort_flag)) return;
+        ptx::mbar_arrive_expect_tx(&ctl->full[stage], bytes);
+        ptx::bulk_load_1d(r.base + (size_t)stage * STAGE_BYTES, src + ((size_t)tile * kb_total + kb) * KB_BYTES, bytes, &ctl->full[stage]);
+        if (++ci == chunks_per_tile) { ci = 0; ++tile; }
+    }
+}
+
+// issuer: chunks first, first + stride, ... < n of the phase, all k-blocks of each into accumulator d_tmem.
+// b_base is the shared-memory address of the resident B operand, b_kb_bytes its bytes per k-block.
+// kb0_of_first is the k-block index (within the tile) of chunk `first`; consecutive chunks of one issuer are
+// `stride` chunks apart in the same tile.
+__device__ __forceinline__ bool ring_issue(RecCtl *ctl, const Ring &r, uint32_t seq0, int first, int n, int stride, int kb0,
+                                           int kb_total, uint32_t b_base, uint32_t b_kb_bytes, uint32_t d_tmem, uint32_t idesc,
+                                           volatile int *abort_flag)
+{
+    const uint64_t a_desc0 = ptx::smem_desc_k_sw128(ptx::smem_u32(r.base));
+    const uint64_t b_desc0 = ptx::smem_desc_k_sw128(b_base);
+    bool acc = false;
+    for (int i = first; i < n; i += stride, kb0 += stride * STAGE_KB) {
+        const uint32_t seq = seq0 + (uint32_t)i, stage = seq & r.mask, par = (seq >> r.log2) & 1u;
+        if (!wait_or_abort(&ctl->full[stage], par, abort_flag)) return false;
+        ptx::tc_fence_after();
+        uint64_t a_desc = a_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
+        uint64_t b_desc = b_desc0 + (uint64_t)(((uint32_t)kb0 * b_kb_bytes) >> 4);
+        const int nk = kb_total - kb0 < STAGE_KB ? kb_total - kb0 : STAGE_KB;
+        for (int j = 0; j < nk; ++j) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                ptx::mma_i8_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, acc);
+                acc = true;
+            }
+            a_desc += KB_BYTES >> 4;
+            b_desc += b_kb_bytes >> 4;
+        }
+        ptx::mma_commit(&ctl->empty[stage]);
+    }
+    return true;
+}
 
 __global__ void __launch_bounds__(RTHREADS, 1)
-k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_R,
-                  const __grid_constant__ CUtensorMap map_m, const __grid_constant__ CUtensorMap map_Wp, RecParams p)
+k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_constant__ CUtensorMap map_Wp, RecParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const bool proj = (p.flags & F_PROJECTION) != 0;
     // layout: [ring stages][R slice][Wproj slice][row buffer][bias slice][control]
     uint8_t *ring = smem;
-    uint8_t *R_s = ring + (size_t)p.stages * A_STAGE_BYTES;
+    uint8_t *R_s = ring + (size_t)p.stages * STAGE_BYTES;
     uint8_t *Wp_s = R_s + (size_t)p.kb_h * p.nc_pad * 128;
     uint8_t *after_w = Wp_s + (proj ? (size_t)p.kb_c * p.pn * 128 : 0);
     int16_t *row_s = (int16_t *)after_w;
@@ -606,17 +693,20 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
     const int tile_mi = has_ptile ? cta / p.npn : 0, tile_p0 = has_ptile ? (cta % p.npn) * p.pn : 0;
     const uint32_t acc_cols_a = (uint32_t)(p.MT * p.nc_pad);
     uint32_t tmem_cols = 32;
-    while (tmem_cols < acc_cols_a + (uint32_t)(proj ? p.pn : 0)) tmem_cols <<= 1;
+    while (tmem_cols < acc_cols_a + (uint32_t)(proj ? p.pn * p.n_issue_c : 0)) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&ctl->full[s], 1); ptx::mbar_init(&ctl->empty[s], 1); }
-        for (int i = 0; i < 3; ++i) ptx::mbar_init(&ctl->acc_full[i], 1);
+        for (int i = 0; i < 2; ++i) ptx::mbar_init(&ctl->acc_full[i], 1);
+        {
+            const int nc = (p.kb_c + STAGE_KB - 1) / STAGE_KB;
+            ptx::mbar_init(&ctl->acc_full[2], (uint32_t)(nc < p.n_issue_c ? nc : p.n_issue_c));      // one arrival per projection issuer
+        }
         ptx::mbar_init(&ctl->w_full, 1);
         ctl->abort_flag = 0;
         ptx::fence_barrier_init();
-        ptx::prefetch_tensormap(&map_h);
         ptx::prefetch_tensormap(&map_R);
-        if (proj) { ptx::prefetch_tensormap(&map_m); ptx::prefetch_tensormap(&map_Wp); }
+        if (proj) ptx::prefetch_tensormap(&map_Wp);
     }
     if (warp == 1) {
         ptx::tmem_alloc(&ctl->tmem_base, tmem_cols);
@@ -624,7 +714,7 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
     }
     for (int i = threadIdx.x; i < p.nc_pad; i += RTHREADS) bh_s[i] = (has_cells && i < n_cnt) ? p.bh[n0 + i] : 0;
     ptx::tc_fence_before();
-    __syncthreads();
+    ptx::cta_sync();
     ptx::tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
@@ -660,10 +750,15 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
         }
     }
     if (warp == 1 && lane == 0) wait_or_abort(&ctl->w_full, 0, abort_flag);
-    __syncthreads();
+    ptx::cta_sync();
 
     unsigned epoch = 0;
-    int stage = 0; uint32_t ring_phase = 0;      // advanced identically by producer and MMA issuer
+    uint32_t seq = 0;                            // chunks this CTA has put through the ring so far (uniform over its threads)
+    Ring rg;
+    rg.base = ring; rg.mask = (uint32_t)p.stages - 1u; rg.log2 = (uint32_t)__ffs(p.stages) - 1u;
+    const int cpt_a = (p.kb_h + STAGE_KB - 1) / STAGE_KB, n_chunks_a = p.MT * cpt_a;      // recurrent matmul: chunks per batch tile
+    const int n_chunks_c = (p.kb_c + STAGE_KB - 1) / STAGE_KB;
+    const int n_issue_c = n_chunks_c < p.n_issue_c ? n_chunks_c : p.n_issue_c;
     const uint32_t idesc_a = ptx::idesc_i8(128, p.nc_pad), idesc_c = ptx::idesc_i8(128, p.pn);
 
     const bool timing = p.phase_ns != nullptr && cta == 0 && threadIdx.x == 0;
@@ -678,7 +773,7 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
 
     for (int t = 0; t < p.T; ++t) {
         const int cur = t & 1;
-        int8_t *h_next = p.hbuf + (size_t)(cur ^ 1) * p.Bpad * p.O;
+        int8_t *h_next = p.hbuf + (size_t)(cur ^ 1) * p.h_stride;
         const uint32_t par = (uint32_t)t & 1u;
 
         // ================= phase A: gate sums =================
@@ -693,37 +788,18 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
         } else if (has_cells) {
             if (warp == 0) {
                 if (lane == 0) {
-                    fence_proxy_async_all();
-                    for (int mi = 0; mi < p.MT && !*abort_flag; ++mi)
-                        for (int kb = 0; kb < p.kb_h; ++kb) {
-                            if (!wait_or_abort(&ctl->empty[stage], ring_phase ^ 1, abort_flag)) break;
-                            ptx::mbar_arrive_expect_tx(&ctl->full[stage], A_STAGE_BYTES);
-                            ptx::tma_load_2d(ring + (size_t)stage * A_STAGE_BYTES, &map_h, &ctl->full[stage], kb * 128,
-                                             cur * p.Bpad + mi * 128);
-                            if (++stage == p.stages) { stage = 0; ring_phase ^= 1; }
-                        }
+                    fence_proxy_async_global();
+                    ring_produce(ctl, rg, seq, n_chunks_a, p.kb_h, cpt_a, p.hbuf + (size_t)cur * p.h_stride, abort_flag);
                 }
                 __syncwarp();
-            } else if (warp == 1) {
-                if (lane == 0) {
+            } else if (warp == 1 || warp == 18) {
+                // one issuer per batch tile, each with its own accumulator
+                const int mi = warp == 1 ? 0 : 1;
+                if (lane == 0 && mi < p.MT) {
                     ptx::tc_fence_after();
-                    for (int mi = 0; mi < p.MT && !*abort_flag; ++mi) {
-                        bool ok = true;
-                        for (int kb = 0; kb < p.kb_h; ++kb) {
-                            if (!wait_or_abort(&ctl->full[stage], ring_phase, abort_flag)) { ok = false; break; }
-                            ptx::tc_fence_after();
-                            const uint64_t a_desc = ptx::smem_desc_k_sw128(ptx::smem_u32(ring + (size_t)stage * A_STAGE_BYTES));
-                            const uint64_t b_desc = ptx::smem_desc_k_sw128(ptx::smem_u32(R_s + (size_t)kb * p.nc_pad * 128));
-#pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                ptx::mma_i8_ss(tmem_base + (uint32_t)(mi * p.nc_pad), a_desc + 2 * k, b_desc + 2 * k, idesc_a,
-                                               (kb | k) != 0);
-                            ptx::mma_commit(&ctl->empty[stage]);
-                            if (++stage == p.stages) { stage = 0; ring_phase ^= 1; }
-                        }
-                        if (!ok) break;
+                    if (ring_issue(ctl, rg, seq + (uint32_t)(mi * cpt_a), 0, cpt_a, 1, 0, p.kb_h, ptx::smem_u32(R_s),
+                                   (uint32_t)p.nc_pad * 128u, tmem_base + (uint32_t)(mi * p.nc_pad), idesc_a, abort_flag))
                         ptx::mma_commit(&ctl->acc_full[mi]);
-                    }
                 }
                 __syncwarp();
             } else if (warp < 18) {
@@ -747,17 +823,18 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
                 }
             }
         }
-        __syncthreads();
+        if (!p.small && has_cells) seq += (uint32_t)n_chunks_a;
+        ptx::cta_sync();
         lap(0);
-        grid_sync(p, epoch, abort_flag);
+        grid_sync(p, epoch, abort_flag, false);
         lap(1);
         if (*abort_flag) break;
 
         // ================= phase B: elementwise =================
         phase_b(p, ctl, t, h_next, row_s);
-        __syncthreads();
+        ptx::cta_sync();
         lap(2);
-        grid_sync(p, epoch, abort_flag);
+        grid_sync(p, epoch, abort_flag, !p.small);
         lap(3);
         if (*abort_flag) break;
 
@@ -774,63 +851,78 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_h, const __grid_consta
             } else if (has_ptile) {
                 if (warp == 0) {
                     if (lane == 0) {
-                        fence_proxy_async_all();
-                        for (int kb = 0; kb < p.kb_c; ++kb) {
-                            if (!wait_or_abort(&ctl->empty[stage], ring_phase ^ 1, abort_flag)) break;
-                            ptx::mbar_arrive_expect_tx(&ctl->full[stage], A_STAGE_BYTES);
-                            ptx::tma_load_2d(ring + (size_t)stage * A_STAGE_BYTES, &map_m, &ctl->full[stage], kb * 128,
-                                             tile_mi * 128);
-                            if (++stage == p.stages) { stage = 0; ring_phase ^= 1; }
-                        }
+                        fence_proxy_async_global();
+                        ring_produce(ctl, rg, seq, n_chunks_c, p.kb_c, n_chunks_c, p.mbuf + (size_t)tile_mi * p.kb_c * KB_BYTES, abort_flag);
                     }
                     __syncwarp();
-                } else if (warp == 1) {
-                    if (lane == 0) {
-                        ptx::tc_fence_after();
-                        bool ok = true;
-                        for (int kb = 0; kb < p.kb_c; ++kb) {
-                            if (!wait_or_abort(&ctl->full[stage], ring_phase, abort_flag)) { ok = false; break; }
+                } else {
+                    // several issuers share the K range: issuer w takes chunks w, w + n_issue_c, ... into its own
+                    // accumulator; the epilogue adds the partial sums (exact in int32).  Issuers are the three warps
+                    // without an epilogue role and, for a fourth, the last epilogue warp before it turns to its part
+                    const int w = warp == 1 ? 0 : warp == 18 ? 1 : warp == 19 ? 2 : warp == 17 ? 3 : 4;
+                    if (w < n_issue_c) {
+                        if (lane == 0) {
                             ptx::tc_fence_after();
-                            const uint64_t a_desc = ptx::smem_desc_k_sw128(ptx::smem_u32(ring + (size_t)stage * A_STAGE_BYTES));
-                            const uint64_t b_desc = ptx::smem_desc_k_sw128(ptx::smem_u32(Wp_s + (size_t)kb * p.pn * 128));
-#pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                ptx::mma_i8_ss(tmem_base + acc_cols_a, a_desc + 2 * k, b_desc + 2 * k, idesc_c, (kb | k) != 0);
-                            ptx::mma_commit(&ctl->empty[stage]);
-                            if (++stage == p.stages) { stage = 0; ring_phase ^= 1; }
+                            if (ring_issue(ctl, rg, seq, w, n_chunks_c, n_issue_c, w * STAGE_KB, p.kb_c, ptx::smem_u32(Wp_s),
+                                           (uint32_t)p.pn * 128u, tmem_base + acc_cols_a + (uint32_t)(w * p.pn), idesc_c, abort_flag))
+                                ptx::mma_commit(&ctl->acc_full[2]);
                         }
-                        if (ok) ptx::mma_commit(&ctl->acc_full[2]);
+                        __syncwarp();
                     }
-                    __syncwarp();
-                } else if (warp - 2 < 4) {
-                    const int quarter = warp & 3;
-                    if (__all_sync(0xffffffffu, wait_or_abort(&ctl->acc_full[2], par, abort_flag))) {
-                        ptx::tc_fence_after();
-                        const int b = tile_mi * 128 + quarter * 32 + lane;
-                        phase_c_row(p, tmem_base + ((uint32_t)(quarter * 32) << 16) + acc_cols_a, b, t, tile_p0, h_next, b < p.B);
-                        ptx::tc_fence_before();
+                    if (warp >= 2 && warp < 18) {
+                        // 16 epilogue warps: 4 TMEM lane quarters x 4 column parts of the tile
+                        const int quarter = warp & 3, part = (warp - 2) >> 2;
+                        const int ngroups = p.pn >> 2;
+                        const int c_begin = 4 * (part * ngroups / 4), c_end = 4 * ((part + 1) * ngroups / 4);
+                        if (__all_sync(0xffffffffu, wait_or_abort(&ctl->acc_full[2], par, abort_flag))) {
+                            ptx::tc_fence_after();
+                            const int b = tile_mi * 128 + quarter * 32 + lane;
+                            phase_c_row(p, tmem_base + ((uint32_t)(quarter * 32) << 16) + acc_cols_a, n_issue_c, b, t, tile_p0, c_begin,
+                                        c_end, h_next, b < p.B);
+                            ptx::tc_fence_before();
+                        }
                     }
                 }
             }
-            __syncthreads();
+            if (!p.small && has_ptile) seq += (uint32_t)n_chunks_c;
+            ptx::cta_sync();
             lap(4);
-            grid_sync(p, epoch, abort_flag);
+            grid_sync(p, epoch, abort_flag, !p.small && warp >= 2);      // the epilogue warps wrote h
             lap(5);
             if (*abort_flag) break;
         }
     }
 
     // ---------------- teardown ----------------
-    __syncthreads();
+    ptx::cta_sync();
     if (*abort_flag) {
         for (int i = 0; i < 200; ++i) __nanosleep(500);      // let copies in flight land before the CTA retires
         if (threadIdx.x == 0) atomicExch(p.status, 2);
     }
-    __syncthreads();
+    ptx::cta_sync();
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, tmem_cols);
     }
+}
+
+// Caller's h [B][K] (plain rows) -> tiled operand image, 16 bytes per thread.
+__global__ void k_tile_rows(const int8_t *src, int8_t *dst, int B, int K, int nkb, bool aligned)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int per_row = K >> 4;
+    if (i >= B * per_row) return;
+    const int row = i / per_row, k = (i - row * per_row) << 4;
+    const int8_t *s = src + (size_t)row * K + k;
+    uint4 v;
+    if (aligned) {
+        v = *reinterpret_cast<const uint4 *>(s);
+    } else {
+        uint32_t w[4] = {0, 0, 0, 0};
+        for (int j = 0; j < 16; ++j) w[j >> 2] |= (uint32_t)(uint8_t)s[j] << (8 * (j & 3));
+        v = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    *reinterpret_cast<uint4 *>(dst + tile_off(row, k, nkb)) = v;
 }
 
 size_t rec_smem_bytes(const LayerParams &p, int stages, int nc_pad, int pn, int kb_h, int kb_c)
@@ -838,7 +930,7 @@ size_t rec_smem_bytes(const LayerParams &p, int stages, int nc_pad, int pn, int 
     const bool proj = (p.flags & F_PROJECTION) != 0;
     size_t row_bytes = ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE)) ? ((size_t)p.C * p.G + p.C) * 2 : 0;
     row_bytes = (row_bytes + 15) & ~(size_t)15;
-    return 1024 + (size_t)stages * A_STAGE_BYTES + (size_t)kb_h * nc_pad * 128 + (proj ? (size_t)kb_c * pn * 128 : 0) +
+    return 1024 + (size_t)stages * STAGE_BYTES + (size_t)kb_h * nc_pad * 128 + (proj ? (size_t)kb_c * pn * 128 : 0) +
            row_bytes + (size_t)nc_pad * 4 + sizeof(RecCtl) + 64;
 }
 
@@ -850,8 +942,8 @@ int fast_scratch_init(FastScratch &s, int max_B, int maxC, int maxO, int maxN, i
 {
     s.Bpad = round_up(max_B, 128);
     s.sm_count = sm_count;
-    s.hbuf_bytes = (size_t)2 * s.Bpad * maxO;
-    s.mbuf_bytes = (size_t)s.Bpad * maxC;
+    s.hbuf_bytes = (size_t)2 * s.Bpad * round_up(maxO, 128);      // whole 128 x 128-byte k-blocks
+    s.mbuf_bytes = (size_t)s.Bpad * round_up(maxC, 128);
     if (cudaMalloc(&s.hbuf, s.hbuf_bytes) != cudaSuccess) return QLSTM_ERR_NOMEM;
     if (cudaMalloc(&s.mbuf, s.mbuf_bytes) != cudaSuccess) return QLSTM_ERR_NOMEM;
     if (cudaMalloc(&s.pre, (size_t)max_B * maxN * sizeof(int32_t)) != cudaSuccess) return QLSTM_ERR_NOMEM;
@@ -894,22 +986,22 @@ int fast_recurrent_init(FastLayer &f, const LayerParams &p, const FastScratch &s
         f.npn = (p.O + pn - 1) / pn;
     }
     if (MT_max * f.nc_pad + f.pn > 512) return QLSTM_OK;
+    f.n_issue_c = 1;
+    if (proj)
+        while (f.n_issue_c < 4 && MT_max * f.nc_pad + f.pn * f.n_issue_c * 2 <= 512) f.n_issue_c *= 2;
     int dev = 0, max_smem = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    int stages = MAX_STAGES;
-    while (stages >= 2 && rec_smem_bytes(p, stages, f.nc_pad, f.pn, f.kb_h, f.kb_c) > (size_t)max_smem) --stages;
+    int stages = MAX_STAGES;                      // a power of two
+    while (stages >= 2 && rec_smem_bytes(p, stages, f.nc_pad, f.pn, f.kb_h, f.kb_c) > (size_t)max_smem) stages >>= 1;
     if (stages < 2) return QLSTM_OK;
     f.stages = stages;
     f.smem = rec_smem_bytes(p, stages, f.nc_pad, f.pn, f.kb_h, f.kb_c);
     if (!make_tensor_map_i8(&f.map_R, p.R, (uint64_t)p.N, (uint64_t)p.O, (uint32_t)f.nc_pad, 128)) return QLSTM_OK;
-    if (!make_tensor_map_i8(&f.map_h, s.hbuf, (uint64_t)2 * s.Bpad, (uint64_t)p.O, 128, 128)) return QLSTM_OK;
     if (proj) {
         if (!make_tensor_map_i8(&f.map_Wp, p.Wproj, (uint64_t)p.O, (uint64_t)p.C, (uint32_t)f.pn, 128)) return QLSTM_OK;
-        if (!make_tensor_map_i8(&f.map_m, s.mbuf, (uint64_t)s.Bpad, (uint64_t)p.C, 128, 128)) return QLSTM_OK;
     } else {
         f.map_Wp = f.map_R;
-        f.map_m = f.map_h;
     }
     if (cudaFuncSetAttribute(k_recurrent_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
         return QLSTM_OK;
@@ -939,11 +1031,12 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     RecParams rp;
     memset(&rp, 0, sizeof(rp));
     rp.T = T; rp.B = B; rp.MT = (B + 127) / 128; rp.Bpad = s.Bpad;
+    rp.h_stride = (size_t)s.Bpad * f.kb_h * 128;
     rp.C = p.C; rp.O = p.O; rp.G = p.G; rp.N = p.N;
     rp.flags = p.flags; rp.m_bits = p.m_bits; rp.zp_m = p.zp_m; rp.zp_h = p.zp_h;
     rp.cpc = f.cpc; rp.n_cta_a = f.n_cta_a; rp.nc_pad = f.nc_pad;
     rp.pn = f.pn; rp.npn = f.npn; rp.n_ptiles = rp.MT * f.npn;
-    rp.kb_h = f.kb_h; rp.kb_c = f.kb_c; rp.stages = f.stages;
+    rp.kb_h = f.kb_h; rp.kb_c = f.kb_c; rp.stages = f.stages; rp.n_issue_c = f.n_issue_c;
     // elementwise phase: contiguous ranges of the B x C cell grid (whole rows with layer norm + peephole)
     if ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE))
         rp.items_per_cta = ((B + f.grid - 1) / f.grid) * p.C;
@@ -953,7 +1046,7 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     rp.rpc = (p.O + f.grid - 1) / f.grid;
     {
         const int maxk = p.O > p.C ? p.O : p.C;
-        const bool fits = (size_t)16 * maxk <= (size_t)f.stages * A_STAGE_BYTES && (!(p.flags & F_PROJECTION) || rp.rpc <= f.pn);
+        const bool fits = (size_t)16 * maxk <= (size_t)f.stages * STAGE_BYTES && (!(p.flags & F_PROJECTION) || rp.rpc <= f.pn);
         rp.small = (allow_small && B <= 16 && fits) ? 1 : 0;
     }
     rp.fast_rescale_ok = 1;
@@ -978,17 +1071,26 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
 
     // h^{-1} into operand buffer 0; barrier words cleared
     if (cudaMemsetAsync(s.bar, 0, 64, st) != cudaSuccess) return QLSTM_ERR_CUDA;
-    if (cudaMemcpyAsync(s.hbuf, h, (size_t)B * p.O, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return QLSTM_ERR_CUDA;
+    int n_launch = 1;
+    if (rp.small) {
+        if (cudaMemcpyAsync(s.hbuf, h, (size_t)B * p.O, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return QLSTM_ERR_CUDA;
+    } else {
+        const int chunks = B * (p.O >> 4);
+        k_tile_rows<<<(chunks + 255) / 256, 256, 0, st>>>(h, s.hbuf, B, p.O, f.kb_h, ((uintptr_t)h & 15) == 0);
+        if (cudaGetLastError() != cudaSuccess) return QLSTM_ERR_CUDA;
+        ++n_launch;
+    }
 
-    void *args[] = {(void *)&f.map_h, (void *)&f.map_R, (void *)&f.map_m, (void *)&f.map_Wp, (void *)&rp};
+    void *args[] = {(void *)&f.map_R, (void *)&f.map_Wp, (void *)&rp};
     cudaError_t e = cudaLaunchCooperativeKernel((const void *)k_recurrent_sm100, dim3(f.grid), dim3(RTHREADS), args, f.smem, st);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return e == cudaErrorCooperativeLaunchTooLarge ? QLSTM_ERR_LAUNCH : QLSTM_ERR_CUDA;
     }
-    if (cudaMemcpyAsync(h, s.hbuf + (size_t)(T & 1) * s.Bpad * p.O, (size_t)B * p.O, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    // h^{T-1} is the last row block of y
+    if (T > 0 && cudaMemcpyAsync(h, y + (size_t)(T - 1) * B * p.O, (size_t)B * p.O, cudaMemcpyDeviceToDevice, st) != cudaSuccess)
         return QLSTM_ERR_CUDA;
-    if (launches) *launches = 1;
+    if (launches) *launches = n_launch;
     return QLSTM_OK;
 }
 
