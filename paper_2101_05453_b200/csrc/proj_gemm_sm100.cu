@@ -62,15 +62,16 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
     return false;
 }
 
-template <int G>
-__device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], const int32_t *bias, const ProjParams &p,
+// 16 adjacent columns of one output row: + folded bias -> rescale -> sat16 -> one 32-byte store.
+template <int G, bool GENERIC>
+__device__ __forceinline__ void epilogue_piece(const uint32_t (&r)[16], const int32_t *bias, const ProjParams &p,
                                                int n_first, int16_t *dst, int n_valid, bool wide_ok)
 {
-    // column j of this chunk is global column n_first + j; its gate slot is (n_first + j) % G
-    uint32_t packed[16];
+    // column j of this piece is global column n_first + j; its gate slot is (n_first + j) % G
+    uint32_t packed[8];
     const int phase = n_first % G;
 #pragma unroll
-    for (int j = 0; j < 32; j += 4) {
+    for (int j = 0; j < 16; j += 4) {
         const int4 b4 = *reinterpret_cast<const int4 *>(bias + j);
         const int32_t bb[4] = {b4.x, b4.y, b4.z, b4.w};
         int32_t y[4];
@@ -78,27 +79,26 @@ __device__ __forceinline__ void epilogue_chunk(const uint32_t (&r)[32], const in
         for (int i = 0; i < 4; ++i) {
             const int32_t v = (int32_t)r[j + i] + bb[i];          // |acc| + |bias| < 2^30: no overflow
             const int g = (G == 4) ? i : (phase + j + i) % 3;
-            y[i] = p.generic ? mbqm(v, p.sc[g]) : fast_rescale(v, p.fs[g]);
+            y[i] = GENERIC ? mbqm(v, p.sc[g]) : fast_rescale(v, p.fs[g]);
         }
         packed[j >> 1] = ptx::pack_sat_s16(y[0], y[1]);
         packed[(j >> 1) + 1] = ptx::pack_sat_s16(y[2], y[3]);
     }
-    if (n_valid >= 32 && wide_ok) {
-        // 32-byte stores: every store fills whole 32-byte sectors
-#pragma unroll
-        for (int v = 0; v < 2; ++v)
-            asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 16 * v),
-                         "r"(packed[8 * v]), "r"(packed[8 * v + 1]), "r"(packed[8 * v + 2]), "r"(packed[8 * v + 3]),
-                         "r"(packed[8 * v + 4]), "r"(packed[8 * v + 5]), "r"(packed[8 * v + 6]), "r"(packed[8 * v + 7])
-                         : "memory");
+    if (n_valid >= 16 && wide_ok) {
+        // a 32-byte store fills a whole sector
+        asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(packed[0]), "r"(packed[1]),
+                     "r"(packed[2]), "r"(packed[3]), "r"(packed[4]), "r"(packed[5]), "r"(packed[6]), "r"(packed[7])
+                     : "memory");
         return;
     }
 #pragma unroll
-    for (int v = 0; v < 4; ++v)
+    for (int v = 0; v < 2; ++v)
         if (8 * v + 8 <= n_valid)
             *reinterpret_cast<uint4 *>(dst + 8 * v) = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
 }
 
+// G: gate slots per cell (4, or 3 with CIFG); GENERIC: some gate has a positive shift and takes the general rescale
+template <int G, bool GENERIC>
 __global__ void __launch_bounds__(THREADS, 1)
 k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w, ProjParams p)
 {
@@ -210,43 +210,44 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
         const int c0 = 2 * cgrp, c1 = 2 * cgrp + 1;
         const bool has0 = c0 < n_chunks, has1 = c1 < n_chunks;
         const bool wide_ok = (p.N % 16) == 0;            // every row starts on a 32-byte boundary
-        int it = 0;
+        int it = 0, cur_n0 = -1;
         for (int t = t_begin; t < t_end; ++t, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1;
             const int n0 = (t / tiles_m) * p.bn, m0 = (t % tiles_m) * BM;
-            __syncwarp();
-            {
+            if (n0 != cur_n0) {                          // the folded bias changes only with the panel
+                __syncwarp();
                 const int na = n0 + c0 * 32 + lane, nb = n0 + c1 * 32 + lane;
                 bias[lane] = (has0 && na < p.N) ? p.bx[na] : 0;
                 bias[32 + lane] = (has1 && nb < p.N) ? p.bx[nb] : 0;
+                cur_n0 = n0;
+                __syncwarp();
             }
-            __syncwarp();
             if (!__all_sync(0xffffffffu, wait_or_abort(&ctl->tmem_full[buf], acc_phase, abort_flag))) break;
             ptx::tc_fence_after();
             const int row = m0 + quarter * 32 + lane;
             const uint32_t tbase = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.bn);
-            // the second chunk's TMEM load is in flight while the first chunk is processed
-            uint32_t r0[32], r1[32];
-            if (has0) ptx::tmem_ld_32x32(tbase + (uint32_t)(c0 * 32), r0);
-            ptx::tmem_ld_wait();
-            if (has1) ptx::tmem_ld_32x32(tbase + (uint32_t)(c1 * 32), r1);
-            if (has0) {
-                const int n_first = n0 + c0 * 32, n_valid = p.N - n_first;
-                if (row < p.M && n_valid > 0) {
-                    int16_t *dst = p.out + (size_t)row * p.N + n_first;
-                    if (p.G == 4) epilogue_chunk<4>(r0, bias, p, n_first, dst, n_valid, wide_ok);
-                    else epilogue_chunk<3>(r0, bias, p, n_first, dst, n_valid, wide_ok);
+            // the warp's 64 columns in four pieces of 16; the next piece's TMEM load is in flight while one is processed
+            uint32_t ra[16], rb[16];
+            const int np = (has0 ? 2 : 0) + (has1 ? 2 : 0);
+            const uint32_t tcol = tbase + (uint32_t)(c0 * 32);
+            const int n_base = n0 + c0 * 32;
+            int16_t *dst_row = p.out + (size_t)row * p.N + n_base;
+            const bool row_ok = row < p.M;
+            if (np > 0) ptx::tmem_ld_32x16(tcol, ra);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (i >= np) break;                                  // warp-uniform
+                ptx::tmem_ld_wait();
+                __syncwarp();
+                if (i + 1 < np) {
+                    if (i & 1) ptx::tmem_ld_32x16(tcol + (uint32_t)(16 * (i + 1)), ra);
+                    else ptx::tmem_ld_32x16(tcol + (uint32_t)(16 * (i + 1)), rb);
                 }
-            }
-            __syncwarp();
-            ptx::tmem_ld_wait();
-            if (has1) {
-                const int n_first = n0 + c1 * 32, n_valid = p.N - n_first;
-                if (row < p.M && n_valid > 0) {
-                    int16_t *dst = p.out + (size_t)row * p.N + n_first;
-                    if (p.G == 4) epilogue_chunk<4>(r1, bias + 32, p, n_first, dst, n_valid, wide_ok);
-                    else epilogue_chunk<3>(r1, bias + 32, p, n_first, dst, n_valid, wide_ok);
+                const int n_valid = p.N - (n_base + 16 * i);
+                if (row_ok && n_valid > 0) {
+                    if (i & 1) epilogue_piece<G, GENERIC>(rb, bias + 16 * i, p, n_base + 16 * i, dst_row + 16 * i, n_valid, wide_ok);
+                    else epilogue_piece<G, GENERIC>(ra, bias + 16 * i, p, n_base + 16 * i, dst_row + 16 * i, n_valid, wide_ok);
                 }
             }
             ptx::tc_fence_before();
@@ -305,7 +306,11 @@ int fast_projection_init(FastLayer &f, const LayerParams &p)
     f.proj_bn = bn;
     f.proj_stages = stages;
     if (!make_tensor_map_i8(&f.map_W, p.W, (uint64_t)p.N, (uint64_t)p.I, (uint32_t)bn, BK)) return 0;
-    if (cudaFuncSetAttribute(k_projection_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess) return 0;
+    if (cudaFuncSetAttribute(k_projection_sm100<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(k_projection_sm100<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(k_projection_sm100<3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(k_projection_sm100<3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
+        return 0;
     f.proj_ok = true;
     return 0;
 }
@@ -327,7 +332,14 @@ cudaError_t launch_projection_fast(const FastLayer &f, const LayerParams &p, con
     }
     const int tiles = ((rows + BM - 1) / BM) * ((p.N + pp.bn - 1) / pp.bn);
     const int grid = tiles < sm_count ? tiles : sm_count;
-    k_projection_sm100<<<grid, THREADS, smem_bytes(pp.bn, pp.kb, pp.stages), st>>>(map_x, f.map_W, pp);
+    const size_t smem = smem_bytes(pp.bn, pp.kb, pp.stages);
+    if (p.G == 4) {
+        if (pp.generic) k_projection_sm100<4, true><<<grid, THREADS, smem, st>>>(map_x, f.map_W, pp);
+        else k_projection_sm100<4, false><<<grid, THREADS, smem, st>>>(map_x, f.map_W, pp);
+    } else {
+        if (pp.generic) k_projection_sm100<3, true><<<grid, THREADS, smem, st>>>(map_x, f.map_W, pp);
+        else k_projection_sm100<3, false><<<grid, THREADS, smem, st>>>(map_x, f.map_W, pp);
+    }
     return cudaGetLastError();
 }
 
