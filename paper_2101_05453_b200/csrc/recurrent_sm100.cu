@@ -40,6 +40,14 @@ constexpr int STAGE_BYTES = STAGE_KB * KB_BYTES;
 constexpr int MAX_STAGES = 4;
 constexpr unsigned long long SPIN_LIMIT_NS = 2000000000ull;   // 2 s per grid barrier
 
+// How one matmul phase uses the ring: owner o of n_own (one MMA issuer each) owns the stages o, o + n_own, ...
+// (cnt[o] of them) and consumes n_chunks[o] chunks; uses[s]: times stage s is filled in the phase.
+struct RingPlan {
+    int n_own, n_max;
+    int n_chunks[4], cnt[4];
+    int uses[MAX_STAGES];
+};
+
 struct RecParams {
     int T, B, MT, Bpad;
     size_t h_stride;              // bytes between the two h operand buffers
@@ -50,8 +58,11 @@ struct RecParams {
     int pn, npn, n_ptiles;
     int kb_h, kb_c, stages;
     int n_issue_c;                // projection: MMA issuers (= partial accumulators) sharing the K range
+    RingPlan plan_a, plan_c;      // ring use of the recurrent matmul and of the projection
     int items_per_cta;            // cells of the B x C grid per CTA in the elementwise phase
     int small;                    // small batch: dp4a mat-vec with warp reductions instead of TMA + tcgen05
+    int npc;                      // gate rows per CTA = columns of its X box
+    uint32_t x_bytes;             // bytes of one X box: MT * 128 rows x npc int16
     int rpc;                      // small batch: projection rows per CTA
     const int8_t *R, *Wproj;      // packed weights (small-batch prologue copies its slices with plain loads)
     int fast_rescale_ok;          // every rescale of this layer has shift <= 0
@@ -73,8 +84,9 @@ struct RecParams {
 };
 
 struct RecCtl {
-    uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[3], w_full;
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[3], w_full, x_full;
     uint32_t tmem_base;
+    uint32_t rounds[MAX_STAGES];
     int abort_flag;
     long long red_sum[RTHREADS / 32][4], red_sq[RTHREADS / 32][4];
     LnRow ln_rows[MAX_LN_ROWS][4];
@@ -174,51 +186,30 @@ __device__ __forceinline__ size_t operand_off(const RecParams &p, int row, int k
 // Phase A epilogue for one thread = one batch row and a range of 8-column groups of this CTA's gate sums.
 //   out = sat16( X + sat16(rescale(sat32(acc + bh), eff_h)) )            (no peephole: final gate sum, int16)
 //   out = X + sat16(rescale(...))                                        (peephole: int32, finished in phase B)
-// The X values do not depend on the recurrence: the first groups are fetched before the accumulator is awaited.
-constexpr int XPRE = 2;
-
-__device__ __forceinline__ void phase_a_prefetch(const RecParams &p, int b, int t, int n0, int g_begin, int g_end,
-                                                 bool row_valid, uint4 (&xv)[XPRE])
-{
-    const int16_t *xrow = p.X + ((size_t)t * p.B + b) * p.N + n0;
-#pragma unroll
-    for (int i = 0; i < XPRE; ++i)
-        xv[i] = (row_valid && g_begin + i < g_end) ? __ldg(reinterpret_cast<const uint4 *>(xrow + 8 * (g_begin + i)))
-                                                    : make_uint4(0, 0, 0, 0);
-}
-
+// X_t of the CTA's gate rows is in shared memory, [batch row][npc] int16.  Without peephole the result replaces X
+// in place and leaves through a tensor-map store; the int32 form of the peephole variant is stored directly.
 template <int G>
-__device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, int b, int t, int n0, int g_begin,
-                                            int g_end, const int32_t *bh_s, bool row_valid, const uint4 (&xv)[XPRE])
+__device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, int b, int n0, int g_begin, int g_end,
+                                            const int32_t *bh_s, int16_t *x_s, bool row_valid)
 {
+    constexpr int NB = 2;                                    // groups per batch of tensor-memory loads
     const bool peep = (p.flags & F_PEEPHOLE) != 0;
-    const int16_t *xrow = p.X + ((size_t)t * p.B + b) * p.N + n0;
-    uint4 xn[XPRE];
-#pragma unroll
-    for (int i = 0; i < XPRE; ++i) xn[i] = xv[i];
+    int16_t *xrow = x_s + (size_t)b * p.npc;
 #pragma unroll 1
-    for (int gbase = g_begin; gbase < g_end; gbase += XPRE) {
-        // X of the next batch of groups is requested before this batch is processed
-        uint4 xc[XPRE];
-#pragma unroll
-        for (int i = 0; i < XPRE; ++i) {
-            xc[i] = xn[i];
-            if (row_valid && gbase + XPRE + i < g_end) xn[i] = __ldg(reinterpret_cast<const uint4 *>(xrow + 8 * (gbase + XPRE + i)));
-        }
-        // all TMEM loads of this batch first, one wait, then the arithmetic
-        uint32_t r[XPRE][8];
+    for (int gbase = g_begin; gbase < g_end; gbase += NB) {
+        uint32_t r[NB][8];
         __syncwarp();                                        // the TMEM loads are warp-collective
 #pragma unroll
-        for (int i = 0; i < XPRE; ++i)
+        for (int i = 0; i < NB; ++i)
             if (gbase + i < g_end) ptx::tmem_ld_32x8(taddr + (uint32_t)((gbase + i) * 8), r[i]);   // warp-uniform
         ptx::tmem_ld_wait();
         if (!row_valid) continue;
 #pragma unroll
-        for (int i = 0; i < XPRE; ++i) {
+        for (int i = 0; i < NB; ++i) {
             const int grp = gbase + i;
             if (grp >= g_end) break;
             const int c8 = grp * 8;
-            const uint4 x4 = xc[i];
+            const uint4 x4 = *reinterpret_cast<const uint4 *>(xrow + c8);
             const uint32_t xw[4] = {x4.x, x4.y, x4.z, x4.w};
             const int4 b0 = *reinterpret_cast<const int4 *>(bh_s + c8), b1 = *reinterpret_cast<const int4 *>(bh_s + c8 + 4);
             const int32_t bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
@@ -237,8 +228,7 @@ __device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, 
                 *reinterpret_cast<int4 *>(dst) = make_int4(o[0], o[1], o[2], o[3]);
                 *reinterpret_cast<int4 *>(dst + 4) = make_int4(o[4], o[5], o[6], o[7]);
             } else {
-                int16_t *dst = (int16_t *)p.pre + (size_t)b * p.N + n0 + c8;
-                *reinterpret_cast<uint4 *>(dst) = make_uint4(pack16(o[0], o[1]), pack16(o[2], o[3]), pack16(o[4], o[5]), pack16(o[6], o[7]));
+                *reinterpret_cast<uint4 *>(xrow + c8) = make_uint4(pack16(o[0], o[1]), pack16(o[2], o[3]), pack16(o[4], o[5]), pack16(o[6], o[7]));
             }
         }
     }
@@ -418,14 +408,27 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, in
             if (r < nrows) {
                 const int16_t *row = (const int16_t *)p.pre + (size_t)(rb + r) * p.N;
                 const int tig = (warp - r * wpr) * 32 + lane, gs = wpr * 32;
-                for (int u = 2 * tig; u < p.C; u += 2 * gs) {
-                    int32_t v[2][4];
-                    load_pair_i16<G>(row + (size_t)u * G, false, v);
+                // four independent loads in flight per thread: the row comes from L2, and one load per trip would
+                // pay its latency C / (2 gs) times in a row
+                for (int u0 = 2 * tig; u0 < p.C; u0 += 8 * gs) {
+                    int32_t v[4][2][4];
 #pragma unroll
-                    for (int g = 0; g < G; ++g) {
-                        sum[g] += v[0][g] + v[1][g];
-                        sq[g] += (long long)(v[0][g] * v[0][g]) + (long long)(v[1][g] * v[1][g]);
+                    for (int k = 0; k < 4; ++k) {
+                        const int u = u0 + 2 * gs * k;
+                        if (u < p.C) {
+                            load_pair_i16<G>(row + (size_t)u * G, false, v[k]);
+                        } else {
+#pragma unroll
+                            for (int g = 0; g < 4; ++g) { v[k][0][g] = 0; v[k][1][g] = 0; }
+                        }
                     }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+#pragma unroll
+                        for (int g = 0; g < G; ++g) {
+                            sum[g] += v[k][0][g] + v[k][1][g];
+                            sq[g] += (long long)(v[k][0][g] * v[k][0][g]) + (long long)(v[k][1][g] * v[k][1][g]);
+                        }
                 }
             }
             warp_reduce_stats<G>(ctl, sum, sq);
@@ -605,54 +608,71 @@ __device__ __forceinline__ void phase_c_small(const RecParams &p, int t, int p_l
 }
 
 // ------------------------------------------------------------------------------------------------
-// Operand ring of the tensor-core phases.  Chunks (up to STAGE_KB k-blocks, contiguous in the tiled global
-// image) are numbered by a per-CTA sequence number that runs over both matmul phases of all steps:
-// stage = seq mod stages, mbarrier parity = (seq / stages) mod 2; stages is a power of two.
-// One producer thread issues the bulk copies; several issuer threads (one per accumulator) consume the
-// chunks: a single thread's issue latency (wait, descriptors, 4 MMAs per k-block, commit), not the copy
+// Operand ring of the tensor-core phases.  A chunk is up to STAGE_KB k-blocks, contiguous in the tiled global
+// image.  One producer thread issues the bulk copies; several issuer threads, each with its own accumulator,
+// consume them: a single thread's issue latency (wait, descriptors, 4 MMAs per k-block, commit), not the copy
 // rate, is what bounds a one-issuer loop.
+// Within a phase every stage belongs to exactly one issuer: owner o of n_own uses the stages o, o + n_own, ...
+// in turn for its chunks.  A thread therefore only ever waits for the next round of a stage whose previous round
+// it has consumed itself (an mbarrier parity wait cannot tell round r + 1 from round r - 1).  Between phases the
+// CTA-wide barriers order everything, so a stage may change owner from one phase to the next.  rounds[s] counts
+// the uses of stage s so far: the parity of a use is its round number mod 2.
 
 struct Ring {
     uint8_t *base;
-    uint32_t mask, log2;
+    volatile uint32_t *rounds;       // shared memory, advanced by one thread between phases
 };
 
-// producer: chunk i of the phase (i < n) is `bytes_of(i)` bytes at src_of(i)
-__device__ __forceinline__ void ring_produce(RecCtl *ctl, const Ring &r, uint32_t seq0, int n, int kb_total, int chunks_per_tile,
+// Chunks of a phase: `contig`: owner o streams operand tile o, chunk j = k-blocks [j STAGE_KB, ...) of that tile;
+// else all owners share one tile and owner o takes its chunks o, o + n_own, ...  kb_total: k-blocks per tile.
+// The producer visits the owners round-robin, so that it only ever waits for a stage of the owner whose chunk
+// is due.  No division in these single-thread loops: their latency is the pace of the whole phase.
+__device__ __forceinline__ void ring_produce(RecCtl *ctl, const Ring &r, const RingPlan &pl, bool contig, int kb_total,
                                              const int8_t *src, volatile int *abort_flag)
 {
-    // tile j of the operand starts at src + j * kb_total * KB_BYTES; its chunks are consecutive
-    int tile = 0, ci = 0;
-    for (int i = 0; i < n; ++i) {
-        const uint32_t seq = seq0 + (uint32_t)i, stage = seq & r.mask, par = (seq >> r.log2) & 1u;
-        const int kb = ci * STAGE_KB;
-        const uint32_t bytes = (uint32_t)((kb_total - kb < STAGE_KB ? kb_total - kb : STAGE_KB) * KB_BYTES);
-        if (!wait_or_abort(&ctl->empty[stage], par ^ 1u, abort_flag)) return;
-        ptx::mbar_arrive_expect_tx(&ctl->full[stage], bytes);
-        ptx::bulk_load_1d(r.base + (size_t)stage * STAGE_BYTES, src + ((size_t)tile * kb_total + kb) * KB_BYTES, bytes, &ctl->full[stage]);
-        if (++ci == chunks_per_tile) { ci = 0; ++tile; }
+    int kk[4] = {0, 0, 0, 0};
+    uint32_t rr[4] = {0, 0, 0, 0};
+    for (int j = 0; j < pl.n_max; ++j) {
+#pragma unroll
+        for (int o = 0; o < 4; ++o) {
+            if (o >= pl.n_own || j >= pl.n_chunks[o]) continue;
+            const int c = contig ? j : o + j * pl.n_own;          // chunk number inside the tile
+            const uint32_t stage = (uint32_t)(o + pl.n_own * kk[o]);
+            const uint32_t par = (r.rounds[stage] + rr[o]) & 1u;
+            if (++kk[o] == pl.cnt[o]) { kk[o] = 0; ++rr[o]; }
+            const int kb = c * STAGE_KB;
+            const uint32_t bytes = (uint32_t)((kb_total - kb < STAGE_KB ? kb_total - kb : STAGE_KB) * KB_BYTES);
+            if (!wait_or_abort(&ctl->empty[stage], par ^ 1u, abort_flag)) return;
+            ptx::mbar_arrive_expect_tx(&ctl->full[stage], bytes);
+            ptx::bulk_load_1d(r.base + (size_t)stage * STAGE_BYTES, src + ((size_t)(contig ? o : 0) * kb_total + kb) * KB_BYTES, bytes,
+                              &ctl->full[stage]);
+        }
     }
 }
 
-// issuer: chunks first, first + stride, ... < n of the phase, all k-blocks of each into accumulator d_tmem.
+// issuer = owner `me`: all k-blocks of each of its chunks into accumulator d_tmem.
 // b_base is the shared-memory address of the resident B operand, b_kb_bytes its bytes per k-block.
-// kb0_of_first is the k-block index (within the tile) of chunk `first`; consecutive chunks of one issuer are
-// `stride` chunks apart in the same tile.
-__device__ __forceinline__ bool ring_issue(RecCtl *ctl, const Ring &r, uint32_t seq0, int first, int n, int stride, int kb0,
-                                           int kb_total, uint32_t b_base, uint32_t b_kb_bytes, uint32_t d_tmem, uint32_t idesc,
+__device__ __forceinline__ bool ring_issue(RecCtl *ctl, const Ring &r, const RingPlan &pl, int me, bool contig, int kb_total,
+                                           uint32_t b_base, uint32_t b_kb_bytes, uint32_t d_tmem, uint32_t idesc,
                                            volatile int *abort_flag)
 {
     const uint64_t a_desc0 = ptx::smem_desc_k_sw128(ptx::smem_u32(r.base));
     const uint64_t b_desc0 = ptx::smem_desc_k_sw128(b_base);
+    const int n_mine = pl.n_chunks[me], cnt = pl.cnt[me];
+    int kk = 0;
+    uint32_t rr = 0;
     bool acc = false;
-    for (int i = first; i < n; i += stride, kb0 += stride * STAGE_KB) {
-        const uint32_t seq = seq0 + (uint32_t)i, stage = seq & r.mask, par = (seq >> r.log2) & 1u;
+    for (int j = 0; j < n_mine; ++j) {
+        const uint32_t stage = (uint32_t)(me + pl.n_own * kk);
+        const uint32_t par = (r.rounds[stage] + rr) & 1u;
+        if (++kk == cnt) { kk = 0; ++rr; }
         if (!wait_or_abort(&ctl->full[stage], par, abort_flag)) return false;
         ptx::tc_fence_after();
+        const int kb0 = (contig ? j : me + j * pl.n_own) * STAGE_KB;
         uint64_t a_desc = a_desc0 + (uint64_t)(stage * (STAGE_BYTES >> 4));
         uint64_t b_desc = b_desc0 + (uint64_t)(((uint32_t)kb0 * b_kb_bytes) >> 4);
         const int nk = kb_total - kb0 < STAGE_KB ? kb_total - kb0 : STAGE_KB;
-        for (int j = 0; j < nk; ++j) {
+        for (int k2 = 0; k2 < nk; ++k2) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 ptx::mma_i8_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, acc);
@@ -666,17 +686,28 @@ __device__ __forceinline__ bool ring_issue(RecCtl *ctl, const Ring &r, uint32_t 
     return true;
 }
 
+// after a phase: advance the round counters by the uses of each stage in that phase
+__device__ __forceinline__ void ring_advance(const Ring &r, const RingPlan &pl)
+{
+#pragma unroll
+    for (int s = 0; s < MAX_STAGES; ++s) r.rounds[s] += (uint32_t)pl.uses[s];
+}
+
 __global__ void __launch_bounds__(RTHREADS, 1)
-k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_constant__ CUtensorMap map_Wp, RecParams p)
+k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_constant__ CUtensorMap map_Wp,
+                  const __grid_constant__ CUtensorMap map_X, const __grid_constant__ CUtensorMap map_pre, RecParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const bool proj = (p.flags & F_PROJECTION) != 0;
-    // layout: [ring stages][R slice][Wproj slice][row buffer][bias slice][control]
+    // layout: [ring stages][R slice][Wproj slice][X box][row buffer][bias slice][control]
     uint8_t *ring = smem;
     uint8_t *R_s = ring + (size_t)p.stages * STAGE_BYTES;
-    uint8_t *Wp_s = R_s + (size_t)p.kb_h * p.nc_pad * 128;
-    uint8_t *after_w = Wp_s + (proj ? (size_t)p.kb_c * p.pn * 128 : 0);
+    // R slice: npc rows per k-block.  The MMA reads nc_pad (npc rounded up to 16) rows per k-block: the up to 8 extra
+    // rows are the head of the next k-block (of the next region after the last one), and their columns are never read
+    uint8_t *Wp_s = R_s + (size_t)p.kb_h * p.npc * 128;
+    int16_t *x_s = (int16_t *)(Wp_s + (proj ? (size_t)p.kb_c * p.pn * 128 : 0));
+    uint8_t *after_w = (uint8_t *)x_s + (((size_t)p.x_bytes + 1023) & ~(size_t)1023);
     int16_t *row_s = (int16_t *)after_w;
     const size_t row_bytes = ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE)) ? ((size_t)p.C * p.G + p.C) * 2 : 0;
     int32_t *bh_s = (int32_t *)(after_w + ((row_bytes + 15) & ~(size_t)15));
@@ -696,16 +727,20 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
     while (tmem_cols < acc_cols_a + (uint32_t)(proj ? p.pn * p.n_issue_c : 0)) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&ctl->full[s], 1); ptx::mbar_init(&ctl->empty[s], 1); }
+        for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&ctl->full[s], 1); ptx::mbar_init(&ctl->empty[s], 1); ctl->rounds[s] = 0; }
         for (int i = 0; i < 2; ++i) ptx::mbar_init(&ctl->acc_full[i], 1);
         {
             const int nc = (p.kb_c + STAGE_KB - 1) / STAGE_KB;
-            ptx::mbar_init(&ctl->acc_full[2], (uint32_t)(nc < p.n_issue_c ? nc : p.n_issue_c));      // one arrival per projection issuer
+            (void)nc;
+            ptx::mbar_init(&ctl->acc_full[2], (uint32_t)(p.plan_c.n_own > 0 ? p.plan_c.n_own : 1));      // one arrival per projection issuer
         }
         ptx::mbar_init(&ctl->w_full, 1);
+        ptx::mbar_init(&ctl->x_full, 1);
         ctl->abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&map_R);
+        ptx::prefetch_tensormap(&map_X);
+        ptx::prefetch_tensormap(&map_pre);
         if (proj) ptx::prefetch_tensormap(&map_Wp);
     }
     if (warp == 1) {
@@ -735,13 +770,13 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
     // resident weights of the tensor-core path: one TMA box per k-block
     if (threadIdx.x == 0) {
         uint32_t bytes = 0;
-        if (has_cells && !p.small) bytes += (uint32_t)(p.kb_h * p.nc_pad * 128);
+        if (has_cells && !p.small) bytes += (uint32_t)(p.kb_h * p.npc * 128);
         if (has_ptile && !p.small) bytes += (uint32_t)(p.kb_c * p.pn * 128);
         if (bytes) {
             ptx::mbar_arrive_expect_tx(&ctl->w_full, bytes);
             if (has_cells)
                 for (int kb = 0; kb < p.kb_h; ++kb)
-                    ptx::tma_load_2d(R_s + (size_t)kb * p.nc_pad * 128, &map_R, &ctl->w_full, kb * 128, n0);
+                    ptx::tma_load_2d(R_s + (size_t)kb * p.npc * 128, &map_R, &ctl->w_full, kb * 128, n0);
             if (has_ptile)
                 for (int kb = 0; kb < p.kb_c; ++kb)
                     ptx::tma_load_2d(Wp_s + (size_t)kb * p.pn * 128, &map_Wp, &ctl->w_full, kb * 128, tile_p0);
@@ -753,13 +788,21 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
     ptx::cta_sync();
 
     unsigned epoch = 0;
-    uint32_t seq = 0;                            // chunks this CTA has put through the ring so far (uniform over its threads)
     Ring rg;
-    rg.base = ring; rg.mask = (uint32_t)p.stages - 1u; rg.log2 = (uint32_t)__ffs(p.stages) - 1u;
+    rg.base = ring; rg.rounds = ctl->rounds;
     const int cpt_a = (p.kb_h + STAGE_KB - 1) / STAGE_KB, n_chunks_a = p.MT * cpt_a;      // recurrent matmul: chunks per batch tile
     const int n_chunks_c = (p.kb_c + STAGE_KB - 1) / STAGE_KB;
-    const int n_issue_c = n_chunks_c < p.n_issue_c ? n_chunks_c : p.n_issue_c;
+    const int n_issue_c = p.plan_c.n_own;
     const uint32_t idesc_a = ptx::idesc_i8(128, p.nc_pad), idesc_c = ptx::idesc_i8(128, p.pn);
+    const int iss = warp == 1 ? 0 : warp == 18 ? 1 : warp == 19 ? 2 : warp == 17 ? 3 : -1;      // issuer thread number of lane 0
+
+    // the CTA's box of X_t: rows [t * B, t * B + MT * 128) x its gate rows (rows past the end of X read as zero)
+    const bool tensor_a = !p.small && has_cells;
+    auto fetch_x = [&](int t) {
+        ptx::mbar_arrive_expect_tx(&ctl->x_full, p.x_bytes);
+        ptx::tma_load_2d(x_s, &map_X, &ctl->x_full, n0, t * p.B);
+    };
+    if (tensor_a && threadIdx.x == 0) fetch_x(0);
 
     const bool timing = p.phase_ns != nullptr && cta == 0 && threadIdx.x == 0;
     unsigned long long t_mark = timing ? globaltimer() : 0ull;
@@ -789,42 +832,55 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
             if (warp == 0) {
                 if (lane == 0) {
                     fence_proxy_async_global();
-                    ring_produce(ctl, rg, seq, n_chunks_a, p.kb_h, cpt_a, p.hbuf + (size_t)cur * p.h_stride, abort_flag);
+                    ring_produce(ctl, rg, p.plan_a, true, p.kb_h, p.hbuf + (size_t)cur * p.h_stride, abort_flag);
                 }
                 __syncwarp();
-            } else if (warp == 1 || warp == 18) {
+            } else {
+              if (iss >= 0 && iss < p.MT) {
                 // one issuer per batch tile, each with its own accumulator
-                const int mi = warp == 1 ? 0 : 1;
-                if (lane == 0 && mi < p.MT) {
+                if (lane == 0) {
                     ptx::tc_fence_after();
-                    if (ring_issue(ctl, rg, seq + (uint32_t)(mi * cpt_a), 0, cpt_a, 1, 0, p.kb_h, ptx::smem_u32(R_s),
-                                   (uint32_t)p.nc_pad * 128u, tmem_base + (uint32_t)(mi * p.nc_pad), idesc_a, abort_flag))
-                        ptx::mma_commit(&ctl->acc_full[mi]);
+                    if (ring_issue(ctl, rg, p.plan_a, iss, true, p.kb_h, ptx::smem_u32(R_s), (uint32_t)p.npc * 128u,
+                                   tmem_base + (uint32_t)(iss * p.nc_pad), idesc_a, abort_flag))
+                        ptx::mma_commit(&ctl->acc_full[iss]);
                 }
                 __syncwarp();
-            } else if (warp < 18) {
+              }
+              if (warp >= 2 && warp < 18) {
                 // 16 epilogue warps: 4 TMEM lane quarters x (batch tile, column part)
                 const int e = warp - 2, quarter = warp & 3, slot = e >> 2;
                 const int mi = slot % p.MT, part = slot / p.MT, nparts = 4 / p.MT;
                 const int ngroups = n_cnt >> 3;
                 const int g_begin = part * ngroups / nparts, g_end = (part + 1) * ngroups / nparts;
                 const int b = mi * 128 + quarter * 32 + lane;
-                uint4 xv[XPRE];
                 const bool probe = p.phase_ns != nullptr && cta == 0 && warp == 2 && lane == 0;
                 const unsigned long long t_in = probe ? globaltimer() : 0ull;
-                phase_a_prefetch(p, b, t, n0, g_begin, g_end, b < p.B, xv);
-                if (__all_sync(0xffffffffu, wait_or_abort(&ctl->acc_full[mi], par, abort_flag))) {
+                const bool okx = wait_or_abort(&ctl->x_full, par, abort_flag);        // fetched a step ago
+                const bool oka = wait_or_abort(&ctl->acc_full[mi], par, abort_flag);
+                if (__all_sync(0xffffffffu, okx && oka)) {
                     if (probe) p.phase_ns[6] += globaltimer() - t_in;      // operand load + matmul latency
                     ptx::tc_fence_after();
                     const uint32_t ta = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * p.nc_pad);
-                    if (p.G == 4) phase_a_row<4>(p, ta, b, t, n0, g_begin, g_end, bh_s, b < p.B, xv);
-                    else phase_a_row<3>(p, ta, b, t, n0, g_begin, g_end, bh_s, b < p.B, xv);
+                    if (p.G == 4) phase_a_row<4>(p, ta, b, n0, g_begin, g_end, bh_s, x_s, b < p.B);
+                    else phase_a_row<3>(p, ta, b, n0, g_begin, g_end, bh_s, x_s, b < p.B);
                     ptx::tc_fence_before();
+                    ptx::fence_proxy_async();                              // the box leaves through the async proxy
                 }
+              }
             }
         }
-        if (!p.small && has_cells) seq += (uint32_t)n_chunks_a;
         ptx::cta_sync();
+        if (tensor_a && threadIdx.x == 0) ring_advance(rg, p.plan_a);
+        if (tensor_a && threadIdx.x == 0 && !*abort_flag) {
+            if (!(p.flags & F_PEEPHOLE)) {
+                // gate sums of all batch rows x this CTA's gate rows: one store, complete before the barrier publishes it
+                ptx::tma_store_2d(&map_pre, x_s, n0, 0);
+                ptx::bulk_commit_group();
+                ptx::bulk_wait_group_all();
+                fence_proxy_async_global();
+            }
+            if (t + 1 < p.T) fetch_x(t + 1);                               // the box is free again
+        }
         lap(0);
         grid_sync(p, epoch, abort_flag, false);
         lap(1);
@@ -852,19 +908,18 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
                 if (warp == 0) {
                     if (lane == 0) {
                         fence_proxy_async_global();
-                        ring_produce(ctl, rg, seq, n_chunks_c, p.kb_c, n_chunks_c, p.mbuf + (size_t)tile_mi * p.kb_c * KB_BYTES, abort_flag);
+                        ring_produce(ctl, rg, p.plan_c, false, p.kb_c, p.mbuf + (size_t)tile_mi * p.kb_c * KB_BYTES, abort_flag);
                     }
                     __syncwarp();
                 } else {
-                    // several issuers share the K range: issuer w takes chunks w, w + n_issue_c, ... into its own
+                    // several issuers share the K range: issuer w owns chunks w, w + n_issue_c, ... with its own
                     // accumulator; the epilogue adds the partial sums (exact in int32).  Issuers are the three warps
-                    // without an epilogue role and, for a fourth, the last epilogue warp before it turns to its part
-                    const int w = warp == 1 ? 0 : warp == 18 ? 1 : warp == 19 ? 2 : warp == 17 ? 3 : 4;
-                    if (w < n_issue_c) {
+                    // without an epilogue role and the last epilogue warp, before it turns to its part
+                    if (iss >= 0 && iss < n_issue_c) {
                         if (lane == 0) {
                             ptx::tc_fence_after();
-                            if (ring_issue(ctl, rg, seq, w, n_chunks_c, n_issue_c, w * STAGE_KB, p.kb_c, ptx::smem_u32(Wp_s),
-                                           (uint32_t)p.pn * 128u, tmem_base + acc_cols_a + (uint32_t)(w * p.pn), idesc_c, abort_flag))
+                            if (ring_issue(ctl, rg, p.plan_c, iss, false, p.kb_c, ptx::smem_u32(Wp_s), (uint32_t)p.pn * 128u,
+                                           tmem_base + acc_cols_a + (uint32_t)(iss * p.pn), idesc_c, abort_flag))
                                 ptx::mma_commit(&ctl->acc_full[2]);
                         }
                         __syncwarp();
@@ -884,8 +939,8 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
                     }
                 }
             }
-            if (!p.small && has_ptile) seq += (uint32_t)n_chunks_c;
             ptx::cta_sync();
+            if (!p.small && has_ptile && threadIdx.x == 0) ring_advance(rg, p.plan_c);
             lap(4);
             grid_sync(p, epoch, abort_flag, !p.small && warp >= 2);      // the epilogue warps wrote h
             lap(5);
@@ -925,16 +980,33 @@ __global__ void k_tile_rows(const int8_t *src, int8_t *dst, int B, int K, int nk
     *reinterpret_cast<uint4 *>(dst + tile_off(row, k, nkb)) = v;
 }
 
-size_t rec_smem_bytes(const LayerParams &p, int stages, int nc_pad, int pn, int kb_h, int kb_c)
+size_t x_box_bytes(int MT, int npc) { return (size_t)MT * 128 * npc * 2; }
+
+size_t rec_smem_bytes(const LayerParams &p, int stages, int nc_pad, int pn, int kb_h, int kb_c, int MT, int npc)
 {
     const bool proj = (p.flags & F_PROJECTION) != 0;
     size_t row_bytes = ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE)) ? ((size_t)p.C * p.G + p.C) * 2 : 0;
     row_bytes = (row_bytes + 15) & ~(size_t)15;
-    return 1024 + (size_t)stages * STAGE_BYTES + (size_t)kb_h * nc_pad * 128 + (proj ? (size_t)kb_c * pn * 128 : 0) +
-           row_bytes + (size_t)nc_pad * 4 + sizeof(RecCtl) + 64;
+    return 1024 + (size_t)stages * STAGE_BYTES + (size_t)kb_h * npc * 128 + (proj ? (size_t)kb_c * pn * 128 : 0) +
+           ((x_box_bytes(MT, npc) + 1023) & ~(size_t)1023) + row_bytes + (size_t)nc_pad * 4 + sizeof(RecCtl) + 64;
 }
 
 int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+// contig: n_own operand tiles of `per` chunks each, one owner per tile; else n_total chunks of one tile dealt round-robin
+RingPlan make_ring_plan(int stages, int n_own, bool contig, int per, int n_total)
+{
+    RingPlan pl;
+    memset(&pl, 0, sizeof(pl));
+    pl.n_own = n_own;
+    for (int o = 0; o < n_own && o < 4; ++o) {
+        pl.n_chunks[o] = contig ? per : (n_total - o + n_own - 1) / n_own;
+        pl.cnt[o] = (stages - o + n_own - 1) / n_own;
+        if (pl.n_chunks[o] > pl.n_max) pl.n_max = pl.n_chunks[o];
+        for (int j = 0; j < pl.n_chunks[o]; ++j) pl.uses[o + n_own * (j % pl.cnt[o])] += 1;
+    }
+    return pl;
+}
 
 }  // namespace
 
@@ -992,12 +1064,12 @@ int fast_recurrent_init(FastLayer &f, const LayerParams &p, const FastScratch &s
     int dev = 0, max_smem = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    int stages = MAX_STAGES;                      // a power of two
-    while (stages >= 2 && rec_smem_bytes(p, stages, f.nc_pad, f.pn, f.kb_h, f.kb_c) > (size_t)max_smem) stages >>= 1;
+    int stages = MAX_STAGES;
+    while (stages >= 2 && rec_smem_bytes(p, stages, f.nc_pad, f.pn, f.kb_h, f.kb_c, MT_max, cpc * p.G) > (size_t)max_smem) --stages;
     if (stages < 2) return QLSTM_OK;
     f.stages = stages;
-    f.smem = rec_smem_bytes(p, stages, f.nc_pad, f.pn, f.kb_h, f.kb_c);
-    if (!make_tensor_map_i8(&f.map_R, p.R, (uint64_t)p.N, (uint64_t)p.O, (uint32_t)f.nc_pad, 128)) return QLSTM_OK;
+    f.smem = rec_smem_bytes(p, stages, f.nc_pad, f.pn, f.kb_h, f.kb_c, MT_max, cpc * p.G);
+    if (!make_tensor_map_i8(&f.map_R, p.R, (uint64_t)p.N, (uint64_t)p.O, (uint32_t)(cpc * p.G), 128)) return QLSTM_OK;
     if (proj) {
         if (!make_tensor_map_i8(&f.map_Wp, p.Wproj, (uint64_t)p.O, (uint64_t)p.C, (uint32_t)f.pn, 128)) return QLSTM_OK;
     } else {
@@ -1037,6 +1109,17 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     rp.cpc = f.cpc; rp.n_cta_a = f.n_cta_a; rp.nc_pad = f.nc_pad;
     rp.pn = f.pn; rp.npn = f.npn; rp.n_ptiles = rp.MT * f.npn;
     rp.kb_h = f.kb_h; rp.kb_c = f.kb_c; rp.stages = f.stages; rp.n_issue_c = f.n_issue_c;
+    rp.npc = f.cpc * p.G;
+    {
+        // every MMA issuer owns at least one ring stage
+        const int cpt_a = (f.kb_h + STAGE_KB - 1) / STAGE_KB, n_chunks_c = (f.kb_c + STAGE_KB - 1) / STAGE_KB;
+        int ni = f.n_issue_c < n_chunks_c ? f.n_issue_c : n_chunks_c;
+        if (ni > f.stages) ni = f.stages;
+        if (ni < 1) ni = 1;
+        rp.plan_a = make_ring_plan(f.stages, rp.MT, true, cpt_a, 0);
+        rp.plan_c = make_ring_plan(f.stages, ni, false, 0, n_chunks_c);
+    }
+    rp.x_bytes = (uint32_t)x_box_bytes(rp.MT, rp.npc);
     // elementwise phase: contiguous ranges of the B x C cell grid (whole rows with layer norm + peephole)
     if ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE))
         rp.items_per_cta = ((B + f.grid - 1) / f.grid) * p.C;
@@ -1081,7 +1164,12 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
         ++n_launch;
     }
 
-    void *args[] = {(void *)&f.map_R, (void *)&f.map_Wp, (void *)&rp};
+    // X as a tensor [T * B][N] int16 and the gate sums as [B][N] int16; a CTA's box is all batch tiles x its gate rows
+    CUtensorMap map_X, map_pre;
+    if (!make_tensor_map_i16(&map_X, X, (uint64_t)T * B, (uint64_t)p.N, (uint32_t)rp.MT * 128, (uint32_t)rp.npc) ||
+        !make_tensor_map_i16(&map_pre, s.pre, (uint64_t)B, (uint64_t)p.N, (uint32_t)rp.MT * 128, (uint32_t)rp.npc))
+        return QLSTM_ERR_CUDA;
+    void *args[] = {(void *)&f.map_R, (void *)&f.map_Wp, (void *)&map_X, (void *)&map_pre, (void *)&rp};
     cudaError_t e = cudaLaunchCooperativeKernel((const void *)k_recurrent_sm100, dim3(f.grid), dim3(RTHREADS), args, f.smem, st);
     if (e != cudaSuccess) {
         cudaGetLastError();
