@@ -95,10 +95,37 @@ class ClockSampler:
 
 
 # DRAM traffic of the recurrent kernel from one ncu capture (its summary is kept with the other profile summaries):
-# dram__bytes_read.sum + dram__bytes_write.sum = 188.0 MB for 40 steps of config 5 at batch 256; per-step traffic is
-# steady, so a launch of T steps moves T / 40 of that.  Valid only for the kernel sources the counters were taken
-# from: if they changed since, the figure is reported as null.
-NCU_RECURRENT = {"bytes": 188.04e6, "steps": 40, "config": 5, "batch": 256, "source_sha": "8fc728514bc393f5"}
+# dram__bytes_read.sum + dram__bytes_write.sum = 175.86 + 10.03 MB for 40 steps of config 5 at batch 256; per-step
+# traffic is steady, so a launch of T steps moves T / 40 of that.  Valid only for the kernel sources the counters
+# were taken from: if they changed since, the figure is reported as null.
+NCU_RECURRENT = {"bytes": 185.89e6, "steps": 40, "config": 5, "batch": 256, "source_sha": "5446131e4e4de62b"}
+
+# The recurrent kernel is bound by plain integer arithmetic (the fixed-point epilogues), not by its matmuls or by
+# memory.  Peak: 148 SMs x 64 int32 lanes (4 schedulers x 16-lane integer pipe) x the SM clock; a microbenchmark of
+# this very arithmetic saturates at 64-68 thread instructions per clock per SM.  Algorithmic integer operations per
+# unit, counted as machine integer instructions of the leanest exact form of each step (measured in isolation):
+INT_LANES_PER_SM = 64
+OPS_ACTIVATION = 53          # integer sigmoid / tanh: polynomial of degree 6 + one exact division
+OPS_LAYERNORM = 38           # one layer-norm value: exact quotient, multiply-add, rescale
+OPS_GATE_SUM = 20            # one gate pre-activation: + bias, rescale, + X, saturate
+OPS_CELL = 30                # cell update, hidden state product, rescale, requantize
+OPS_PEEPHOLE = 15            # one peephole term
+OPS_PROJ_OUT = 12            # one projection output: + bias, rescale, requantize
+
+
+def algorithmic_int_ops(layers, B, T):
+    """Integer operations of the recurrent part per pass over the whole stack (see the constants above)."""
+    total = 0
+    for q in layers:
+        G = 3 if (q.flags & 8) else 4
+        per_cell = (G + 1) * OPS_ACTIVATION + OPS_CELL + G * OPS_GATE_SUM
+        if q.flags & 4:
+            per_cell += G * OPS_LAYERNORM
+        if q.flags & 2:
+            per_cell += (G - 1) * OPS_PEEPHOLE
+        per_row = q.n_cell * per_cell + (q.n_output * OPS_PROJ_OUT if (q.flags & 1) else 0)
+        total += per_row * B * T
+    return total
 
 
 def recurrent_source_sha():
@@ -295,9 +322,16 @@ def main():
     roof_proj = {"kernel": "input_projection", "bound": "tensor", "achieved": proj_tops, "peak": int8_peak,
                  "unit": "TOP/s", "frac": proj_tops / int8_peak, "traffic": None,
                  "peak_source": f"2 x bf16 sustained, {peaks['source']}", "ms_per_launch": proj_ms / n_l}
-    roof_rec = {"kernel": "recurrent", "bound": "tensor", "achieved": rec_tops, "peak": int8_peak, "unit": "TOP/s",
-                "frac": rec_tops / int8_peak, "traffic": None,
-                "peak_source": f"2 x bf16 sustained, {peaks['source']}", "ms_per_launch": rec_ms / n_l,
+    int_ops = algorithmic_int_ops(w.layers, B, T)
+    sm_ghz = (clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0) / 1e3
+    alu_peak = 148 * INT_LANES_PER_SM * sm_ghz / 1e3                     # T int-op/s at the clock seen during the run
+    rec_alu = int_ops / (rec_ms * 1e-3) / 1e12 if rec_ms > 0 else 0.0
+    roof_rec = {"kernel": "recurrent", "bound": "alu", "achieved": rec_alu, "peak": alu_peak, "unit": "Tint-op/s",
+                "frac": rec_alu / alu_peak, "traffic": None,
+                "peak_source": f"148 SMs x {INT_LANES_PER_SM} int32 lanes x {sm_ghz:.3f} GHz (SM clock sampled during the run)",
+                "algorithmic_int_ops_per_launch": int_ops / n_l,
+                "matmul_tops": rec_tops, "matmul_frac_of_int8_peak": rec_tops / int8_peak,
+                "ms_per_launch": rec_ms / n_l,
                 "us_per_layer_step": 1e3 * rec_ms / (n_l * T),
                 "phase_us_per_layer_step": {k: 1e3 * prof_phase[k] / (n_l * T) for k in
                                             ("phase_a_ms", "matmul_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms", "phase_c_ms", "wait_c_ms")},

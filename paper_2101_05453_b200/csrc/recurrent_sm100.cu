@@ -123,6 +123,10 @@ __device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence
 // phase before it wrote data that other CTAs fetch with bulk copies (async proxy: the operands h and m),
 // each writer first orders its generic-proxy writes against that proxy; the thread that issues the copies
 // fences again on its side after the barrier.  Gate sums are read with ordinary loads and need neither.
+// (Spreading the arrivals over several counters was tried: polling four words costs more than the serial
+// tail of 148 atomics on one word.)
+constexpr size_t BAR_BYTES = 64;                  // [0] counter, [1] abort word
+
 __device__ __forceinline__ void grid_sync(const RecParams &p, unsigned &epoch, volatile int *abort_flag, bool wrote_operands)
 {
     if (wrote_operands) fence_proxy_async_global();
@@ -221,14 +225,15 @@ __device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, 
                 const int32_t acc = add_sat((int32_t)r[i][j], bb[j]);
                 const int32_t H = sat16(rescale_sel(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
                 const int32_t X = (j & 1) ? hi16(xw[j >> 1]) : lo16(xw[j >> 1]);
-                o[j] = peep ? X + H : sat16(X + H);
+                o[j] = X + H;                                        // saturated to int16 when packed (no peephole)
             }
             if (peep) {
                 int32_t *dst = p.pre + (size_t)b * p.N + n0 + c8;
                 *reinterpret_cast<int4 *>(dst) = make_int4(o[0], o[1], o[2], o[3]);
                 *reinterpret_cast<int4 *>(dst + 4) = make_int4(o[4], o[5], o[6], o[7]);
             } else {
-                *reinterpret_cast<uint4 *>(xrow + c8) = make_uint4(pack16(o[0], o[1]), pack16(o[2], o[3]), pack16(o[4], o[5]), pack16(o[6], o[7]));
+                *reinterpret_cast<uint4 *>(xrow + c8) = make_uint4(ptx::pack_sat_s16(o[0], o[1]), ptx::pack_sat_s16(o[2], o[3]),
+                                                                   ptx::pack_sat_s16(o[4], o[5]), ptx::pack_sat_s16(o[6], o[7]));
             }
         }
     }
@@ -1019,10 +1024,10 @@ int fast_scratch_init(FastScratch &s, int max_B, int maxC, int maxO, int maxN, i
     if (cudaMalloc(&s.hbuf, s.hbuf_bytes) != cudaSuccess) return QLSTM_ERR_NOMEM;
     if (cudaMalloc(&s.mbuf, s.mbuf_bytes) != cudaSuccess) return QLSTM_ERR_NOMEM;
     if (cudaMalloc(&s.pre, (size_t)max_B * maxN * sizeof(int32_t)) != cudaSuccess) return QLSTM_ERR_NOMEM;
-    if (cudaMalloc(&s.bar, 64) != cudaSuccess) return QLSTM_ERR_NOMEM;
+    if (cudaMalloc(&s.bar, BAR_BYTES) != cudaSuccess) return QLSTM_ERR_NOMEM;
     cudaMemset(s.hbuf, 0, s.hbuf_bytes);
     cudaMemset(s.mbuf, 0, s.mbuf_bytes);
-    cudaMemset(s.bar, 0, 64);
+    cudaMemset(s.bar, 0, BAR_BYTES);
     return QLSTM_OK;
 }
 
@@ -1153,7 +1158,7 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     rp.bh = p.bh; rp.bp = p.bp; rp.bln = p.bln; rp.P = p.P; rp.L = p.L;
 
     // h^{-1} into operand buffer 0; barrier words cleared
-    if (cudaMemsetAsync(s.bar, 0, 64, st) != cudaSuccess) return QLSTM_ERR_CUDA;
+    if (cudaMemsetAsync(s.bar, 0, BAR_BYTES, st) != cudaSuccess) return QLSTM_ERR_CUDA;
     int n_launch = 1;
     if (rp.small) {
         if (cudaMemcpyAsync(s.hbuf, h, (size_t)B * p.O, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return QLSTM_ERR_CUDA;
