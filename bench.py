@@ -391,6 +391,32 @@ def main():
                                                                   ("phase_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms",
                                                                    "phase_c_ms", "wait_c_ms")}}
             q1.close()
+            # the other batch sizes of the configuration's sweep (1 is above, the timed workload is the largest)
+            sweep = {}
+            for Bs in (8, 64):
+                if Bs == B:
+                    continue
+                ws = make_workload(5, batch=Bs, T=T)
+                qs = qlstm.QLSTM(ws.layers, T, Bs, device=local)
+                xs = torch.from_numpy(ws.x).to(dev)
+                hs0, cs0 = ws.initial_state()
+                hs, cs = torch.from_numpy(hs0).to(dev), torch.from_numpy(cs0).to(dev)
+                ys = torch.zeros((T, Bs, O), dtype=torch.int8, device=dev)
+                tsw = []
+                for i in range(6):
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    qs.run(xs, T, Bs, hs, cs, ys, stream=stream)
+                    b.record()
+                    torch.cuda.synchronize()
+                    if i >= 3:
+                        tsw.append(a.elapsed_time(b))
+                qs.last_status()
+                qs.close()
+                ms = statistics.median(tsw)
+                sweep[str(Bs)] = {"value": Bs * T / (ms * 1e-3), "unit": UNIT, "ms_per_pass": ms,
+                                  "us_per_layer_step": 1e3 * ms / (T * n_l)}
+            line["batch_sweep"] = sweep
         if not args.no_cpu_baseline:
             from oracle import qlstm_ref
             cores = qlstm_ref.num_threads()
