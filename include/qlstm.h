@@ -144,6 +144,15 @@ int qlstm_set_impl(qlstm_t *q, int projection_impl, int recurrent_impl);
  * reports QLSTM_ERR_TIMEOUT.  Nothing faults or hangs and the handle stays usable; 0 restores normal operation. */
 int qlstm_debug_barrier_timeout(qlstm_t *q, int missing_arrivals, unsigned long long limit_ns);
 
+/* Host logic of the persistent kernel's operand ring, exposed for tests (no device is touched).  The matmuls of
+ * Section 3.2.4 / 3.2.8 stream their batch operand through `stages` ring stages that one producer fills and
+ * `n_owners` MMA issuers drain; within a phase owner o uses the stages o, o + n_owners, ... only, so that no
+ * thread ever waits for a round of a stage whose previous round it did not consume itself.
+ * contiguous != 0: one operand tile of chunks_per_tile chunks per owner; else chunks_total chunks of one tile dealt
+ * round-robin.  out14 (host) receives n_owners, the largest chunk count of an owner, chunks[4] and stages[4] per
+ * owner, and the fills of each of the 4 stages in the phase.  QLSTM_ERR_ARG unless 1 <= n_owners <= stages <= 4. */
+int qlstm_debug_ring_plan(int stages, int n_owners, int contiguous, int chunks_per_tile, int chunks_total, int *out14);
+
 /* Per-kernel device times of the runs since the last reset, measured with CUDA events on the
  * run's stream when profiling is on (it adds two event records per launch).
  * qlstm_set_profiling levels: 0 off; 1 the per-kernel event times; 2 also the device phase timers inside the

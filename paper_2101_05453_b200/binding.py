@@ -22,7 +22,7 @@ IMPL_AUTO, IMPL_SIMPLE, IMPL_FAST = 0, 1, 2
 EXPORTS = ["qlstm_create", "qlstm_run", "qlstm_run_host", "qlstm_input_projection", "qlstm_last_status",
            "qlstm_destroy", "qlstm_strerror", "qlstm_trace_bytes", "qlstm_set_impl", "qlstm_set_profiling",
            "qlstm_get_profile", "qlstm_device_info", "qlstm_eval_activations", "qlstm_eval_layernorm_row",
-           "qlstm_layernorm_rows_static", "qlstm_debug_barrier_timeout"]
+           "qlstm_layernorm_rows_static", "qlstm_debug_barrier_timeout", "qlstm_debug_ring_plan"]
 
 
 class Scale(C.Structure):
@@ -102,6 +102,8 @@ def lib():
         L.qlstm_eval_layernorm_row.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p, C.c_void_p]
         L.qlstm_debug_barrier_timeout.restype = C.c_int
         L.qlstm_debug_barrier_timeout.argtypes = [C.c_void_p, C.c_int, C.c_ulonglong]
+        L.qlstm_debug_ring_plan.restype = C.c_int
+        L.qlstm_debug_ring_plan.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)]
         L.qlstm_layernorm_rows_static.restype = C.c_int
         L.qlstm_layernorm_rows_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p,
                                                   C.c_void_p]
@@ -279,3 +281,12 @@ def parse_trace(buf: np.ndarray, dims: Sequence, T: int, B: int):
         out.append(d)
         off += T * rec
     return out
+
+
+def ring_plan(stages: int, n_owners: int, contiguous: bool, chunks_per_tile: int = 0, chunks_total: int = 0):
+    """The operand-ring plan of the recurrent kernel for one matmul phase (host logic only; needs no GPU)."""
+    out = (C.c_int * 14)()
+    _check(lib().qlstm_debug_ring_plan(stages, n_owners, int(contiguous), chunks_per_tile, chunks_total, out),
+           "qlstm_debug_ring_plan")
+    v = list(out)
+    return {"n_own": v[0], "n_max": v[1], "n_chunks": v[2:6], "cnt": v[6:10], "uses": v[10:14]}

@@ -61,4 +61,8 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
                           int8_t *h, int16_t *c, int8_t *y, int *status, unsigned long long *phase_ns, bool allow_small,
                           cudaStream_t st, int *launches);
 
+// Host logic of the recurrent kernel's operand ring, for tests: fills out[14] = n_own, n_max, n_chunks[4], cnt[4],
+// uses[4] of the plan for `stages` ring stages and `n_own` issuers (see RingPlan in recurrent_sm100.cu).
+int debug_ring_plan(int stages, int n_own, int contig, int per, int n_total, int *out);
+
 }  // namespace ql

@@ -426,6 +426,11 @@ int qlstm_input_projection(qlstm_t *q, int layer, const int8_t *x_dev, int rows,
     return run_projection(q, q->layers[layer], x_dev, rows, out_dev, (cudaStream_t)cuda_stream);
 }
 
+int qlstm_debug_ring_plan(int stages, int n_owners, int contiguous, int chunks_per_tile, int chunks_total, int *out14)
+{
+    return debug_ring_plan(stages, n_owners, contiguous, chunks_per_tile, chunks_total, out14);
+}
+
 int qlstm_last_status(qlstm_t *q)
 {
     if (!q) return QLSTM_ERR_ARG;

@@ -1185,4 +1185,18 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     return QLSTM_OK;
 }
 
+int debug_ring_plan(int stages, int n_own, int contig, int per, int n_total, int *out)
+{
+    if (!out || stages < 1 || stages > MAX_STAGES || n_own < 1 || n_own > 4 || n_own > stages) return QLSTM_ERR_ARG;
+    if (contig ? per < 0 : n_total < 0) return QLSTM_ERR_ARG;
+    const RingPlan pl = make_ring_plan(stages, n_own, contig != 0, per, n_total);
+    int k = 0;
+    out[k++] = pl.n_own;
+    out[k++] = pl.n_max;
+    for (int o = 0; o < 4; ++o) out[k++] = pl.n_chunks[o];
+    for (int o = 0; o < 4; ++o) out[k++] = pl.cnt[o];
+    for (int s = 0; s < MAX_STAGES; ++s) out[k++] = pl.uses[s];
+    return QLSTM_OK;
+}
+
 }  // namespace ql
