@@ -135,7 +135,8 @@ size_t qlstm_trace_bytes(const qlstm_t *q, int T, int B);
 /* Kernel selection, for tests and measurements.  0 = automatic (default), 1 = simple kernels
  * (one thread per output, one launch per phase), 2 = fast kernels (tensor-core projection,
  * persistent recurrent kernel); 2 fails with QLSTM_ERR_DIM at run time if a shape is unsupported.
- * recurrent_impl 3 = like 2 but with the tensor-core matmuls even at batch <= 4, where 0 and 2 use dp4a mat-vecs. */
+ * recurrent_impl 3 = like 2 but with the tensor-core matmuls even at batch <= 4, where 0 and 2 use dp4a mat-vecs;
+ * 4 = like 2 but with the dp4a mat-vecs up to batch 16 (the crossover is a measured default, not a limit). */
 int qlstm_set_impl(qlstm_t *q, int projection_impl, int recurrent_impl);
 
 /* Failure-path check: with missing_arrivals > 0 every grid barrier of the persistent recurrent kernel waits for

@@ -56,9 +56,10 @@ cudaError_t launch_projection_fast(const FastLayer &f, const LayerParams &p, con
                                    int sm_count, int *status, cudaStream_t st);
 
 bool fast_recurrent_supported(const FastLayer &f, const LayerParams &p, int B);
-// h / c are the caller's state (B rows); y is [T][B][O].  Returns a qlstm_error.
+// h / c are the caller's state (B rows); y is [T][B][O].  Batches up to small_batch_max (at most 16) run the matmuls
+// as dp4a mat-vecs.  Returns a qlstm_error.
 int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastScratch &s, const int16_t *X, int T, int B,
-                          int8_t *h, int16_t *c, int8_t *y, int *status, unsigned long long *phase_ns, bool allow_small,
+                          int8_t *h, int16_t *c, int8_t *y, int *status, unsigned long long *phase_ns, int small_batch_max,
                           cudaStream_t st, int *launches);
 
 // Host logic of the recurrent kernel's operand ring, for tests: fills out[14] = n_own, n_max, n_chunks[4], cnt[4],

@@ -374,7 +374,8 @@ int qlstm_run(qlstm_t *q, const int8_t *x_dev, int T, int B, int8_t *h_dev, int1
             cudaError_t e;
             if (use_fast) {
                 int frc = launch_recurrent_fast(L.fast, p, q->fscratch, q->X, T, B, h_dev + h_off, c_dev + c_off, outp,
-                                                q->status, q->phase_timers ? q->phase_ns : nullptr, impl != 3, st, &launches);
+                                                q->status, q->phase_timers ? q->phase_ns : nullptr, impl == 3 ? 0 : (impl == 4 ? 16 : 4), st,
+                                                &launches);
                 if (frc != QLSTM_OK) return frc;
                 e = cudaSuccess;
             } else {
@@ -444,7 +445,7 @@ int qlstm_last_status(qlstm_t *q)
 
 int qlstm_set_impl(qlstm_t *q, int projection_impl, int recurrent_impl)
 {
-    if (!q || projection_impl < 0 || projection_impl > 2 || recurrent_impl < 0 || recurrent_impl > 3) return QLSTM_ERR_ARG;
+    if (!q || projection_impl < 0 || projection_impl > 2 || recurrent_impl < 0 || recurrent_impl > 4) return QLSTM_ERR_ARG;
     q->impl_proj = projection_impl;
     q->impl_rec = recurrent_impl;
     return QLSTM_OK;

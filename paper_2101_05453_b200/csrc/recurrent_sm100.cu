@@ -38,7 +38,7 @@ constexpr int KB_BYTES = 128 * 128;           // one k-block of the A operand: 1
 constexpr int STAGE_KB = 2;                   // k-blocks per ring stage: one bulk copy brings up to 32 KB
 constexpr int STAGE_BYTES = STAGE_KB * KB_BYTES;
 constexpr int MAX_STAGES = 4;
-constexpr int SMALL_BATCH_MAX = 4;            // up to this batch the matmuls run as dp4a mat-vecs
+constexpr int SMALL_BATCH_MAX = 16;           // the dp4a mat-vec path exists up to this batch; the default crossover is lower
 constexpr unsigned long long SPIN_LIMIT_NS = 2000000000ull;   // 2 s per grid barrier
 
 // How one matmul phase uses the ring: owner o of n_own (one MMA issuer each) owns the stages o, o + n_own, ...
@@ -541,7 +541,8 @@ __device__ __forceinline__ void phase_b(const RecParams &p, RecCtl *ctl, int t, 
 }
 
 // ------------------------------------------------------------------------------------------------
-// Small batch (B <= SMALL_BATCH_MAX = 4; measured crossover: from 8 rows on the tensor-core path is faster):
+// Small batch (default: B <= 4; measured crossover: from 8 rows on the tensor-core path is faster; selectable up to
+// SMALL_BATCH_MAX = 16 rows):
 // the matmuls are mat-vec products, far too small for a 128-row tensor-core tile
 // and dominated by TMA / TMEM round-trip latency.  Each warp takes whole weight rows from shared memory,
 // lanes split K in 128-byte strides (conflict-free), dp4a accumulates, one warp reduction per (row, batch).
@@ -831,7 +832,9 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
             if (has_cells) {
                 if (p.B == 1) phase_a_small<1>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
                 else if (p.B <= 2) phase_a_small<2>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
-                else phase_a_small<4>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
+                else if (p.B <= 4) phase_a_small<4>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
+                else if (p.B <= 8) phase_a_small<8>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
+                else phase_a_small<16>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
             }
         } else if (has_cells) {
             if (warp == 0) {
@@ -905,7 +908,9 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
                 if (sp_cnt > 0) {
                     if (p.B == 1) phase_c_small<1>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
                     else if (p.B <= 2) phase_c_small<2>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
-                    else phase_c_small<4>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
+                    else if (p.B <= 4) phase_c_small<4>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
+                    else if (p.B <= 8) phase_c_small<8>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
+                    else phase_c_small<16>(p, t, sp_lo, sp_cnt, (const int8_t *)Wp_s, (int8_t *)ring, h_next);
                 }
             } else if (has_ptile) {
                 if (warp == 0) {
@@ -1100,7 +1105,7 @@ void fast_layer_destroy(FastLayer &) {}
 bool fast_recurrent_supported(const FastLayer &f, const LayerParams &, int B) { return f.rec_ok && B <= 256; }
 
 int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastScratch &s, const int16_t *X, int T, int B,
-                          int8_t *h, int16_t *c, int8_t *y, int *status, unsigned long long *phase_ns, bool allow_small,
+                          int8_t *h, int16_t *c, int8_t *y, int *status, unsigned long long *phase_ns, int small_batch_max,
                           cudaStream_t st, int *launches)
 {
     RecParams rp;
@@ -1133,7 +1138,8 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     {
         const int maxk = p.O > p.C ? p.O : p.C;
         const bool fits = (size_t)SMALL_BATCH_MAX * maxk <= (size_t)f.stages * STAGE_BYTES && (!(p.flags & F_PROJECTION) || rp.rpc <= f.pn);
-        rp.small = (allow_small && B <= SMALL_BATCH_MAX && fits) ? 1 : 0;
+        const int lim = small_batch_max < SMALL_BATCH_MAX ? small_batch_max : SMALL_BATCH_MAX;
+        rp.small = (B <= lim && fits) ? 1 : 0;
     }
     rp.fast_rescale_ok = 1;
     for (int g = 0; g < p.G; ++g) {

@@ -93,11 +93,13 @@ def test_fast_kernels_batch_sizes(B):
 @pytest.mark.parametrize("kw", [dict(projection=True, layernorm=True), dict(cifg=True), dict(peephole=True, projection=True),
                                 dict(peephole=True, layernorm=True)], ids=lambda k: "+".join(sorted(k)))
 def test_small_batch_both_matmul_paths(B, kw):
-    """At batch <= 4 the recurrent kernel uses dp4a mat-vecs by default; impl 3 forces the tensor-core path."""
+    """At batch <= 4 the recurrent kernel uses dp4a mat-vecs by default; impl 3 forces the tensor-core path, impl 4
+    the dp4a path up to batch 16."""
     w = random_layer_stack(300 + B, 2, 32, 112, 48, T=6, B=B, **kw)
     want = oracle(w)
     check_equal(run_gpu(w, impl=(FAST, FAST)), want, f"default path B={B} {kw}")
     check_equal(run_gpu(w, impl=(FAST, 3)), want, f"tcgen05 B={B} {kw}")
+    check_equal(run_gpu(w, impl=(FAST, 4)), want, f"dp4a B={B} {kw}")
 
 
 def test_trace_parity_config3_slice():
