@@ -390,6 +390,20 @@ def main():
                                       "phase_us_per_layer_step": {k: 1e3 * p1_phase[k] / (n_l * T) for k in
                                                                   ("phase_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms",
                                                                    "phase_c_ms", "wait_c_ms")}}
+            # streaming use: one timestep per call, state carried by the caller (every call pays all launches of the stack)
+            n_calls = 60
+            xs1 = x1[:1].contiguous()
+            ys1 = torch.zeros((1, 1, O), dtype=torch.int8, device=dev)
+            q1.set_profiling(0)
+            for i in range(10):
+                q1.run(xs1, 1, 1, h1, c1, ys1, stream=stream)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for i in range(n_calls):
+                q1.run(xs1, 1, 1, h1, c1, ys1, stream=stream)
+            torch.cuda.synchronize()
+            line["latency_batch1"]["streaming_us_per_call_T1"] = 1e6 * (time.perf_counter() - t0) / n_calls
+            q1.last_status()
             q1.close()
             # the other batch sizes of the configuration's sweep (1 is above, the timed workload is the largest)
             sweep = {}
