@@ -154,6 +154,15 @@ int qlstm_debug_barrier_timeout(qlstm_t *q, int missing_arrivals, unsigned long 
  * owner, and the fills of each of the 4 stages in the phase.  QLSTM_ERR_ARG unless 1 <= n_owners <= stages <= 4. */
 int qlstm_debug_ring_plan(int stages, int n_owners, int contiguous, int chunks_per_tile, int chunks_total, int *out14);
 
+/* Host logic of the input-projection kernel's tiling (Section 3.2.4, first rescale term), exposed for tests (no
+ * device is touched).  For a projection of `rows` rows onto n_gate_rows = cells x gates outputs with n_input
+ * columns, on a device of sm_count SMs with smem_bytes of shared memory per block, out5 (host) receives the panel
+ * width (gate rows of W resident per block), the depth of the x ring, the output tiles per block, the number of
+ * m-tile ranges (> 0: block b keeps panel b % panels and walks range b / panels; 0: equal contiguous ranges of the
+ * panel-major tile numbering) and the grid size.  QLSTM_ERR_ARG on a non-positive argument or NULL; QLSTM_ERR_DIM
+ * when no panel of these shapes fits in shared memory (such layers take the simple kernel). */
+int qlstm_debug_projection_plan(long long rows, int n_gate_rows, int n_input, int sm_count, int smem_bytes, int *out5);
+
 /* Per-kernel device times of the runs since the last reset, measured with CUDA events on the
  * run's stream when profiling is on (it adds two event records per launch).
  * qlstm_set_profiling levels: 0 off; 1 the per-kernel event times; 2 also the device phase timers inside the

@@ -22,7 +22,8 @@ IMPL_AUTO, IMPL_SIMPLE, IMPL_FAST = 0, 1, 2
 EXPORTS = ["qlstm_create", "qlstm_run", "qlstm_run_host", "qlstm_input_projection", "qlstm_last_status",
            "qlstm_destroy", "qlstm_strerror", "qlstm_trace_bytes", "qlstm_set_impl", "qlstm_set_profiling",
            "qlstm_get_profile", "qlstm_device_info", "qlstm_eval_activations", "qlstm_eval_layernorm_row",
-           "qlstm_layernorm_rows_static", "qlstm_debug_barrier_timeout", "qlstm_debug_ring_plan"]
+           "qlstm_layernorm_rows_static", "qlstm_debug_barrier_timeout", "qlstm_debug_ring_plan",
+           "qlstm_debug_projection_plan"]
 
 
 class Scale(C.Structure):
@@ -104,6 +105,8 @@ def lib():
         L.qlstm_debug_barrier_timeout.argtypes = [C.c_void_p, C.c_int, C.c_ulonglong]
         L.qlstm_debug_ring_plan.restype = C.c_int
         L.qlstm_debug_ring_plan.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)]
+        L.qlstm_debug_projection_plan.restype = C.c_int
+        L.qlstm_debug_projection_plan.argtypes = [C.c_longlong, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)]
         L.qlstm_layernorm_rows_static.restype = C.c_int
         L.qlstm_layernorm_rows_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p,
                                                   C.c_void_p]
@@ -290,3 +293,12 @@ def ring_plan(stages: int, n_owners: int, contiguous: bool, chunks_per_tile: int
            "qlstm_debug_ring_plan")
     v = list(out)
     return {"n_own": v[0], "n_max": v[1], "n_chunks": v[2:6], "cnt": v[6:10], "uses": v[10:14]}
+
+
+def projection_plan(rows: int, n_gate_rows: int, n_input: int, sm_count: int = 148, smem_bytes: int = 232448):
+    """The tiling of the input-projection kernel for one launch shape (host logic only; needs no GPU)."""
+    out = (C.c_int * 5)()
+    _check(lib().qlstm_debug_projection_plan(rows, n_gate_rows, n_input, sm_count, smem_bytes, out),
+           "qlstm_debug_projection_plan")
+    v = list(out)
+    return {"bn": v[0], "stages": v[1], "per_cta": v[2], "m_ranges": v[3], "grid": v[4]}

@@ -25,6 +25,7 @@ struct FastLayer {
     bool proj_ok = false;        // tensor-core projection usable for this layer
     CUtensorMap map_W;           // W [N][I] int8, K-major, 128B swizzle, box = one k-block of the resident panel
     int proj_bn = 0;             // panel width (rows of W resident in shared memory)
+    long long proj_rows_hint = 0; // rows (max_T * max_B) the panel width is tuned for; set before fast_layer_init
     int proj_stages = 0;         // depth of the x ring
     // persistent recurrent kernel plan
     bool rec_ok = false;
@@ -65,5 +66,6 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
 // Host logic of the recurrent kernel's operand ring, for tests: fills out[14] = n_own, n_max, n_chunks[4], cnt[4],
 // uses[4] of the plan for `stages` ring stages and `n_own` issuers (see RingPlan in recurrent_sm100.cu).
 int debug_ring_plan(int stages, int n_own, int contig, int per, int n_total, int *out);
+int debug_projection_plan(long long rows, int N, int K, int sm_count, int max_smem, int *out5);
 
 }  // namespace ql

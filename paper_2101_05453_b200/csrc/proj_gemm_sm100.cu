@@ -17,8 +17,14 @@
 //   warp 1       MMA issuer:   4 x (M128 N=BN K32) per k-block into one of two TMEM accumulators
 //   warps 2..17  epilogue:     tcgen05.ld -> + folded bias -> fixed-point rescale -> sat16 -> stores,
 //                              overlapping the next tile's MMAs through the second TMEM accumulator
-// Tiles are numbered panel-major and split into equal contiguous ranges, so a CTA touches at most two
-// panels.  No cluster launch and no multicast.
+// Tiles are numbered panel-major.  Where the SMs hold at least one CTA per panel, CTA b keeps panel
+// b % panels for the whole launch and walks one of floor(SMs / panels) ranges of M tiles; the CTAs of a
+// range then ask for the same x tiles at about the same time, so x reaches L2 from HBM once instead of
+// once per panel (the int16 output, 2 N / K times the size of x, would otherwise push it out between
+// uses).  The panel width is chosen so that panels x ranges fills the SMs.  Otherwise the tiles are
+// split into equal contiguous ranges and a CTA touches at most two panels.  x is loaded with an L2
+// evict-last hint and the output stored with evict-first.  No cluster launch and no multicast.
+#include "../../include/qlstm.h"
 #include "fast_kernels.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
@@ -42,6 +48,7 @@ struct ProjParams {
     FastScale fs[4];
     Scale sc[4];
     int generic;                 // some gate has a positive shift: use the generic rescale
+    int m_ranges;                // > 0: CTA b owns panel b % tiles_n and the m-tile range b / tiles_n of m_ranges
     int *status;
 };
 
@@ -50,6 +57,31 @@ struct SharedCtl {
     uint32_t tmem_base;
     int abort_flag;
 };
+
+// L2 eviction policies for per-access cache hints: lines touched with evict-last stay in L2 in preference to lines
+// touched with evict-first.
+__device__ __forceinline__ uint64_t l2_policy_evict_last()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+// 2-D tiled load global -> shared with an L2 eviction policy for the lines it reads; otherwise as ptx::tma_load_2d
+// (c0 is the innermost coordinate and c0 * element size a multiple of 16 bytes).
+__device__ __forceinline__ void tma_load_2d_hint(void *dst, const CUtensorMap *map, uint64_t *bar, int32_t c0, int32_t c1,
+                                                 uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(ptx::smem_u32(dst)), "l"((uint64_t)map), "r"(ptx::smem_u32(bar)), "r"(c0), "r"(c1), "l"(policy)
+        : "memory");
+}
 
 __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
 {
@@ -65,7 +97,7 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
 // 16 adjacent columns of one output row: + folded bias -> rescale -> sat16 -> one 32-byte store.
 template <int G, bool GENERIC>
 __device__ __forceinline__ void epilogue_piece(const uint32_t (&r)[16], const int32_t *bias, const ProjParams &p,
-                                               int n_first, int16_t *dst, int n_valid, bool wide_ok)
+                                               int n_first, int16_t *dst, int n_valid, bool wide_ok, uint64_t st_policy)
 {
     // column j of this piece is global column n_first + j; its gate slot is (n_first + j) % G
     uint32_t packed[8];
@@ -86,8 +118,8 @@ __device__ __forceinline__ void epilogue_piece(const uint32_t (&r)[16], const in
     }
     if (n_valid >= 16 && wide_ok) {
         // a 32-byte store fills a whole sector
-        asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(packed[0]), "r"(packed[1]),
-                     "r"(packed[2]), "r"(packed[3]), "r"(packed[4]), "r"(packed[5]), "r"(packed[6]), "r"(packed[7])
+        asm volatile("st.global.L2::cache_hint.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8}, %9;" ::"l"(dst), "r"(packed[0]), "r"(packed[1]),
+                     "r"(packed[2]), "r"(packed[3]), "r"(packed[4]), "r"(packed[5]), "r"(packed[6]), "r"(packed[7]), "l"(st_policy)
                      : "memory");
         return;
     }
@@ -113,9 +145,22 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tiles_m = (p.M + BM - 1) / BM, tiles_n = (p.N + p.bn - 1) / p.bn;
     const int n_tiles = tiles_m * tiles_n;
-    const int per_cta = (n_tiles + gridDim.x - 1) / gridDim.x;
-    const int t_begin = blockIdx.x * per_cta;
-    const int t_end = (t_begin + per_cta < n_tiles) ? t_begin + per_cta : n_tiles;
+    // Tiles are numbered panel-major.  Either every CTA takes an equal contiguous range of them, or (m_ranges > 0)
+    // CTA b keeps panel b % tiles_n and walks the m-tile range b / tiles_n: the CTAs of one range then read the
+    // same x tiles at about the same time, so each x tile comes from HBM once and from L2 for the other panels.
+    int t_begin, t_end;
+    if (p.m_ranges > 0) {
+        const int n_tile = blockIdx.x % tiles_n, r = blockIdx.x / tiles_n;
+        const int per = (tiles_m + p.m_ranges - 1) / p.m_ranges;
+        const int mb = r * per < tiles_m ? r * per : tiles_m;
+        const int me = mb + per < tiles_m ? mb + per : tiles_m;
+        t_begin = n_tile * tiles_m + mb;
+        t_end = n_tile * tiles_m + me;
+    } else {
+        const int per_cta = (n_tiles + gridDim.x - 1) / gridDim.x;
+        t_begin = blockIdx.x * per_cta;
+        t_end = (t_begin + per_cta < n_tiles) ? t_begin + per_cta : n_tiles;
+    }
     volatile int *abort_flag = &ctl->abort_flag;
 
     if (threadIdx.x == 0) {
@@ -142,6 +187,7 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
         if (lane == 0) {
             int stage = 0; uint32_t phase = 0, wfree_par = 0;
             int cur_n = -1;
+            const uint64_t x_policy = l2_policy_evict_last();      // x is re-read once per panel: keep it in L2
             for (int t = t_begin; t < t_end && !*abort_flag; ++t) {
                 const int n_tile = t / tiles_m, m0 = (t % tiles_m) * BM;
                 if (n_tile != cur_n) {
@@ -157,7 +203,7 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
                 for (int kb = 0; kb < p.kb; ++kb) {
                     if (!wait_or_abort(&ctl->a_empty[stage], phase ^ 1, abort_flag)) break;
                     ptx::mbar_arrive_expect_tx(&ctl->a_full[stage], A_BYTES);
-                    ptx::tma_load_2d(ring + (size_t)stage * A_BYTES, &map_x, &ctl->a_full[stage], kb * BK, m0);
+                    tma_load_2d_hint(ring + (size_t)stage * A_BYTES, &map_x, &ctl->a_full[stage], kb * BK, m0, x_policy);
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
             }
@@ -211,6 +257,7 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
         const bool has0 = c0 < n_chunks, has1 = c1 < n_chunks;
         const bool wide_ok = (p.N % 16) == 0;            // every row starts on a 32-byte boundary
         int it = 0, cur_n0 = -1;
+        const uint64_t st_policy = l2_policy_evict_first();        // the output is written once and read much later
         for (int t = t_begin; t < t_end; ++t, ++it) {
             const int buf = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1;
@@ -246,8 +293,8 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
                 }
                 const int n_valid = p.N - (n_base + 16 * i);
                 if (row_ok && n_valid > 0) {
-                    if (i & 1) epilogue_piece<G, GENERIC>(rb, bias + 16 * i, p, n_base + 16 * i, dst_row + 16 * i, n_valid, wide_ok);
-                    else epilogue_piece<G, GENERIC>(ra, bias + 16 * i, p, n_base + 16 * i, dst_row + 16 * i, n_valid, wide_ok);
+                    if (i & 1) epilogue_piece<G, GENERIC>(rb, bias + 16 * i, p, n_base + 16 * i, dst_row + 16 * i, n_valid, wide_ok, st_policy);
+                    else epilogue_piece<G, GENERIC>(ra, bias + 16 * i, p, n_base + 16 * i, dst_row + 16 * i, n_valid, wide_ok, st_policy);
                 }
             }
             ptx::tc_fence_before();
@@ -270,20 +317,77 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
     }
 }
 
-int panel_width(int K)
-{
-    const int kb = (K + BK - 1) / BK;
-    int bn = (W_BYTES_MAX / (kb * BK)) / 32 * 32;
-    return bn > 256 ? 256 : bn;
-}
-
 size_t smem_bytes(int bn, int kb, int stages)
 {
     return 1024 + (size_t)kb * bn * BK + (size_t)stages * A_BYTES + EPI_WARPS * BIAS_PER_WARP * sizeof(int32_t) +
            sizeof(SharedCtl) + 64;
 }
 
+int ring_stages(int bn, int kb, int max_smem)
+{
+    int stages = MAX_STAGES;
+    while (stages >= 2 && smem_bytes(bn, kb, stages) > (size_t)max_smem) --stages;
+    return stages;
+}
+
+// How a launch of `rows` rows is cut: tiles per CTA and, if one panel per CTA costs no more tiles per CTA than equal
+// contiguous ranges, the number of m-tile ranges (else 0).
+struct TilePlan { int per_cta, m_ranges, grid; };
+
+TilePlan plan_tiles(long long rows, int N, int bn, int sm_count)
+{
+    const int tiles_m = (int)((rows + BM - 1) / BM), tiles_n = (N + bn - 1) / bn;
+    const long long tiles = (long long)tiles_m * tiles_n;
+    TilePlan pl;
+    pl.grid = tiles < sm_count ? (int)tiles : sm_count;
+    pl.per_cta = pl.grid > 0 ? (int)((tiles + pl.grid - 1) / pl.grid) : 0;
+    pl.m_ranges = 0;
+    int ranges = sm_count / tiles_n;
+    if (ranges > tiles_m) ranges = tiles_m;
+    if (ranges > 0) {
+        const int per = (tiles_m + ranges - 1) / ranges;
+        ranges = (tiles_m + per - 1) / per;                  // drop ranges that would be empty
+        if (per <= pl.per_cta) { pl.m_ranges = ranges; pl.grid = ranges * tiles_n; pl.per_cta = per; }
+    }
+    return pl;
+}
+
+// Panel width for launches of about `rows` rows.  A tile costs the larger of the epilogue (about 14.3 ns per column)
+// and of streaming the x tile from L2 (128 rows x K bytes at about 29 GB/s per SM), a tenth more when the ring is
+// too shallow to hold a whole x tile (the MMA issuer then waits on copies); all three figures were measured on
+// B200.  Take the width, among those whose panel fits in shared memory, with the least tile time x tiles per CTA.
+int panel_width(int K, int N, long long rows, int sm_count, int max_smem)
+{
+    const int kb = (K + BK - 1) / BK;
+    int bn = (W_BYTES_MAX / (kb * BK)) / 32 * 32;
+    bn = bn > 256 ? 256 : bn;
+    if (rows <= 0) return bn;
+    int best = bn;
+    double best_cost = 1e30;
+    for (int w = bn; w >= 32; w -= 32) {
+        const int stages = ring_stages(w, kb, max_smem);
+        if (stages < 2) continue;
+        const double epilogue_ns = 14.3 * w, stream_ns = 128.0 * (kb * BK) / 29.0;
+        const double tile_ns = (epilogue_ns > stream_ns ? epilogue_ns : stream_ns) * (stages < kb ? 1.1 : 1.0);
+        const double cost = tile_ns * plan_tiles(rows, N, w, sm_count).per_cta;
+        if (cost < best_cost) { best_cost = cost; best = w; }
+    }
+    return best;
+}
+
 }  // namespace
+
+int debug_projection_plan(long long rows, int N, int K, int sm_count, int max_smem, int *out5)
+{
+    if (!out5 || rows <= 0 || N <= 0 || K <= 0 || sm_count <= 0 || max_smem <= 0) return QLSTM_ERR_ARG;
+    const int kb = (K + BK - 1) / BK;
+    const int bn = panel_width(K, N, rows, sm_count, max_smem);
+    const int stages = bn >= 32 ? ring_stages(bn, kb, max_smem) : 0;
+    if (bn < 32 || stages < 2) return QLSTM_ERR_DIM;         // no resident panel for this K: the simple kernel runs
+    const TilePlan pl = plan_tiles(rows, N, bn, sm_count);
+    out5[0] = bn; out5[1] = stages; out5[2] = pl.per_cta; out5[3] = pl.m_ranges; out5[4] = pl.grid;
+    return smem_bytes(bn, kb, stages) <= (size_t)max_smem ? QLSTM_OK : QLSTM_ERR_DIM;
+}
 
 bool fast_projection_supported(const FastLayer &f, const LayerParams &p)
 {
@@ -294,14 +398,14 @@ int fast_projection_init(FastLayer &f, const LayerParams &p)
 {
     f.proj_ok = false;
     if (p.I % 16 != 0 || p.N % 8 != 0) return 0;
-    const int bn = panel_width(p.I);
-    if (bn < 32) return 0;                                   // K too large for a resident panel
-    const int kb = (p.I + BK - 1) / BK;
-    int dev = 0, max_smem = 0;
+    int dev = 0, max_smem = 0, sm_count = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    int stages = MAX_STAGES;
-    while (stages >= 2 && smem_bytes(bn, kb, stages) > (size_t)max_smem) --stages;
+    cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    const int bn = panel_width(p.I, p.N, f.proj_rows_hint, sm_count, max_smem);
+    if (bn < 32) return 0;                                   // K too large for a resident panel
+    const int kb = (p.I + BK - 1) / BK;
+    const int stages = ring_stages(bn, kb, max_smem);
     if (stages < 2) return 0;
     f.proj_bn = bn;
     f.proj_stages = stages;
@@ -330,8 +434,9 @@ cudaError_t launch_projection_fast(const FastLayer &f, const LayerParams &p, con
         if (s.shift > 0) pp.generic = 1;
         pp.fs[g] = make_fast_scale(s);
     }
-    const int tiles = ((rows + BM - 1) / BM) * ((p.N + pp.bn - 1) / pp.bn);
-    const int grid = tiles < sm_count ? tiles : sm_count;
+    const TilePlan pl = plan_tiles(rows, p.N, pp.bn, sm_count);
+    const int grid = pl.grid;
+    pp.m_ranges = pl.m_ranges;
     const size_t smem = smem_bytes(pp.bn, pp.kb, pp.stages);
     if (p.G == 4) {
         if (pp.generic) k_projection_sm100<4, true><<<grid, THREADS, smem, st>>>(map_x, f.map_W, pp);

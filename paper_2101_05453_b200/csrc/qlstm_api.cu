@@ -303,6 +303,7 @@ int qlstm_create(const qlstm_layer_t *layers, int n_layers, int max_T, int max_B
         if (frc != QLSTM_OK) { ok = false; rc = frc; }
     }
     for (int l = 0; l < n_layers && ok; ++l) {
+        q->layers[l].fast.proj_rows_hint = (long long)max_T * max_B;
         int frc = fast_layer_init(q->layers[l].fast, q->layers[l].p, q->fscratch, max_T, max_B);
         if (frc != QLSTM_OK) { ok = false; rc = frc; }
     }
@@ -430,6 +431,11 @@ int qlstm_input_projection(qlstm_t *q, int layer, const int8_t *x_dev, int rows,
 int qlstm_debug_ring_plan(int stages, int n_owners, int contiguous, int chunks_per_tile, int chunks_total, int *out14)
 {
     return debug_ring_plan(stages, n_owners, contiguous, chunks_per_tile, chunks_total, out14);
+}
+
+int qlstm_debug_projection_plan(long long rows, int n_gate_rows, int n_input, int sm_count, int smem_bytes, int *out5)
+{
+    return debug_projection_plan(rows, n_gate_rows, n_input, sm_count, smem_bytes, out5);
 }
 
 int qlstm_last_status(qlstm_t *q)
