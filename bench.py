@@ -100,6 +100,12 @@ class ClockSampler:
 # were taken from: if they changed since, the figure is reported as null.
 NCU_RECURRENT = {"bytes": 186.57e6, "steps": 40, "config": 5, "batch": 256, "source_sha": "984460bfd146d3a8"}
 
+# DRAM traffic of the input-projection kernel from one ncu capture of a full-size launch (three counters, one pass):
+# dram__bytes_read.sum + dram__bytes_write.sum = 54.7 + 1203.9 MB at 76800 rows of config 5 (algorithmic: 49.2 MB of x,
+# 5.2 MB of W, 1258.3 MB of int16 output, part of which is still in L2 when the kernel ends).  Valid only for the
+# kernel sources the counters were taken from and for that launch shape: otherwise reported as null.
+NCU_PROJECTION = {"bytes": 1258.6e6, "rows": 76800, "config": 5, "source_sha": "386f2013cbc0dbac"}
+
 # The recurrent kernel is bound by plain integer arithmetic (the fixed-point epilogues), not by its matmuls or by
 # memory.  Peak: 148 SMs x 64 int32 lanes (4 schedulers x 16-lane integer pipe) x the SM clock; a microbenchmark of
 # this very arithmetic saturates at 64-68 thread instructions per clock per SM.  Algorithmic integer operations per
@@ -128,13 +134,21 @@ def algorithmic_int_ops(layers, B, T):
     return total
 
 
-def recurrent_source_sha():
+def _source_sha(files):
     import hashlib
     m = hashlib.sha256()
-    for f in ("recurrent_sm100.cu", "qmath.cuh", "sm100_ptx.cuh"):
+    for f in files:
         with open(os.path.join(ROOT, "paper_2101_05453_b200", "csrc", f), "rb") as fh:
             m.update(fh.read())
     return m.hexdigest()[:16]
+
+
+def recurrent_source_sha():
+    return _source_sha(("recurrent_sm100.cu", "qmath.cuh", "sm100_ptx.cuh"))
+
+
+def projection_source_sha():
+    return _source_sha(("proj_gemm_sm100.cu", "qmath.cuh", "sm100_ptx.cuh"))
 
 
 def algorithmic_ops(layers, B, T):
@@ -322,6 +336,12 @@ def main():
     roof_proj = {"kernel": "input_projection", "bound": "tensor", "achieved": proj_tops, "peak": int8_peak,
                  "unit": "TOP/s", "frac": proj_tops / int8_peak, "traffic": None,
                  "peak_source": f"2 x bf16 sustained, {peaks['source']}", "ms_per_launch": proj_ms / n_l}
+    if (args.config == NCU_PROJECTION["config"] and B * T == NCU_PROJECTION["rows"]
+            and projection_source_sha() == NCU_PROJECTION["source_sha"]):
+        roof_proj["traffic"] = NCU_PROJECTION["bytes"]                                   # bytes per launch (one layer)
+    q0 = w.layers[0]
+    roof_proj["algorithmic_hbm_bytes"] = B * T * q0.n_input + q0.n_input * q0.n_cell * (3 if (q0.flags & 8) else 4) \
+        + 2 * B * T * q0.n_cell * (3 if (q0.flags & 8) else 4)
     int_ops = algorithmic_int_ops(w.layers, B, T)
     sm_ghz = (clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0) / 1e3
     alu_peak = 148 * INT_LANES_PER_SM * sm_ghz / 1e3                     # T int-op/s at the clock seen during the run

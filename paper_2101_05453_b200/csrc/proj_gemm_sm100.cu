@@ -95,13 +95,15 @@ __device__ __forceinline__ bool wait_or_abort(uint64_t *bar, uint32_t parity, vo
 }
 
 // 16 adjacent columns of one output row: + folded bias -> rescale -> sat16 -> one 32-byte store.
+// fs / sc hold the gates' scales in the order of the columns of the warp's first piece: slot k is the gate of
+// its column k.  Pieces are 16 columns wide, so piece `piece` starts piece slots later (16 = 1 mod 3, 0 mod 4) and
+// column j of it takes slot (piece + j) % 3, or j % 4: a constant once the piece loop is unrolled.
 template <int G, bool GENERIC>
-__device__ __forceinline__ void epilogue_piece(const uint32_t (&r)[16], const int32_t *bias, const ProjParams &p,
-                                               int n_first, int16_t *dst, int n_valid, bool wide_ok, uint64_t st_policy)
+__device__ __forceinline__ void epilogue_piece(const uint32_t (&r)[16], const int32_t *bias, const FastScale (&fs)[4],
+                                               const Scale (&sc)[4], int piece, int16_t *dst, int n_valid, bool wide_ok,
+                                               uint64_t st_policy)
 {
-    // column j of this piece is global column n_first + j; its gate slot is (n_first + j) % G
     uint32_t packed[8];
-    const int phase = n_first % G;
 #pragma unroll
     for (int j = 0; j < 16; j += 4) {
         const int4 b4 = *reinterpret_cast<const int4 *>(bias + j);
@@ -110,8 +112,8 @@ __device__ __forceinline__ void epilogue_piece(const uint32_t (&r)[16], const in
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int32_t v = (int32_t)r[j + i] + bb[i];          // |acc| + |bias| < 2^30: no overflow
-            const int g = (G == 4) ? i : (phase + j + i) % 3;
-            y[i] = GENERIC ? mbqm(v, p.sc[g]) : fast_rescale(v, p.fs[g]);
+            const int g = (G == 4) ? i : (piece + j + i) % 3;
+            y[i] = GENERIC ? mbqm(v, sc[g]) : fast_rescale(v, fs[g]);
         }
         packed[j >> 1] = ptx::pack_sat_s16(y[0], y[1]);
         packed[(j >> 1) + 1] = ptx::pack_sat_s16(y[2], y[3]);
@@ -281,6 +283,22 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
             const int n_base = n0 + c0 * 32;
             int16_t *dst_row = p.out + (size_t)row * p.N + n_base;
             const bool row_ok = row < p.M;
+            // the gates' scales in the order of this warp's columns (with three gates the first column's gate varies)
+            FastScale fs[4];
+            Scale sc[4];
+            if (G == 4) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { fs[k] = p.fs[k]; sc[k] = p.sc[k]; }
+            } else {
+                const int first = n_base % 3;
+#pragma unroll
+                for (int k = 0; k < 3; ++k) {
+                    const int g = first + k >= 3 ? first + k - 3 : first + k;
+                    fs[k] = g == 0 ? p.fs[0] : g == 1 ? p.fs[1] : p.fs[2];
+                    sc[k] = g == 0 ? p.sc[0] : g == 1 ? p.sc[1] : p.sc[2];
+                }
+                fs[3] = fs[0]; sc[3] = sc[0];
+            }
             if (np > 0) ptx::tmem_ld_32x16(tcol, ra);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -293,8 +311,8 @@ k_projection_sm100(const __grid_constant__ CUtensorMap map_x, const __grid_const
                 }
                 const int n_valid = p.N - (n_base + 16 * i);
                 if (row_ok && n_valid > 0) {
-                    if (i & 1) epilogue_piece<G, GENERIC>(rb, bias + 16 * i, p, n_base + 16 * i, dst_row + 16 * i, n_valid, wide_ok, st_policy);
-                    else epilogue_piece<G, GENERIC>(ra, bias + 16 * i, p, n_base + 16 * i, dst_row + 16 * i, n_valid, wide_ok, st_policy);
+                    if (i & 1) epilogue_piece<G, GENERIC>(rb, bias + 16 * i, fs, sc, i, dst_row + 16 * i, n_valid, wide_ok, st_policy);
+                    else epilogue_piece<G, GENERIC>(ra, bias + 16 * i, fs, sc, i, dst_row + 16 * i, n_valid, wide_ok, st_policy);
                 }
             }
             ptx::tc_fence_before();
