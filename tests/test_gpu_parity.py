@@ -170,6 +170,29 @@ def test_input_projection_matches_oracle(impl):
     assert np.array_equal(got, tr[0]["xg"])
 
 
+@pytest.mark.parametrize("cifg", [False, True], ids=["four-gates", "three-gates"])
+def test_input_projection_many_tiles_per_block(cifg):
+    """6000 rows x 600 cells: several output tiles per block, a ragged last m-tile and a ragged last panel; with four
+    gates the blocks take equal contiguous tile ranges, with three (CIFG) one panel per block and shared m-tile ranges."""
+    import torch
+    import paper_2101_05453_b200 as qlstm
+    from paper_2101_05453_b200.binding import projection_plan
+    w = random_layer_stack(78, 1, 96, 600, 600, T=40, B=150, cifg=cifg)
+    q = w.layers[0]
+    G = 3 if cifg else 4
+    rows = w.T * w.B
+    pl = projection_plan(rows, q.n_cell * G, q.n_input)
+    assert pl["per_cta"] > 1 and (pl["m_ranges"] > 0) == cifg
+    _, _, _, tr = oracle(w, trace=True)
+    with qlstm.QLSTM(w.layers, w.T, w.B) as hnd:
+        xd = torch.from_numpy(w.x).cuda()
+        out = torch.zeros((rows, q.n_cell, G), dtype=torch.int16, device="cuda")
+        hnd.input_projection(0, xd, rows, out, stream=torch.cuda.current_stream().cuda_stream)
+        hnd.last_status()
+        got = out.cpu().numpy().reshape(w.T, w.B, q.n_cell, G).transpose(0, 3, 1, 2)
+    assert np.array_equal(got, tr[0]["xg"][:, 4 - G:])
+
+
 def test_streaming_equivalence_and_state_carry():
     import paper_2101_05453_b200 as qlstm
     w = random_layer_stack(81, 2, 32, 64, 48, projection=True, layernorm=True, T=10, B=6)
