@@ -155,13 +155,15 @@ int qlstm_debug_barrier_timeout(qlstm_t *q, int missing_arrivals, unsigned long 
 int qlstm_debug_ring_plan(int stages, int n_owners, int contiguous, int chunks_per_tile, int chunks_total, int *out14);
 
 /* Host logic of the input-projection kernel's tiling (Section 3.2.4, first rescale term), exposed for tests (no
- * device is touched).  For a projection of `rows` rows onto n_gate_rows = cells x gates outputs with n_input
- * columns, on a device of sm_count SMs with smem_bytes of shared memory per block, out5 (host) receives the panel
- * width (gate rows of W resident per block), the depth of the x ring, the output tiles per block, the number of
- * m-tile ranges (> 0: block b keeps panel b % panels and walks range b / panels; 0: equal contiguous ranges of the
- * panel-major tile numbering) and the grid size.  QLSTM_ERR_ARG on a non-positive argument or NULL; QLSTM_ERR_DIM
- * when no panel of these shapes fits in shared memory (such layers take the simple kernel). */
-int qlstm_debug_projection_plan(long long rows, int n_gate_rows, int n_input, int sm_count, int smem_bytes, int *out5);
+ * device is touched).  For a handle created for max_rows = max_T x max_B rows, a projection of rows <= max_rows rows
+ * onto n_gate_rows = cells x gates outputs with n_input columns, on a device of sm_count SMs with smem_bytes of
+ * shared memory per block: out5 (host) receives the panel width (gate rows of W resident per block; fixed at create
+ * time from max_rows), the depth of the x ring, the output tiles per block, the number of m-tile ranges (> 0: block b
+ * keeps panel b % panels and walks range b / panels; 0: equal contiguous ranges of the panel-major tile numbering)
+ * and the grid size.  QLSTM_ERR_ARG on a non-positive argument, rows > max_rows or NULL; QLSTM_ERR_DIM when no panel
+ * of these shapes fits in shared memory (such layers take the simple kernel). */
+int qlstm_debug_projection_plan(long long max_rows, long long rows, int n_gate_rows, int n_input, int sm_count,
+                                int smem_bytes, int *out5);
 
 /* Per-kernel device times of the runs since the last reset, measured with CUDA events on the
  * run's stream when profiling is on (it adds two event records per launch).

@@ -106,7 +106,8 @@ def lib():
         L.qlstm_debug_ring_plan.restype = C.c_int
         L.qlstm_debug_ring_plan.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)]
         L.qlstm_debug_projection_plan.restype = C.c_int
-        L.qlstm_debug_projection_plan.argtypes = [C.c_longlong, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)]
+        L.qlstm_debug_projection_plan.argtypes = [C.c_longlong, C.c_longlong, C.c_int, C.c_int, C.c_int, C.c_int,
+                                                  C.POINTER(C.c_int)]
         L.qlstm_layernorm_rows_static.restype = C.c_int
         L.qlstm_layernorm_rows_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p,
                                                   C.c_void_p]
@@ -295,10 +296,13 @@ def ring_plan(stages: int, n_owners: int, contiguous: bool, chunks_per_tile: int
     return {"n_own": v[0], "n_max": v[1], "n_chunks": v[2:6], "cnt": v[6:10], "uses": v[10:14]}
 
 
-def projection_plan(rows: int, n_gate_rows: int, n_input: int, sm_count: int = 148, smem_bytes: int = 232448):
-    """The tiling of the input-projection kernel for one launch shape (host logic only; needs no GPU)."""
+def projection_plan(rows: int, n_gate_rows: int, n_input: int, sm_count: int = 148, smem_bytes: int = 232448,
+                    max_rows: Optional[int] = None):
+    """The tiling of the input-projection kernel for one launch shape, on a handle created for max_rows rows
+    (default: rows).  Host logic only; needs no GPU."""
     out = (C.c_int * 5)()
-    _check(lib().qlstm_debug_projection_plan(rows, n_gate_rows, n_input, sm_count, smem_bytes, out),
+    _check(lib().qlstm_debug_projection_plan(rows if max_rows is None else max_rows, rows, n_gate_rows, n_input,
+                                             sm_count, smem_bytes, out),
            "qlstm_debug_projection_plan")
     v = list(out)
     return {"bn": v[0], "stages": v[1], "per_cta": v[2], "m_ranges": v[3], "grid": v[4]}

@@ -66,6 +66,6 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
 // Host logic of the recurrent kernel's operand ring, for tests: fills out[14] = n_own, n_max, n_chunks[4], cnt[4],
 // uses[4] of the plan for `stages` ring stages and `n_own` issuers (see RingPlan in recurrent_sm100.cu).
 int debug_ring_plan(int stages, int n_own, int contig, int per, int n_total, int *out);
-int debug_projection_plan(long long rows, int N, int K, int sm_count, int max_smem, int *out5);
+int debug_projection_plan(long long rows_hint, long long rows, int N, int K, int sm_count, int max_smem, int *out5);
 
 }  // namespace ql

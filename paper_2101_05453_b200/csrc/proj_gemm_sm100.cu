@@ -395,11 +395,12 @@ int panel_width(int K, int N, long long rows, int sm_count, int max_smem)
 
 }  // namespace
 
-int debug_projection_plan(long long rows, int N, int K, int sm_count, int max_smem, int *out5)
+int debug_projection_plan(long long rows_hint, long long rows, int N, int K, int sm_count, int max_smem, int *out5)
 {
-    if (!out5 || rows <= 0 || N <= 0 || K <= 0 || sm_count <= 0 || max_smem <= 0) return QLSTM_ERR_ARG;
+    if (!out5 || rows_hint <= 0 || rows <= 0 || rows > rows_hint || N <= 0 || K <= 0 || sm_count <= 0 || max_smem <= 0)
+        return QLSTM_ERR_ARG;
     const int kb = (K + BK - 1) / BK;
-    const int bn = panel_width(K, N, rows, sm_count, max_smem);
+    const int bn = panel_width(K, N, rows_hint, sm_count, max_smem);
     const int stages = bn >= 32 ? ring_stages(bn, kb, max_smem) : 0;
     if (bn < 32 || stages < 2) return QLSTM_ERR_DIM;         // no resident panel for this K: the simple kernel runs
     const TilePlan pl = plan_tiles(rows, N, bn, sm_count);

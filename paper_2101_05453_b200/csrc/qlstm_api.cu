@@ -433,9 +433,10 @@ int qlstm_debug_ring_plan(int stages, int n_owners, int contiguous, int chunks_p
     return debug_ring_plan(stages, n_owners, contiguous, chunks_per_tile, chunks_total, out14);
 }
 
-int qlstm_debug_projection_plan(long long rows, int n_gate_rows, int n_input, int sm_count, int smem_bytes, int *out5)
+int qlstm_debug_projection_plan(long long max_rows, long long rows, int n_gate_rows, int n_input, int sm_count,
+                                int smem_bytes, int *out5)
 {
-    return debug_projection_plan(rows, n_gate_rows, n_input, sm_count, smem_bytes, out5);
+    return debug_projection_plan(max_rows, rows, n_gate_rows, n_input, sm_count, smem_bytes, out5);
 }
 
 int qlstm_last_status(qlstm_t *q)

@@ -44,8 +44,10 @@ SHAPES = [
 
 @pytest.mark.parametrize("rows,n,k", SHAPES)
 @pytest.mark.parametrize("sm_count", [1, 7, 132, 148])
-def test_every_tile_belongs_to_exactly_one_block(rows, n, k, sm_count):
-    pl = projection_plan(rows, n, k, sm_count=sm_count)
+@pytest.mark.parametrize("max_rows_factor", [1, 3, 400], ids=["as-created", "third", "tiny-part"])
+def test_every_tile_belongs_to_exactly_one_block(rows, n, k, sm_count, max_rows_factor):
+    # the panel width is fixed when the handle is created (for max_rows); launches may be much smaller
+    pl = projection_plan(rows, n, k, sm_count=sm_count, max_rows=rows * max_rows_factor)
     assert 32 <= pl["bn"] <= 256 and pl["bn"] % 32 == 0
     assert 2 <= pl["stages"] <= 6
     kb = -(-k // BK)
@@ -80,5 +82,7 @@ def test_arguments_are_checked():
     for bad in [(0, 8, 16), (1, 0, 16), (1, 8, 0)]:
         with pytest.raises(QlstmError):
             projection_plan(*bad)
+    with pytest.raises(QlstmError):
+        projection_plan(200, 8, 16, max_rows=100)         # more rows than the handle was created for
     with pytest.raises(QlstmError):
         projection_plan(1000, 1024, 8192)               # a 32-row panel of 8192 columns does not fit
