@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 
 #include "../../include/qlstm.h"
+#include "../../include/qlstm_debug.h"
 #include "qmath.cuh"
 
 namespace ql {
@@ -51,6 +52,7 @@ int qlstm_eval_layernorm_row(const int16_t *q_dev, int n, const int16_t *L_dev, 
                              int16_t *out_dev, void *cuda_stream)
 {
     if (!q_dev || !L_dev || !b_dev || !out_dev || n <= 0 || n > 8191) return QLSTM_ERR_ARG;
+    if (eff_ln.multiplier != 0 && (eff_ln.multiplier < (1 << 30) || eff_ln.shift < -31 || eff_ln.shift > 30)) return QLSTM_ERR_ARG;
     ql::k_eval_layernorm_row<<<1, 256, 0, (cudaStream_t)cuda_stream>>>(q_dev, n, L_dev, b_dev,
                                                                        ql::Scale{eff_ln.multiplier, eff_ln.shift}, out_dev);
     return cudaGetLastError() == cudaSuccess ? QLSTM_OK : QLSTM_ERR_CUDA;

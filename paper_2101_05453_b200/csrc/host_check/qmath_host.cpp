@@ -4,10 +4,6 @@
 
 extern "C" {
 int32_t qmh_mbqm(int32_t x, int32_t mult, int32_t shift) { return ql::mbqm(x, ql::Scale{mult, shift}); }
-int32_t qmh_sigmoid(int32_t x, int m) { return ql::sigmoid_q(x, m); }
-int32_t qmh_tanh(int32_t x, int m) { return ql::tanh_q(x, m); }
-void qmh_sigmoid_all(int m, int32_t *out) { for (int x = -32768; x < 32768; ++x) out[x + 32768] = ql::sigmoid_q(x, m); }
-void qmh_tanh_all(int m, int32_t *out) { for (int x = -32768; x < 32768; ++x) out[x + 32768] = ql::tanh_q(x, m); }
 void qmh_mbqm_many(const int32_t *x, int n, int32_t mult, int32_t shift, int32_t *out)
 {
     for (int i = 0; i < n; ++i) out[i] = ql::mbqm(x[i], ql::Scale{mult, shift});
@@ -41,13 +37,4 @@ int32_t qmh_hidden_fast(int32_t o, int32_t c, int m, int32_t mult, int32_t shift
     return ql::hidden_q_fast(o, c, m, sc, ql::make_fast_scale(sc), zp);
 }
 uint64_t qmh_isqrt(uint64_t v) { return ql::isqrt64(v); }
-void qmh_layernorm_row(const int16_t *q, int n, const int16_t *L, const int32_t *b, int32_t mult, int32_t shift, int16_t *out)
-{
-    int64_t s = 0, s2 = 0;
-    for (int i = 0; i < n; ++i) { s += q[i]; s2 += (int64_t)q[i] * q[i]; }
-    ql::LnStats st = ql::ln_stats(s, s2, n);
-    for (int i = 0; i < n; ++i) out[i] = (int16_t)ql::ln_apply(q[i], st, L[i], b[i], ql::Scale{mult, shift});
-}
-int32_t qmh_cell_update(int32_t i, int32_t z, int32_t f, int32_t c, int m) { return ql::cell_update(i, z, f, c, m); }
-int32_t qmh_hidden(int32_t o, int32_t c, int m, int32_t mult, int32_t shift, int32_t zp) { return ql::hidden_q(o, c, m, ql::Scale{mult, shift}, zp); }
 }

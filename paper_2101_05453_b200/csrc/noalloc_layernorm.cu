@@ -61,6 +61,8 @@ extern "C" int qlstm_layernorm_rows_static(const int16_t *q_dev, int rows, int n
                                            void *cuda_stream)
 {
     if (rows < 0 || n <= 0 || n > 8191) return QLSTM_ERR_ARG;
+    // same window as qlstm_create: multiplier 0 or in [2^30, 2^31), shift in [-31, 30] (beyond it the shifts are undefined)
+    if (eff_ln.multiplier != 0 && (eff_ln.multiplier < (1 << 30) || eff_ln.shift < -31 || eff_ln.shift > 30)) return QLSTM_ERR_ARG;
     if (rows > MAX_ROWS) return QLSTM_ERR_DIM;                       // beyond the fixed scratch
     if (rows == 0) return QLSTM_OK;
     if (!q_dev || !L_dev || !b_dev || !out_dev) return QLSTM_ERR_ARG;

@@ -25,6 +25,7 @@
 // split into equal contiguous ranges and a CTA touches at most two panels.  x is loaded with an L2
 // evict-last hint and the output stored with evict-first.  No cluster launch and no multicast.
 #include "../../include/qlstm.h"
+#include "../../include/qlstm_debug.h"
 #include "fast_kernels.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"

@@ -11,6 +11,7 @@
 #include <vector>
 
 #include "../../include/qlstm.h"
+#include "../../include/qlstm_debug.h"
 #include "fast_kernels.h"
 #include "qlstm_internal.h"
 
@@ -348,6 +349,9 @@ int qlstm_run(qlstm_t *q, const int8_t *x_dev, int T, int B, int8_t *h_dev, int1
     if (T < 0 || B < 0 || T > q->max_T || B > q->max_B) return QLSTM_ERR_ARG;
     if (T == 0 || B == 0) return QLSTM_OK;
     if (!x_dev || !h_dev || !c_dev || !y_dev) return QLSTM_ERR_ARG;
+    // the kernels use 16-byte vector and bulk accesses on x, y and c (h is re-tiled and may sit anywhere)
+    if ((((uintptr_t)x_dev | (uintptr_t)y_dev | (uintptr_t)c_dev) & 15) != 0) return QLSTM_ERR_ARG;
+    if (trace_dev && ((uintptr_t)trace_dev & 15) != 0) return QLSTM_ERR_ARG;
     if (cudaSetDevice(q->device) != cudaSuccess) return QLSTM_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     q->last_stream = st;
@@ -423,6 +427,7 @@ int qlstm_input_projection(qlstm_t *q, int layer, const int8_t *x_dev, int rows,
     if ((size_t)rows > (size_t)q->max_T * q->max_B) return QLSTM_ERR_ARG;
     if (rows == 0) return QLSTM_OK;
     if (!x_dev || !out_dev) return QLSTM_ERR_ARG;
+    if (((uintptr_t)x_dev & 15) != 0 || ((uintptr_t)out_dev & 31) != 0) return QLSTM_ERR_ARG;   // 32-byte stores to out
     if (cudaSetDevice(q->device) != cudaSuccess) return QLSTM_ERR_CUDA;
     q->last_stream = (cudaStream_t)cuda_stream;
     return run_projection(q, q->layers[layer], x_dev, rows, out_dev, (cudaStream_t)cuda_stream);

@@ -3,7 +3,8 @@
 // Everything here is exact integer arithmetic; where a floating-point unit is used it only
 // produces an estimate that an integer remainder check then corrects, so results never depend
 // on floating-point rounding.  Functions are __host__ __device__ so that the host test harness
-// (csrc/qmath_host_check.cpp) can sweep them on a CPU.
+// (csrc/host_check/qmath_host.cpp) can sweep them on a CPU against fp64 closed forms and exact
+// rational arithmetic.
 //
 // Rounding rule everywhere: to nearest, ties away from zero.
 #pragma once
@@ -22,15 +23,6 @@ struct Scale { int32_t mult; int32_t shift; };   // real = mult * 2^(shift-31)
 QL_HD int32_t sat32(int64_t v) { return v > INT32_MAX ? INT32_MAX : (v < INT32_MIN ? INT32_MIN : (int32_t)v); }
 QL_HD int32_t sat16(int32_t v) { return v > 32767 ? 32767 : (v < -32768 ? -32768 : v); }
 QL_HD int32_t sat8(int32_t v) { return v > 127 ? 127 : (v < -128 ? -128 : v); }
-
-// x / 2^e (0 <= e <= 62), |x| < 2^62
-QL_HD int64_t rdivpot(int64_t x, int e)
-{
-    if (e == 0) return x;
-    uint64_t ax = x < 0 ? (uint64_t)0 - (uint64_t)x : (uint64_t)x;
-    uint64_t q = (ax + ((uint64_t)1 << (e - 1))) >> e;
-    return x < 0 ? -(int64_t)q : (int64_t)q;
-}
 
 // "rescale" (Section 3.2.4): saturating left shift, rounding doubling high multiply, rounding right shift.
 // The multiplier is 0 or in [2^30, 2^31), so the high multiply cannot overflow.
@@ -92,49 +84,9 @@ QL_HD uint64_t isqrt64(uint64_t v)
 }
 
 // ---- integer sigmoid / tanh (Section 3.2.1): int16 Q_{m.15-m} in, Q0.15 out ----------------
-// exp(-k|x|) = 2^-t with t = k|x|log2(e) in Q26; 2^-frac(t) by a degree-6 polynomial around 1/2 in Q30.
-
-QL_HD int64_t exp_neg_q30(int32_t absx, int m, int k)
-{
-    const int64_t LOG2E_Q30 = 1549082005;      // round(2^30 log2 e)
-    const int64_t c0 = 759250125, c1 = -526272083, c2 = 182392005, c3 = -42141501,
-                  c4 = 7302566, c5 = -1012351, c6 = 116951;   // round(2^30 2^-1/2 (-ln 2)^j / j!)
-    int64_t t = rdivpot((int64_t)absx * LOG2E_Q30 * k, 15 - m + 4);
-    int64_t n = t >> 26;
-    if (n > 40) n = 40;
-    int64_t g = (t & (((int64_t)1 << 26) - 1)) - ((int64_t)1 << 25);
-    int64_t acc = c6;
-    acc = rdivpot(acc * g, 26) + c5;
-    acc = rdivpot(acc * g, 26) + c4;
-    acc = rdivpot(acc * g, 26) + c3;
-    acc = rdivpot(acc * g, 26) + c2;
-    acc = rdivpot(acc * g, 26) + c1;
-    acc = rdivpot(acc * g, 26) + c0;
-    return rdivpot(acc, (int)n);
-}
-
-QL_HD int32_t sigmoid_q(int32_t x, int m)
-{
-    int32_t a = x < 0 ? -x : x;
-    int64_t E = exp_neg_q30(a, m, 1);
-    uint64_t D = ((uint64_t)1 << 30) + (uint64_t)E;
-    int32_t S = (int32_t)((((uint64_t)1 << 46) + D) / (2 * D));
-    return x >= 0 ? (S > 32767 ? 32767 : S) : 32768 - S;
-}
-
-QL_HD int32_t tanh_q(int32_t x, int m)
-{
-    int32_t a = x < 0 ? -x : x;
-    int64_t E = exp_neg_q30(a, m, 2);
-    uint64_t D = ((uint64_t)1 << 30) + (uint64_t)E;
-    uint64_t N = ((uint64_t)1 << 30) - (uint64_t)E;
-    int32_t T = (int32_t)((N * 65536 + D) / (2 * D));
-    return x >= 0 ? (T > 32767 ? 32767 : T) : -T;
-}
-
-// ---- the same two functions in 32-bit registers ------------------------------------------------
-// Bit-identical to sigmoid_q / tanh_q above (swept exhaustively on the host and on the GPU), but
-// written for the GPU's integer pipes:
+// exp(-k|x|) = 2^-t with t = k|x|log2(e) in Q26; 2^-frac(t) by a degree-6 polynomial around 1/2 in Q30
+// (coefficients round(2^30 2^-1/2 (-ln 2)^j / j!)), then one division rounded half up.  Written for
+// the GPU's 32-bit integer pipes (swept exhaustively on the host and on the GPU):
 //  * the polynomial variable is pre-shifted by 6 bits so that "/ 2^26" is "take the high word" of one
 //    32x32+64 multiply-add, whose 64-bit addend carries the next coefficient (high word) and the
 //    rounding term (low word).  Rounding half away from zero on a signed product p is
@@ -240,14 +192,8 @@ QL_HD LnStats ln_stats(int64_t sum, int64_t sumsq, int n)
     return s;
 }
 
-// one element: q' = round(2^10 (2^10 q - mean) / sigma); out = sat16(rescale(sat32(q' L + b), eff_ln))
-QL_HD int32_t ln_apply(int32_t q, LnStats s, int32_t L, int32_t b, Scale eff_ln)
-{
-    int64_t qp = s.sigma == 0 ? 0 : rdiv(1024 * (1024 * (int64_t)q - s.mean), s.sigma);
-    return sat16(mbqm(sat32(qp * (int64_t)L + (int64_t)b), eff_ln));
-}
-
-// Per (row, gate) constants of the fast path: fp32 reciprocal of sigma for the quotient estimate.
+// One element: q' = round(2^10 (2^10 q - mean) / sigma); out = sat16(rescale(sat32(q' L + b), eff_ln)).
+// Per (row, gate) constants: mean, sigma and the fp32 reciprocal of sigma for the quotient estimate.
 struct LnRow { int32_t mean; uint32_t sigma; float inv_sigma; };
 
 QL_HD LnRow make_ln_row(LnStats s)
@@ -307,18 +253,6 @@ QL_HD int32_t hidden_q_fast(int32_t o, int32_t c_new, int m, Scale eff_m, const 
 {
     int32_t prod = o * tanh_q_fast(c_new, m);
     return sat8((eff_m.shift <= 0 ? fast_rescale(prod, f_m) : mbqm(prod, eff_m)) + zp_m);
-}
-
-QL_HD int32_t cell_update(int32_t i, int32_t z, int32_t f, int32_t c_old, int m)
-{
-    int64_t iz = rdivpot((int64_t)i * z, 15 + m);
-    int64_t fc = rdivpot((int64_t)f * c_old, 15);
-    return sat16((int32_t)(iz + fc));
-}
-
-QL_HD int32_t hidden_q(int32_t o, int32_t c_new, int m, Scale eff_m, int32_t zp_m)
-{
-    return sat8(mbqm(o * tanh_q(c_new, m), eff_m) + zp_m);
 }
 
 }  // namespace ql

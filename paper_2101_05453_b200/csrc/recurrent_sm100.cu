@@ -23,6 +23,7 @@
 #include <cstring>
 
 #include "../../include/qlstm.h"
+#include "../../include/qlstm_debug.h"
 #include "fast_kernels.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"

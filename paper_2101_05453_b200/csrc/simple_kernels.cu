@@ -96,7 +96,7 @@ __device__ __forceinline__ int32_t gate_input(const LayerParams &p, const Simple
     LnStats st;
     st.mean = s.stats[((size_t)b * p.G + gi) * 2 + 0];
     st.sigma = s.stats[((size_t)b * p.G + gi) * 2 + 1];
-    return ln_apply(pre, st, p.L[n], p.bln[n], p.eff_ln[gi]);
+    return ln_apply_fast(pre, make_ln_row(st), p.L[n], p.bln[n], p.eff_ln[gi], make_fast_scale(p.eff_ln[gi]));
 }
 
 // Everything after the gate sums for one (row, cell).  `finish_o` says whether the output gate can be
@@ -114,16 +114,16 @@ __global__ void k_cell(LayerParams p, int B, int16_t *__restrict__ c, int8_t *__
 
     int32_t af = gate_input(p, s, b, u, sf, pre[sf]);
     int32_t az = gate_input(p, s, b, u, sz, pre[sz]);
-    int32_t f = sigmoid_q(af, 3), z = tanh_q(az, 3), i, ai = 0;
+    int32_t f = sigmoid_q_fast(af, 3), z = tanh_q_fast(az, 3), i, ai = 0;
     if (cifg) {
         i = 32768 - f;                                       // 1 - f in Q0.15 (Section 3.2.9)
         if (i > 32767) i = 32767;
     } else {
         ai = gate_input(p, s, b, u, si, pre[si]);
-        i = sigmoid_q(ai, 3);
+        i = sigmoid_q_fast(ai, 3);
     }
     int32_t c_old = c[tb];
-    int32_t c_new = cell_update(i, z, f, c_old, p.m_bits);
+    int32_t c_new = cell_update_fast(i, z, f, c_old, p.m_bits);
     c[tb] = (int16_t)c_new;
     if (tr.c) {
         tr.ain[0 * tg + tb] = (int16_t)ai; tr.ain[1 * tg + tb] = (int16_t)af; tr.ain[2 * tg + tb] = (int16_t)az;
@@ -142,8 +142,8 @@ __global__ void k_cell(LayerParams p, int B, int16_t *__restrict__ c, int8_t *__
     }
     if (!finish_o) return;
     int32_t ao = gate_input(p, s, b, u, so, pre_o);
-    int32_t o = sigmoid_q(ao, 3);
-    int32_t m = hidden_q(o, c_new, p.m_bits, p.eff_m, p.zp_m);
+    int32_t o = sigmoid_q_fast(ao, 3);
+    int32_t m = hidden_q_fast(o, c_new, p.m_bits, p.eff_m, make_fast_scale(p.eff_m), p.zp_m);
     if (tr.c) { tr.ain[3 * tg + tb] = (int16_t)ao; tr.gate[3 * tg + tb] = (int16_t)o; tr.m[tb] = (int8_t)m; }
     if (proj) {
         s.m[tb] = (int8_t)m;
@@ -163,8 +163,8 @@ __global__ void k_out(LayerParams p, int B, const int16_t *__restrict__ c, int8_
     int u = idx % p.C, b = idx / p.C, so = p.slot_of_gate[3];
     size_t tb = (size_t)b * p.C + u, tg = (size_t)B * p.C;
     int32_t ao = gate_input(p, s, b, u, so, s.pre[(size_t)b * p.N + (size_t)u * p.G + so]);
-    int32_t o = sigmoid_q(ao, 3);
-    int32_t m = hidden_q(o, c[tb], p.m_bits, p.eff_m, p.zp_m);
+    int32_t o = sigmoid_q_fast(ao, 3);
+    int32_t m = hidden_q_fast(o, c[tb], p.m_bits, p.eff_m, make_fast_scale(p.eff_m), p.zp_m);
     if (tr.c) { tr.ain[3 * tg + tb] = (int16_t)ao; tr.gate[3 * tg + tb] = (int16_t)o; tr.m[tb] = (int8_t)m; }
     if (p.flags & F_PROJECTION) {
         s.m[tb] = (int8_t)m;

@@ -1,5 +1,6 @@
-"""The C-ABI library loads and exports every symbol include/qlstm.h declares (no GPU needed)."""
+"""The C-ABI library loads and exports every symbol include/*.h declares (no GPU needed)."""
 import ctypes
+import glob
 import os
 import re
 
@@ -13,9 +14,11 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def declared_symbols():
-    text = open(os.path.join(ROOT, "include", "qlstm.h")).read()
-    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(qlstm_[a-z_]+)\s*\(", text)))
+    names = set()
+    for path in glob.glob(os.path.join(ROOT, "include", "*.h")):
+        text = re.sub(r"/\*.*?\*/", "", open(path).read(), flags=re.S)
+        names |= set(re.findall(r"\b(qlstm_[a-z_0-9]+)\s*\(", text))
+    return sorted(names)
 
 
 def test_header_symbols_are_exported():

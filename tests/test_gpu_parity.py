@@ -150,6 +150,51 @@ def test_full_size_parity_on_sampled_rows(index, rows):
         offs_c += len(rows) * q.n_cell
 
 
+@pytest.mark.parametrize("batch,rows", [(1, [0]), (8, [0, 7]), (64, [0, 63])])
+def test_full_length_parity_config5_batch_sweep(batch, rows):
+    """The production-shaped stack over all 300 steps at the smaller batch sizes of its sweep (the launch
+    configurations whose latency the benchmark reports), against the oracle on sampled rows."""
+    w = make_workload(5, batch=batch)
+    got = run_gpu(w)
+    want = oracle(make_workload(5, rows=rows))
+    assert np.array_equal(got[0][:, rows], want[0]), f"config 5 batch {batch}: y differs on sampled rows"
+    off_h = off_c = offs_h = offs_c = 0
+    for q in w.layers:
+        hg = got[1][off_h:off_h + w.B * q.n_output].reshape(w.B, q.n_output)[rows]
+        cg = got[2][off_c:off_c + w.B * q.n_cell].reshape(w.B, q.n_cell)[rows]
+        hr = want[1][offs_h:offs_h + len(rows) * q.n_output].reshape(len(rows), q.n_output)
+        cr = want[2][offs_c:offs_c + len(rows) * q.n_cell].reshape(len(rows), q.n_cell)
+        assert np.array_equal(hg, hr) and np.array_equal(cg, cr)
+        off_h += w.B * q.n_output
+        off_c += w.B * q.n_cell
+        offs_h += len(rows) * q.n_output
+        offs_c += len(rows) * q.n_cell
+
+
+@pytest.mark.parametrize("kw,B", [(dict(projection=True, layernorm=True), 37), (dict(peephole=True, layernorm=True), 20),
+                                  (dict(cifg=True), 130), (dict(projection=True, peephole=True), 3)],
+                         ids=lambda v: "+".join(sorted(v)) if isinstance(v, dict) else str(v))
+def test_persistent_kernel_cell_state_every_step(kw, B):
+    """The persistent kernel hands back c only at the end of a call, so it is called one step at a time on one
+    handle and c^t, h^t of every layer are compared with the oracle's trace at every step."""
+    import paper_2101_05453_b200 as qlstm
+    w = random_layer_stack(123, 2, 32, 96, 48, T=9, B=B, **kw)
+    _, _, _, tr = oracle(w, trace=True)
+    h, c = w.initial_state()
+    with qlstm.QLSTM(w.layers, 1, w.B) as hnd:
+        for t in range(w.T):
+            y, h, c, _ = run_gpu(w, handle=hnd, impl=(FAST, FAST), x=w.x[t:t + 1], h0=h, c0=c)
+            off_h = off_c = 0
+            for l, q in enumerate(w.layers):
+                ct = c[off_c:off_c + w.B * q.n_cell].reshape(w.B, q.n_cell)
+                ht = h[off_h:off_h + w.B * q.n_output].reshape(w.B, q.n_output)
+                assert np.array_equal(ct, tr[l]["c"][t]), f"{kw}: c of layer {l} differs at step {t}"
+                assert np.array_equal(ht, tr[l]["h"][t]), f"{kw}: h of layer {l} differs at step {t}"
+                off_h += w.B * q.n_output
+                off_c += w.B * q.n_cell
+            assert np.array_equal(y[0], tr[-1]["h"][t])
+
+
 # ------------------------------------------------------------------ pieces and edge cases
 
 @pytest.mark.parametrize("impl", [SIMPLE, AUTO])
@@ -239,6 +284,41 @@ def test_empty_inputs_and_limits():
         with pytest.raises(qlstm.QlstmError) as e:
             hnd.run(None, 4, 2, h, c, y)
         assert e.value.code == qlstm.ERR_ARG
+
+
+def test_misaligned_device_pointers_are_rejected_before_any_launch():
+    """x, c, y (and the projection's output) are accessed with 16- / 32-byte vectors; a sliced pointer is an
+    argument error, not a device fault.  h may sit anywhere."""
+    import torch
+    import paper_2101_05453_b200 as qlstm
+    w = random_layer_stack(57, 1, 32, 64, 64, T=3, B=4)
+    want = oracle(w)
+    h0, c0 = w.initial_state()
+    with qlstm.QLSTM(w.layers, w.T, w.B) as hnd:
+        pad = 64
+        xb = torch.zeros(w.x.size + pad, dtype=torch.int8, device="cuda")
+        yb = torch.zeros(w.T * w.B * 64 + pad, dtype=torch.int8, device="cuda")
+        hb = torch.zeros(h0.size + pad, dtype=torch.int8, device="cuda")
+        cb = torch.zeros(c0.size + pad, dtype=torch.int16, device="cuda")
+        ok = dict(x=xb.data_ptr(), h=hb.data_ptr(), c=cb.data_ptr(), y=yb.data_ptr())
+        for name, off in (("x", 4), ("y", 8), ("c", 2)):
+            args = dict(ok)
+            args[name] += off
+            with pytest.raises(qlstm.QlstmError) as e:
+                hnd.run(args["x"], w.T, w.B, args["h"], args["c"], args["y"])
+            assert e.value.code == qlstm.ERR_ARG, name
+        out = torch.zeros(w.T * w.B * 256 + pad, dtype=torch.int16, device="cuda")
+        with pytest.raises(qlstm.QlstmError) as e:
+            hnd.input_projection(0, ok["x"], w.T * w.B, out.data_ptr() + 16)
+        assert e.value.code == qlstm.ERR_ARG
+        # an odd h pointer is fine
+        xb[:w.x.size] = torch.from_numpy(w.x.reshape(-1)).cuda()
+        hb[3:3 + h0.size] = torch.from_numpy(h0).cuda()
+        cb[:c0.size] = torch.from_numpy(c0).cuda()
+        hnd.run(ok["x"], w.T, w.B, ok["h"] + 3, ok["c"], ok["y"], stream=torch.cuda.current_stream().cuda_stream)
+        hnd.last_status()
+        got = (yb[:w.T * w.B * 64].cpu().numpy().reshape(w.T, w.B, 64), hb[3:3 + h0.size].cpu().numpy(), cb[:c0.size].cpu().numpy())
+        check_equal(got, want, "odd h pointer")
 
 
 def test_bounded_wait_reports_timeout_and_handle_stays_usable():

@@ -1,9 +1,13 @@
-"""The kernels' integer arithmetic (csrc/qmath.cuh), compiled for the host, swept against the oracle.
+"""The kernels' integer arithmetic (csrc/qmath.cuh), compiled for the host and swept on the CPU.
 
-This runs the very source the CUDA kernels compile, on the CPU, so that a wrong shift or rounding in
-the device code shows up without a GPU.  The oracle stays the reference; nothing here feeds it.
+This runs the very source the CUDA kernels compile, so that a wrong shift or rounding in the device
+code shows up without a GPU.  Two kinds of check: against the oracle (the reference; nothing here feeds
+it), and - so that agreement does not rest on the oracle alone - directly against what the mathematics
+fixes: exact rational arithmetic for the rescale, fp64 closed forms for the nonlinearities.
 """
 import ctypes as C
+import math
+from fractions import Fraction
 
 import numpy as np
 import pytest
@@ -19,20 +23,7 @@ def H():
     lib.qmh_mbqm.argtypes = [C.c_int32] * 3
     lib.qmh_isqrt.restype = C.c_uint64
     lib.qmh_isqrt.argtypes = [C.c_uint64]
-    lib.qmh_cell_update.restype = C.c_int32
-    lib.qmh_cell_update.argtypes = [C.c_int32] * 5
-    lib.qmh_hidden.restype = C.c_int32
-    lib.qmh_hidden.argtypes = [C.c_int32] * 6
     return lib
-
-
-@pytest.mark.parametrize("m", [0, 1, 2, 3, 4, 5, 6, 9, 15])
-def test_activations_exhaustive(H, m):
-    out = np.empty(65536, np.int32)
-    H.qmh_sigmoid_all(m, out.ctypes.data_as(C.c_void_p))
-    assert np.array_equal(out, R.sigmoid_all(m))
-    H.qmh_tanh_all(m, out.ctypes.data_as(C.c_void_p))
-    assert np.array_equal(out, R.tanh_all(m))
 
 
 def test_rescale_against_oracle(H):
@@ -78,37 +69,6 @@ def test_isqrt(H):
         assert H.qmh_isqrt(v) == math.isqrt(v)
     for r in [3, 1 << 20, (1 << 25) + 3, (1 << 30) - 1]:
         assert H.qmh_isqrt(r * r) == r and H.qmh_isqrt(r * r - 1) == r - 1
-
-
-@pytest.mark.parametrize("seed", range(8))
-def test_layernorm_rows(H, seed):
-    rng = np.random.default_rng(50 + seed)
-    n = int(rng.integers(1, 2100))
-    q = (rng.integers(-32768, 32768, n) // int(rng.integers(1, 60))).astype(np.int16)
-    if seed == 0:
-        q[:] = 77
-    L = rng.integers(-32767, 32768, n).astype(np.int16)
-    b = (rng.integers(-2 ** 31 + 1, 2 ** 31, n) // int(rng.integers(1, 3000))).astype(np.int32)
-    eff = (int(rng.integers(1 << 30, 1 << 31)), int(rng.integers(-14, -6)))
-    out = np.empty(n, np.int16)
-    H.qmh_layernorm_row(q.ctypes.data_as(C.c_void_p), n, L.ctypes.data_as(C.c_void_p), b.ctypes.data_as(C.c_void_p),
-                        eff[0], eff[1], out.ctypes.data_as(C.c_void_p))
-    assert np.array_equal(out, R.layernorm_row(q, L, b, eff))
-
-
-def test_cell_update_and_hidden(H):
-    rng = np.random.default_rng(2)
-    for _ in range(3000):
-        i, f, o = (int(v) for v in rng.integers(0, 32768, 3))
-        z, c = (int(v) for v in rng.integers(-32768, 32768, 2))
-        m = int(rng.integers(0, 7))
-        want_c = R.rdivpot(i * z, 15 + m) + R.rdivpot(f * c, 15)
-        want_c = max(-32768, min(32767, want_c))
-        assert H.qmh_cell_update(i, z, f, c, m) == want_c
-        eff = (int(rng.integers(1 << 30, 1 << 31)), -22)
-        zp = int(rng.integers(-128, 128))
-        want_m = max(-128, min(127, R.mbqm(o * R.tanh(want_c, m), eff) + zp))
-        assert H.qmh_hidden(o, want_c, m, eff[0], eff[1], zp) == want_m
 
 
 # ---------------------------------------------------------------- the 32-bit / fp32-assisted forms the kernels run
@@ -174,3 +134,71 @@ def test_fast_cell_update_and_hidden(H):
         eff = (int(rng.integers(1 << 30, 1 << 31)), int(rng.integers(-24, -18))); zp = int(rng.integers(-128, 128))
         want = max(-128, min(127, R.mbqm(o * R.tanh(c, m), eff) + zp))
         assert H.qmh_hidden_fast(o, c, m, eff[0], eff[1], zp) == want
+
+
+# ---------------------------------------------------------------- directly against the mathematics
+
+def _round_half_away(fr: Fraction) -> int:
+    n = abs(fr)
+    q = (n.numerator * 2 + n.denominator) // (2 * n.denominator)
+    return -q if fr < 0 else q
+
+
+def test_rescale_forms_against_exact_rationals(H):
+    """rescale(x, (M, s)) = round(round(x 2^max(s,0) M / 2^31) / 2^max(-s,0)), both roundings half away from zero."""
+    rng = np.random.default_rng(21)
+    xs = [int(v) for v in rng.integers(-2 ** 31, 2 ** 31, 400)] + [0, 1, -1, 5, -5, 2 ** 31 - 1, -2 ** 31, 12345, -32768]
+    scales = [(1 << 30, 0), ((1 << 31) - 1, -7), (1 << 30, -1), (1 << 30, 1)] + \
+        [(int(rng.integers(1 << 30, 1 << 31)), int(s)) for s in (-31, -20, -12, -5, -1, 0, 2, 6)]
+    out = np.empty(len(xs), np.int32)
+    xa = np.array(xs, np.int32)
+    for M, s in scales:
+        def exact(x):
+            left, right = max(s, 0), max(-s, 0)
+            xl = max(-2 ** 31, min(2 ** 31 - 1, x << left))
+            first = _round_half_away(Fraction(xl * M, 2 ** 31))
+            return _round_half_away(Fraction(first, 2 ** right))
+        want = np.array([exact(x) for x in xs], np.int64)
+        H.qmh_mbqm_many(xa.ctypes.data_as(C.c_void_p), len(xs), M, s, out.ctypes.data_as(C.c_void_p))
+        assert np.array_equal(out, want), (M, s)
+        if s <= 0:
+            H.qmh_fast_rescale_many(xa.ctypes.data_as(C.c_void_p), len(xs), M, s, out.ctypes.data_as(C.c_void_p))
+            assert np.array_equal(out, want), (M, s)
+
+
+@pytest.mark.parametrize("m", [0, 3, 4, 6])
+def test_fast_activations_against_fp64_closed_forms(H, m):
+    """Section 3.2.1: Q_{m.15-m} in, Q0.15 out, clamped to [-1, 32767/32768]."""
+    x = np.arange(-32768, 32768, dtype=np.float64) * 2.0 ** (m - 15)
+    out = np.empty(65536, np.int32)
+    for fn, f64 in ((H.qmh_sigmoid_fast_all, 1.0 / (1.0 + np.exp(-x))), (H.qmh_tanh_fast_all, np.tanh(x))):
+        fn(m, out.ctypes.data_as(C.c_void_p))
+        true = 32768.0 * f64
+        err = np.abs(out - true)
+        assert err.max() <= 1.0                                  # the forced clamp at +32767 costs up to one step
+        assert err[true <= 32767.0].max() <= 0.51
+        assert np.all(np.diff(out) >= 0)                         # monotone
+    H.qmh_sigmoid_fast_all(m, out.ctypes.data_as(C.c_void_p))
+    assert out[32768] == 16384 and out.min() >= 0 and out.max() <= 32767
+    H.qmh_tanh_fast_all(m, out.ctypes.data_as(C.c_void_p))
+    assert out[32768] == 0 and out.min() >= -32768 and out.max() <= 32767
+
+
+def test_fast_layernorm_against_fp64_layer_norm(H):
+    """Section 3.2.6: out = (x - mean) / std * L + b in Q3.12, within the quantization of its parts."""
+    rng = np.random.default_rng(5)
+    n = 1536
+    q = np.clip(np.rint(rng.normal(300.0, 4000.0, n)), -32768, 32767).astype(np.int16)
+    s_L = 1.3 / 32767.0
+    Lr, br = rng.normal(1.0, 0.1, n), rng.normal(0.0, 0.1, n)
+    L = np.rint(Lr / s_L).astype(np.int16)
+    b = np.rint(br / (s_L * 2.0 ** -10)).astype(np.int32)
+    real = s_L * 2.0 ** -10 / 2.0 ** -12
+    frac, exp = math.frexp(real)
+    eff = (int(round(frac * (1 << 31))), exp)
+    out = np.empty(n, np.int16)
+    H.qmh_layernorm_row_fast(q.ctypes.data_as(C.c_void_p), n, L.ctypes.data_as(C.c_void_p), b.ctypes.data_as(C.c_void_p),
+                             eff[0], eff[1], out.ctypes.data_as(C.c_void_p))
+    qf = q.astype(float)
+    want = (qf - qf.mean()) / qf.std() * (L * s_L) + b * (s_L * 2.0 ** -10)
+    assert np.abs(out / 4096.0 - want).max() <= 3e-3             # q' is on a 2^-10 grid: about 1e-3 per unit of L

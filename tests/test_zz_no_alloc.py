@@ -6,7 +6,7 @@ need a result (a real-time per-frame loop, a process whose own arena owns the wh
 callback); its only scratch is a fixed array inside the library, shared by all calls.  The test calls it
 twice in a row - the second time with fewer rows, a different width and different data, so that anything
 wrongly carried over in that array from the first call would show - and checks every row bit for bit
-against qlstm_eval_layernorm_row.
+against qlstm_eval_layernorm_row, and against the CPU oracle's layer norm as well.
 """
 import numpy as np
 import pytest
@@ -55,6 +55,9 @@ def test_static_scratch_layernorm_matches_per_row_entry_point_twice():
         got = _run_static(binding, torch, q, L, b, eff)
         want = _run_per_row(binding, torch, q, L, b, eff)
         assert np.array_equal(got, want)                 # integer arithmetic: bit exact
+        from oracle import qlstm_ref
+        for r in range(q.shape[0]):
+            assert np.array_equal(got[r], qlstm_ref.layernorm_row(q[r], L, b, eff)), r
 
 
 def test_static_scratch_size_limit_is_reported():
@@ -67,3 +70,19 @@ def test_static_scratch_size_limit_is_reported():
     with pytest.raises(qlstm.QlstmError) as e:
         binding.layernorm_rows_static(q, 4097, 16, L, b, (1 << 30, -10), q)
     assert e.value.code == qlstm.ERR_DIM
+
+
+def test_static_scratch_rejects_scales_outside_the_encodable_window():
+    import torch
+    import paper_2101_05453_b200 as qlstm
+    from paper_2101_05453_b200 import binding
+    q = torch.zeros((1, 16), dtype=torch.int16, device="cuda")
+    L = torch.ones(16, dtype=torch.int16, device="cuda")
+    b = torch.zeros(16, dtype=torch.int32, device="cuda")
+    for eff in ((1 << 30, -32), (1 << 29, -5), (1 << 30, 31)):
+        with pytest.raises(qlstm.QlstmError) as e:
+            binding.layernorm_rows_static(q, 1, 16, L, b, eff, q)
+        assert e.value.code == qlstm.ERR_ARG
+        with pytest.raises(qlstm.QlstmError) as e:
+            binding.eval_layernorm_row(q, 16, L, b, eff, q)
+        assert e.value.code == qlstm.ERR_ARG
