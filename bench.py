@@ -324,33 +324,55 @@ def main():
     e2e_matches = bool(np.array_equal(yh.numpy(), y.cpu().numpy()))
 
     # ---- rooflines.  Input projection: dense int8 contraction on the tensor cores.  Recurrent kernel: the slower of
-    # its int8 matmuls at tensor peak and its per-step bytes; both are far below the time it takes, which is
-    # integer-ALU and barrier time (reported as measured).
+    # its int8 matmuls at tensor peak and its per-step bytes are both far below the time it takes, which is
+    # integer-ALU and barrier time; its headline fraction is against the integer-pipe peak, with the matmul and byte
+    # fractions beside it.
     gemm_ops, rec_ops = algorithmic_ops(w.layers, B, T)
-    int8_peak = 2.0 * peaks["bf16_tflops_sustained"]          # TOP/s: bf16 measured x nominal int8:bf16 ratio of 2
+    int8_sustained = 2.0 * peaks["bf16_tflops_sustained"]     # TOP/s: bf16 measured x nominal int8:bf16 ratio of 2
+    int8_burst = 2.0 * peaks["bf16_tflops"]
     n_l = len(w.layers)
     proj_ms = prof["projection_ms"] / max(args.steps, 1)
     rec_ms = prof["recurrent_ms"] / max(args.steps, 1)
     proj_tops = gemm_ops / (proj_ms * 1e-3) / 1e12 if proj_ms > 0 else 0.0
     rec_tops = rec_ops / (rec_ms * 1e-3) / 1e12 if rec_ms > 0 else 0.0
-    roof_proj = {"kernel": "input_projection", "bound": "tensor", "achieved": proj_tops, "peak": int8_peak,
-                 "unit": "TOP/s", "frac": proj_tops / int8_peak, "traffic": None,
-                 "peak_source": f"2 x bf16 sustained, {peaks['source']}", "ms_per_launch": proj_ms / n_l}
+    sm_mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0
+    sm_max = clocks.get("sm_max_mhz") or 1965.0
+    mma_peak = None
+    if rank == 0:
+        try:
+            from paper_2101_05453_b200 import binding
+            mma_peak = binding.mma_i8_peak(local, 20000)
+        except Exception:
+            mma_peak = None
+    roof_proj = {"kernel": "input_projection", "bound": "tensor", "achieved": proj_tops, "peak": int8_sustained,
+                 "unit": "TOP/s", "frac": proj_tops / int8_sustained, "traffic": None,
+                 "peak_source": f"2 x bf16 sustained ({peaks['source']}): the kernel is timed inside the long pass",
+                 "frac_vs_2x_bf16_burst": proj_tops / int8_burst,
+                 "measured_mma_i8_issue_peak_tops": mma_peak,
+                 "frac_vs_measured_mma_issue_peak": (proj_tops / mma_peak) if mma_peak else None,
+                 "achieved_at_max_clock": proj_tops * sm_max / sm_mhz,
+                 "ms_per_launch": proj_ms / n_l}
     if (args.config == NCU_PROJECTION["config"] and B * T == NCU_PROJECTION["rows"]
             and projection_source_sha() == NCU_PROJECTION["source_sha"]):
         roof_proj["traffic"] = NCU_PROJECTION["bytes"]                                   # bytes per launch (one layer)
     q0 = w.layers[0]
-    roof_proj["algorithmic_hbm_bytes"] = B * T * q0.n_input + q0.n_input * q0.n_cell * (3 if (q0.flags & 8) else 4) \
-        + 2 * B * T * q0.n_cell * (3 if (q0.flags & 8) else 4)
+    G0 = 3 if (q0.flags & 8) else 4
+    roof_proj["algorithmic_hbm_bytes"] = B * T * q0.n_input + q0.n_input * q0.n_cell * G0 + 2 * B * T * q0.n_cell * G0
+    roof_proj["hbm_frac"] = roof_proj["algorithmic_hbm_bytes"] / (proj_ms / n_l * 1e-3) / 1e9 / peaks["hbm_gbs"] if proj_ms > 0 else None
     int_ops = algorithmic_int_ops(w.layers, B, T)
-    sm_ghz = (clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0) / 1e3
+    sm_ghz = sm_mhz / 1e3
     alu_peak = 148 * INT_LANES_PER_SM * sm_ghz / 1e3                     # T int-op/s at the clock seen during the run
     rec_alu = int_ops / (rec_ms * 1e-3) / 1e12 if rec_ms > 0 else 0.0
+    rec_bytes = T * B * (q0.n_cell * G0 * 2 + q0.n_output) + 2 * B * (q0.n_output + 2 * q0.n_cell)
     roof_rec = {"kernel": "recurrent", "bound": "alu", "achieved": rec_alu, "peak": alu_peak, "unit": "Tint-op/s",
                 "frac": rec_alu / alu_peak, "traffic": None,
-                "peak_source": f"148 SMs x {INT_LANES_PER_SM} int32 lanes x {sm_ghz:.3f} GHz (SM clock sampled during the run)",
+                "peak_source": f"148 SMs x {INT_LANES_PER_SM} int32 lanes x {sm_ghz:.3f} GHz (SM clock sampled during the run); "
+                               "a derived model: the per-unit operation counts are this library's own leanest forms",
+                "frac_vs_issue_peak_128_per_clk": rec_alu / (2 * alu_peak),
                 "algorithmic_int_ops_per_launch": int_ops / n_l,
-                "matmul_tops": rec_tops, "matmul_frac_of_int8_peak": rec_tops / int8_peak,
+                "matmul_tops": rec_tops, "matmul_frac_of_int8_peak": rec_tops / int8_sustained,
+                "matmul_frac_of_2x_bf16_burst": rec_tops / int8_burst,
+                "hbm_frac": rec_bytes / (rec_ms / n_l * 1e-3) / 1e9 / peaks["hbm_gbs"] if rec_ms > 0 else None,
                 "ms_per_launch": rec_ms / n_l,
                 "us_per_layer_step": 1e3 * rec_ms / (n_l * T),
                 "phase_us_per_layer_step": {k: 1e3 * prof_phase[k] / (n_l * T) for k in
@@ -361,9 +383,7 @@ def main():
             and recurrent_source_sha() == NCU_RECURRENT["source_sha"]):
         roof_rec["traffic"] = NCU_RECURRENT["bytes"] * T / NCU_RECURRENT["steps"]      # bytes per launch (one layer)
     # algorithmic HBM bytes of the recurrent kernel per launch: X read once, y written once, state in and out
-    q0 = w.layers[0]
-    G0 = 3 if (q0.flags & 8) else 4
-    roof_rec["algorithmic_hbm_bytes"] = T * B * (q0.n_cell * G0 * 2 + q0.n_output) + 2 * B * (q0.n_output + 2 * q0.n_cell)
+    roof_rec["algorithmic_hbm_bytes"] = rec_bytes
     dominant = roof_rec if rec_ms >= proj_ms else roof_proj
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -377,80 +397,110 @@ def main():
             "gpu_launches": prof["projection_launches"] + prof["recurrent_launches"] + prof["other_launches"],
             "roofline": dominant, "roofline_projection": roof_proj, "roofline_recurrent": roof_rec}
 
+    def time_passes(qh, wl, n_warm=3, n_timed=3, impl=None, profile=False):
+        """Median pass time (ms) of workload wl on handle qh with everything resident; optionally the per-kernel profile."""
+        if impl is not None:
+            qh.set_impl(*impl)
+        xs = torch.from_numpy(wl.x).to(dev)
+        hs0, cs0 = wl.initial_state()
+        hs, cs = torch.from_numpy(hs0).to(dev), torch.from_numpy(cs0).to(dev)
+        ys = torch.zeros((wl.T, wl.B, wl.layers[-1].n_output), dtype=torch.int8, device=dev)
+        ts = []
+        qh.set_profiling(1 if profile else 0)
+        for i in range(n_warm + n_timed):
+            if i == n_warm and profile:
+                qh.get_profile(reset=True)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            qh.run(xs, wl.T, wl.B, hs, cs, ys, stream=stream)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= n_warm:
+                ts.append(a.elapsed_time(b))
+        qh.last_status()
+        pr = qh.get_profile(reset=True) if profile else None
+        qh.set_profiling(0)
+        return statistics.median(ts), pr, n_timed
+
+    def streaming_us(qh, wl, n_calls=60):
+        """One time step per call on the default stream, state carried by the caller: microseconds per call."""
+        xs1 = torch.from_numpy(wl.x[:1]).to(dev).contiguous()
+        hs0, cs0 = wl.initial_state()
+        hs, cs = torch.from_numpy(hs0).to(dev), torch.from_numpy(cs0).to(dev)
+        ys1 = torch.zeros((1, wl.B, wl.layers[-1].n_output), dtype=torch.int8, device=dev)
+        for _ in range(10):
+            qh.run(xs1, 1, wl.B, hs, cs, ys1, stream=stream)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(n_calls):
+            qh.run(xs1, 1, wl.B, hs, cs, ys1, stream=stream)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        qh.last_status()
+        return 1e6 * dt / n_calls
+
+    def config_entry(index, Bc, with_oracle=True):
+        """One row of the per-configuration table: whole pass, its two kernels, and the oracle on a bounded sample."""
+        wl = make_workload(index, batch=Bc)
+        qh = qlstm.QLSTM(wl.layers, wl.T, wl.B, device=local)
+        ms, pr, n = time_passes(qh, wl, profile=True)
+        nl = len(wl.layers)
+        g_ops, _ = algorithmic_ops(wl.layers, wl.B, wl.T)
+        ent = {"workload": f"config{index}-{wl.config.name} batch {wl.B} T {wl.T}", "value": wl.B * wl.T / (ms * 1e-3), "unit": UNIT,
+               "ms_per_pass": ms, "us_per_timestep_whole_stack": 1e3 * ms / wl.T}
+        if pr["projection_launches"] > 0:
+            p_ms = pr["projection_ms"] / n
+            tops = g_ops / (p_ms * 1e-3) / 1e12
+            ent.update(path="per layer: projection GEMM + persistent recurrent kernel", projection_us_per_launch=1e3 * p_ms / nl,
+                       projection_tops=tops, projection_frac_of_2x_bf16_sustained=tops / int8_sustained,
+                       projection_frac_of_2x_bf16_burst=tops / int8_burst,
+                       recurrent_us_per_layer_step=1e3 * pr["recurrent_ms"] / (n * nl * wl.T))
+        else:
+            ent.update(path="whole-stack kernel (layers as a wavefront, input projection inside the step)",
+                       us_per_layer_step=1e3 * ms / (nl * wl.T))
+        if wl.B <= 4:
+            ent["streaming_us_per_call_T1"] = streaming_us(qh, wl)
+        qh.close()
+        if with_oracle and not args.no_cpu_baseline:
+            from oracle import qlstm_ref
+            cores = qlstm_ref.num_threads()
+            rows_n = max(1, min(wl.B, cores))
+            v0, dt0, _ = oracle_sample(index, cores, 2, rows_n)
+            T_s = int(max(2, min(wl.T, 2.5 / max(dt0 / 2, 1e-6))))
+            v, dt, cores = oracle_sample(index, cores, T_s, rows_n)
+            ent["cpu_oracle"] = {"value": v, "unit": UNIT, "cores": cores, "sample": f"{rows_n} rows x {T_s} steps, {dt:.1f} s"}
+        return ent
+
     if rank == 0:
         if not args.no_latency and args.config == 5:
-            # batch-1 per-step latency on the same model
+            # batch-1 latency on the same model: whole-stack kernel, against the layer-after-layer path
             w1 = make_workload(5, batch=1, T=T)
             q1 = qlstm.QLSTM(w1.layers, T, 1, device=local)
-            x1 = torch.from_numpy(w1.x).to(dev)
-            hi, ci = w1.initial_state()
-            h1, c1 = torch.from_numpy(hi).to(dev), torch.from_numpy(ci).to(dev)
-            y1 = torch.zeros((T, 1, O), dtype=torch.int8, device=dev)
-            ts = []
-            q1.set_profiling(1)
-            for i in range(7):
-                if i == 3:
-                    q1.get_profile(reset=True)
-                if i == 6:                        # one extra pass with the device phase timers, not part of the latency
-                    p1 = q1.get_profile(reset=True)
-                    q1.set_profiling(2)
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record()
-                q1.run(x1, T, 1, h1, c1, y1, stream=stream)
-                b.record()
-                torch.cuda.synchronize()
-                if 3 <= i < 6:
-                    ts.append(a.elapsed_time(b))
-            q1.last_status()
-            p1_phase = q1.get_profile(reset=True)
-            ms = statistics.median(ts)
-            line["latency_batch1"] = {"us_per_timestep_whole_stack": 1e3 * ms / T,
-                                      "us_per_layer_step": 1e3 * ms / (T * n_l), "ms_per_pass": ms,
-                                      "projection_us_per_layer": 1e3 * p1["projection_ms"] / (len(ts) * n_l),
-                                      "phase_us_per_layer_step": {k: 1e3 * p1_phase[k] / (n_l * T) for k in
-                                                                  ("phase_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms",
-                                                                   "phase_c_ms", "wait_c_ms")}}
-            # streaming use: one timestep per call, state carried by the caller (every call pays all launches of the stack)
-            n_calls = 60
-            xs1 = x1[:1].contiguous()
-            ys1 = torch.zeros((1, 1, O), dtype=torch.int8, device=dev)
-            q1.set_profiling(0)
-            for i in range(10):
-                q1.run(xs1, 1, 1, h1, c1, ys1, stream=stream)
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            for i in range(n_calls):
-                q1.run(xs1, 1, 1, h1, c1, ys1, stream=stream)
-            torch.cuda.synchronize()
-            line["latency_batch1"]["streaming_us_per_call_T1"] = 1e6 * (time.perf_counter() - t0) / n_calls
-            q1.last_status()
+            ms, _, _ = time_passes(q1, w1)
+            ms_layers, pr_l, n = time_passes(q1, w1, impl=(0, 2), profile=True)
+            q1.set_impl(0, 0)
+            line["latency_batch1"] = {"us_per_timestep_whole_stack": 1e3 * ms / T, "us_per_layer_step": 1e3 * ms / (T * n_l),
+                                      "ms_per_pass": ms, "kernel": "whole-stack kernel, one launch for all layers and steps",
+                                      "layer_after_layer_us_per_timestep": 1e3 * ms_layers / T,
+                                      "layer_after_layer_recurrent_us_per_layer_step": 1e3 * pr_l["recurrent_ms"] / (n * n_l * T),
+                                      "streaming_us_per_call_T1": streaming_us(q1, w1)}
             q1.close()
-            # the other batch sizes of the configuration's sweep (1 is above, the timed workload is the largest)
-            sweep = {}
-            for Bs in (8, 64):
-                if Bs == B:
-                    continue
-                ws = make_workload(5, batch=Bs, T=T)
-                qs = qlstm.QLSTM(ws.layers, T, Bs, device=local)
-                xs = torch.from_numpy(ws.x).to(dev)
-                hs0, cs0 = ws.initial_state()
-                hs, cs = torch.from_numpy(hs0).to(dev), torch.from_numpy(cs0).to(dev)
-                ys = torch.zeros((T, Bs, O), dtype=torch.int8, device=dev)
-                tsw = []
-                for i in range(6):
-                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    a.record()
-                    qs.run(xs, T, Bs, hs, cs, ys, stream=stream)
-                    b.record()
-                    torch.cuda.synchronize()
-                    if i >= 3:
-                        tsw.append(a.elapsed_time(b))
-                qs.last_status()
-                qs.close()
-                ms = statistics.median(tsw)
-                sweep[str(Bs)] = {"value": Bs * T / (ms * 1e-3), "unit": UNIT, "ms_per_pass": ms,
-                                  "us_per_layer_step": 1e3 * ms / (T * n_l)}
-            line["batch_sweep"] = sweep
+            try:
+                from paper_2101_05453_b200 import binding
+                bar_us = binding.barrier_latency_us(local, 3000)
+                phases = 3 if (w.layers[0].flags & 1) else 2
+                line["barrier_floor"] = {"us_per_grid_barrier": bar_us, "barriers_per_layer_step": phases,
+                                         "us_per_layer_step": bar_us * phases,
+                                         "how": "3000 grid-wide barriers back to back, one block per SM, nothing in between"}
+            except Exception as exc:                                   # reported, never fatal
+                line["barrier_floor"] = {"error": str(exc)}
+            # the other batch sizes of the configuration's sweep, then the other configurations
+            per = {}
+            for Bs in (1, 8, 64):
+                per[f"config5_batch{Bs}"] = config_entry(5, Bs, with_oracle=False)
+            line["batch_sweep"] = {k.split("batch")[1]: {"value": v["value"], "unit": UNIT, "ms_per_pass": v["ms_per_pass"],
+                                                         "us_per_layer_step": 1e3 * v["ms_per_pass"] / (T * n_l)}
+                                   for k, v in per.items()}
         if not args.no_cpu_baseline:
             from oracle import qlstm_ref
             cores = qlstm_ref.num_threads()
@@ -460,6 +510,11 @@ def main():
             v, dt, cores = oracle_sample(args.config, cores, T_s, rows_n)
             line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                     "sample": f"{rows_n} batch rows x {T_s} timesteps of the same workload, {dt:.1f} s"}
+        if not args.no_latency and args.config == 5:
+            for index in (1, 2, 3, 4):
+                per[f"config{index}"] = config_entry(index, None)
+            per["config1"]["us_per_step_batch1"] = per["config1"]["us_per_timestep_whole_stack"]
+            line["per_config"] = per
         print(json.dumps(line))
     q.close()
     if dist is not None:

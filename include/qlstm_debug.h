@@ -17,11 +17,14 @@ extern "C" {
 /* Kernel selection, for tests and measurements.  0 = automatic (default), 1 = simple kernels
  * (one thread per output, one launch per phase), 2 = fast kernels (tensor-core projection,
  * persistent recurrent kernel); 2 fails with QLSTM_ERR_DIM at run time if a shape is unsupported.
- * recurrent_impl 3 = like 2 but with the tensor-core matmuls even at batch <= 4, where 0 and 2 use dp4a mat-vecs;
- * 4 = like 2 but with the dp4a mat-vecs up to batch 16 (the crossover is a measured default, not a limit). */
+ * recurrent_impl 2 always runs layer after layer (projection launch + persistent kernel per layer), where 0 takes the
+ * whole-stack kernel at batch <= 4; 3 = like 2 but with the tensor-core matmuls even at batch <= 4, where 2 uses dp4a
+ * mat-vecs; 4 = like 2 but with the dp4a mat-vecs up to batch 16 (the crossover is a measured default, not a limit);
+ * 5 = the whole-stack kernel or QLSTM_ERR_DIM (batch > 4, or a dimension that is not a multiple of 16). */
 int qlstm_set_impl(qlstm_t *q, int projection_impl, int recurrent_impl);
 
-/* Failure-path check: with missing_arrivals > 0 every grid barrier of the persistent recurrent kernel waits for
+/* Failure-path check: with missing_arrivals > 0 every grid barrier of the persistent recurrent kernel (and every
+ * counter wait of the whole-stack kernel) waits for
  * that many arrivals that never come, for at most limit_ns (<= 1 s); the wait then runs out, the kernel sets its
  * status word, every block leaves the time loop, frees its tensor memory and returns, and qlstm_last_status
  * reports QLSTM_ERR_TIMEOUT.  Nothing faults or hangs and the handle stays usable; 0 restores normal operation. */
@@ -78,6 +81,16 @@ int qlstm_get_profile(qlstm_t *q, qlstm_profile_t *out, int reset);
 int qlstm_eval_activations(int cell_int_bits, int16_t *sigmoid_dev, int16_t *tanh_dev, void *cuda_stream);
 int qlstm_eval_layernorm_row(const int16_t *q_dev, int n, const int16_t *L_dev, const int32_t *b_dev,
                              qlstm_scale_t eff_ln, int16_t *out_dev, void *cuda_stream);
+
+/* Two measurements the roofline statements rest on, each a kernel of its own on device `device` (no handle needed).
+ *   qlstm_debug_mma_i8_peak: every SM issues `iters` x 4 back-to-back tcgen05.mma kind::i8 (M128 N256 K32) from
+ *     operands resident in shared memory; *tops_out = achieved int8 TOP/s (best of three timed launches).  This is the
+ *     measured issue-rate peak of the tensor path that the input projection of Section 3.2.4 runs on.
+ *   qlstm_debug_barrier_latency: n_barriers grid-wide barriers of the persistent kernel's kind back to back on one
+ *     block per SM; *us_per_barrier_out = microseconds per barrier (the floor of every phase boundary of a time step).
+ * QLSTM_ERR_ARG on bad arguments, QLSTM_ERR_TIMEOUT if a (bounded) wait inside the kernel ran out. */
+int qlstm_debug_mma_i8_peak(int device, int iters, double *tops_out);
+int qlstm_debug_barrier_latency(int device, int n_barriers, double *us_per_barrier_out);
 
 /* Device properties the library sees: SM count, and resident blocks of the persistent kernel. */
 int qlstm_device_info(qlstm_t *q, int *sm_count, int *persistent_blocks);

@@ -23,7 +23,7 @@ EXPORTS = ["qlstm_create", "qlstm_run", "qlstm_run_host", "qlstm_input_projectio
            "qlstm_destroy", "qlstm_strerror", "qlstm_trace_bytes", "qlstm_set_impl", "qlstm_set_profiling",
            "qlstm_get_profile", "qlstm_device_info", "qlstm_eval_activations", "qlstm_eval_layernorm_row",
            "qlstm_layernorm_rows_static", "qlstm_debug_barrier_timeout", "qlstm_debug_ring_plan",
-           "qlstm_debug_projection_plan"]
+           "qlstm_debug_projection_plan", "qlstm_debug_mma_i8_peak", "qlstm_debug_barrier_latency"]
 
 
 class Scale(C.Structure):
@@ -108,6 +108,10 @@ def lib():
         L.qlstm_debug_projection_plan.restype = C.c_int
         L.qlstm_debug_projection_plan.argtypes = [C.c_longlong, C.c_longlong, C.c_int, C.c_int, C.c_int, C.c_int,
                                                   C.POINTER(C.c_int)]
+        L.qlstm_debug_mma_i8_peak.restype = C.c_int
+        L.qlstm_debug_mma_i8_peak.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double)]
+        L.qlstm_debug_barrier_latency.restype = C.c_int
+        L.qlstm_debug_barrier_latency.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double)]
         L.qlstm_layernorm_rows_static.restype = C.c_int
         L.qlstm_layernorm_rows_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p,
                                                   C.c_void_p]
@@ -306,3 +310,17 @@ def projection_plan(rows: int, n_gate_rows: int, n_input: int, sm_count: int = 1
            "qlstm_debug_projection_plan")
     v = list(out)
     return {"bn": v[0], "stages": v[1], "per_cta": v[2], "m_ranges": v[3], "grid": v[4]}
+
+
+def mma_i8_peak(device: int = 0, iters: int = 20000) -> float:
+    """Measured int8 TOP/s of back-to-back tcgen05.mma kind::i8 from resident operands on every SM."""
+    out = C.c_double()
+    _check(lib().qlstm_debug_mma_i8_peak(device, iters, C.byref(out)), "qlstm_debug_mma_i8_peak")
+    return out.value
+
+
+def barrier_latency_us(device: int = 0, n_barriers: int = 2000) -> float:
+    """Microseconds per grid-wide barrier of the persistent kernel's kind, executed back to back."""
+    out = C.c_double()
+    _check(lib().qlstm_debug_barrier_latency(device, n_barriers, C.byref(out)), "qlstm_debug_barrier_latency")
+    return out.value

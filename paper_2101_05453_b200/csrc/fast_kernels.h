@@ -4,6 +4,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <vector>
+
 #include "qlstm_internal.h"
 
 namespace ql {
@@ -15,7 +17,7 @@ struct FastScratch {
     int8_t *hbuf = nullptr;      // [2][Bpad x max O]  h^{t-1} / h^t, the recurrent matmul's A operand (tiled k-block image,
                                  //                    plain rows at small batch)
     int8_t *mbuf = nullptr;      // [Bpad x max C]     hidden state m, the projection's A operand (same layouts)
-    int32_t *pre = nullptr;      // [max B][max N]    gate sums between the matmul and elementwise phases
+    int32_t *pre = nullptr;      // [max B][max N]    layer norm: gate sums between the matmul and elementwise phases
                                  //                   (int16 values, or int32 X+H when a peephole follows)
     unsigned *bar = nullptr;     // [0] grid-barrier counter, [1] abort word
     size_t hbuf_bytes = 0, mbuf_bytes = 0;
@@ -65,6 +67,18 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
 
 // Host logic of the recurrent kernel's operand ring, for tests: fills out[14] = n_own, n_max, n_chunks[4], cnt[4],
 // uses[4] of the plan for `stages` ring stages and `n_own` issuers (see RingPlan in recurrent_sm100.cu).
+// ---- whole-stack kernel for small batches (stack_small_sm100.cu): all layers and steps in one cooperative launch,
+// one group of blocks per layer, layers running as a wavefront; also the path of one-step (streaming) calls.
+constexpr int STACK_SMALL_MAX_B = 4;
+struct StackSmall;
+int stack_small_create(const std::vector<const LayerParams *> &layers, int max_T, int max_B, int sm_count, StackSmall **out);
+void stack_small_destroy(StackSmall *s);
+bool stack_small_supported(const StackSmall *s, int T, int B);
+int launch_stack_small(const StackSmall *s, const int8_t *x, int T, int B, int8_t *h, int16_t *c, int8_t *y, int *status,
+                       cudaStream_t st);
+void stack_small_debug_timeout(StackSmall *s, unsigned missing_arrivals, unsigned long long limit_ns);
+int stack_small_groups(const StackSmall *s, int *blocks_per_layer);     // layers, and the blocks each layer's group has
+
 int debug_ring_plan(int stages, int n_own, int contig, int per, int n_total, int *out);
 int debug_projection_plan(long long rows_hint, long long rows, int N, int K, int sm_count, int max_smem, int *out5);
 

@@ -38,6 +38,7 @@ struct qlstm {
     int8_t *seq[2] = {nullptr, nullptr};
     SimpleScratch scratch = {};
     FastScratch fscratch = {};
+    StackSmall *stack = nullptr;    // whole-stack kernel for small batches, or null
     int *status = nullptr;          // device status word of the persistent kernel
     unsigned long long *phase_ns = nullptr;   // device phase timers of the persistent kernel (profiling)
     // staging for qlstm_run_host
@@ -308,6 +309,12 @@ int qlstm_create(const qlstm_layer_t *layers, int n_layers, int max_T, int max_B
         int frc = fast_layer_init(q->layers[l].fast, q->layers[l].p, q->fscratch, max_T, max_B);
         if (frc != QLSTM_OK) { ok = false; rc = frc; }
     }
+    if (ok) {
+        std::vector<const LayerParams *> lp;
+        for (auto &L : q->layers) lp.push_back(&L.p);
+        int src = stack_small_create(lp, max_T, max_B, q->sm_count, &q->stack);
+        if (src != QLSTM_OK) { ok = false; rc = src; }
+    }
     if (!ok) { qlstm_destroy(q); return rc; }
     *out = q;
     return QLSTM_OK;
@@ -323,6 +330,7 @@ void qlstm_destroy(qlstm_t *q)
         fast_layer_destroy(L.fast);
     }
     fast_scratch_destroy(q->fscratch);
+    stack_small_destroy(q->stack);
     cudaFree(q->X); cudaFree(q->seq[0]); cudaFree(q->seq[1]);
     cudaFree(q->scratch.pre); cudaFree(q->scratch.po); cudaFree(q->scratch.stats); cudaFree(q->scratch.m);
     cudaFree(q->status);
@@ -360,6 +368,18 @@ int qlstm_run(qlstm_t *q, const int8_t *x_dev, int T, int B, int8_t *h_dev, int1
     if (cudaMemsetAsync(q->status, 0, 4 * sizeof(int), st) != cudaSuccess) return QLSTM_ERR_CUDA;
 
     const int nl = (int)q->layers.size();
+    // small batches: the whole stack in one launch (layers as a wavefront, input projection inside the step)
+    if (!trace && (q->impl_rec == 0 || q->impl_rec == 5) && q->impl_proj != 1) {
+        if (stack_small_supported(q->stack, T, B)) {
+            SpanGuard g(q, st, 1);
+            int rc = launch_stack_small(q->stack, x_dev, T, B, h_dev, c_dev, y_dev, q->status, st);
+            g.done(1);
+            return rc;
+        }
+        if (q->impl_rec == 5) return QLSTM_ERR_DIM;
+    } else if (q->impl_rec == 5) {
+        return QLSTM_ERR_ARG;
+    }
     const int8_t *in = x_dev;
     size_t h_off = 0, c_off = 0;
     for (int l = 0; l < nl; ++l) {
@@ -457,7 +477,7 @@ int qlstm_last_status(qlstm_t *q)
 
 int qlstm_set_impl(qlstm_t *q, int projection_impl, int recurrent_impl)
 {
-    if (!q || projection_impl < 0 || projection_impl > 2 || recurrent_impl < 0 || recurrent_impl > 4) return QLSTM_ERR_ARG;
+    if (!q || projection_impl < 0 || projection_impl > 2 || recurrent_impl < 0 || recurrent_impl > 5) return QLSTM_ERR_ARG;
     q->impl_proj = projection_impl;
     q->impl_rec = recurrent_impl;
     return QLSTM_OK;
@@ -471,6 +491,7 @@ int qlstm_debug_barrier_timeout(qlstm_t *q, int missing_arrivals, unsigned long 
         L.fast.dbg_barrier_extra = (unsigned)missing_arrivals;
         L.fast.dbg_spin_limit_ns = missing_arrivals > 0 ? limit_ns : 0;
     }
+    stack_small_debug_timeout(q->stack, (unsigned)missing_arrivals, limit_ns);
     return QLSTM_OK;
 }
 

@@ -1,21 +1,28 @@
 // Persistent recurrent kernel: all T steps of one LSTM layer in one cooperative launch.
 //
-// Per step, three phases separated by grid-wide barriers (each phase partitions the work its own way):
+// A block owns a range of cells for the whole sequence: its rows of R stay in shared memory.  Per step:
 //
-//   A  recurrent matmul   partitioned by gate rows.  CTA i keeps the rows of R for cells
-//                         [i*cpc, (i+1)*cpc) resident in shared memory for the whole sequence, streams
-//                         h^{t-1} (int8 [B][O]) through a TMA ring and runs tcgen05.mma kind::i8 with the
-//                         batch as M and its gate rows as N.  Epilogue: + folded bias (saturating),
-//                         rescale to the gate format, + the input projection X_t -> gate sums to L2.
-//   B  elementwise        partitioned by (batch row, cell chunk).  Integer layer norm (statistics over the
-//                         whole row), integer sigmoid / tanh, CIFG coupling, peephole terms, int16 cell
-//                         update, hidden state requantised to int8.
+//   A  recurrent matmul   the block streams h^{t-1} (int8 [B][O]) through a TMA ring and runs tcgen05.mma kind::i8
+//                         with the batch as M and its gate rows as N (dp4a mat-vecs at small batch).  Epilogue: + folded
+//                         bias (saturating), rescale to the gate format, + the input projection X_t (+ the peephole
+//                         terms on c^{t-1}) -> gate sums.
+//   B  elementwise        integer layer norm, integer sigmoid / tanh, CIFG coupling, cell update, output-gate peephole
+//                         on c^t, hidden state requantised to int8.
+//        without layer norm: same block, same cells, straight after the epilogue - the gate sums never leave shared
+//                         memory and there is no barrier between A and B.
+//        with layer norm:  the statistics need every cell of a row (Section 3.2.6), so the gate sums go to L2 (one
+//                         tensor-map store per block), a grid barrier follows, and phase B is partitioned as a flat
+//                         range of the B x C cell grid (whole rows when layer norm and peephole combine: the output
+//                         gate's statistics need c^t of the whole row).  (Keeping the cells with their block and adding
+//                         per-row partial sums with atomics to totals in L2 was measured: 148 blocks adding to the same
+//                         addresses cost more than the round trip they save - 49.5 against 37.4 us per step.)
+//      -- grid barrier: the projection (or the next step's matmul) needs every m --
 //   C  projection         partitioned by (batch tile, output slice); W_proj slice resident in shared memory,
 //                         m^t streamed through the same TMA ring; epilogue requantises to int8 h^t.
+//      -- grid barrier --
 //
-// Layer norm needs every cell of a row before any activation, and the projection needs every m before any
-// h, so these barriers are inherent to the method (Section 3.2.6, 3.2.8); only the data that crosses
-// CTAs (gate sums, m, h) goes through L2, the weights never move after the prologue.
+// Only the data that crosses blocks (h, m, and with layer norm the gate sums) goes through L2; the weights never move
+// after the prologue.
 //
 // Every wait is bounded.  A wait that runs out sets the abort word; all CTAs observe it at the next
 // barrier, leave the time loop together, free their tensor memory and return; the host reports
@@ -34,7 +41,7 @@ namespace {
 
 constexpr int RTHREADS = 640;                 // warp 0 TMA producer, warp 1 MMA issuer, warps 2..9 matmul epilogues;
                                               // all 20 warps share the elementwise phase
-constexpr int MAX_LN_ROWS = 4;                // rows whose layer-norm statistics are held at once
+constexpr int MAX_LN_ROWS = 4;                // flat elementwise phase: rows whose layer-norm statistics are held at once
 constexpr int KB_BYTES = 128 * 128;           // one k-block of the A operand: 128 rows x 128 bytes
 constexpr int STAGE_KB = 2;                   // k-blocks per ring stage: one bulk copy brings up to 32 KB
 constexpr int STAGE_BYTES = STAGE_KB * KB_BYTES;
@@ -61,10 +68,14 @@ struct RecParams {
     int kb_h, kb_c, stages;
     int n_issue_c;                // projection: MMA issuers (= partial accumulators) sharing the K range
     RingPlan plan_a, plan_c;      // ring use of the recurrent matmul and of the projection
-    int items_per_cta;            // cells of the B x C grid per CTA in the elementwise phase
+    int items_per_cta;            // layer norm: cells of the B x C grid per CTA in the flat elementwise phase
     int small;                    // small batch: dp4a mat-vec with warp reductions instead of TMA + tcgen05
     int npc;                      // gate rows per CTA = columns of its X box
-    uint32_t x_bytes;             // bytes of one X box: MT * 128 rows x npc int16
+    int x_rows;                   // rows of the X box: MT * 128 (B at small batch)
+    uint32_t x_bytes;             // bytes of one X box: x_rows x npc int16
+    uint32_t ho_bytes;            // peephole: bytes of the output gate's recurrent terms, x_rows x cpc int16
+    uint32_t acc_off;             // byte offset in the ring (idle between the matmul phases) of the small-batch accumulators
+    uint32_t row_bytes;           // layer norm + peephole: bytes of the row buffer of the elementwise phase
     int rpc;                      // small batch: projection rows per CTA
     const int8_t *R, *Wproj;      // packed weights (small-batch prologue copies its slices with plain loads)
     int fast_rescale_ok;          // every rescale of this layer has shift <= 0
@@ -72,7 +83,8 @@ struct RecParams {
     int16_t *c;                   // [B][C]
     int8_t *y;                    // [T][B][O]
     int8_t *hbuf, *mbuf;
-    int32_t *pre;
+    int32_t *pre;                 // layer norm: gate sums [B][N] between the matmul and elementwise phases (int16 values,
+                                  // or int32 X + H when a peephole term is still to be added)
     unsigned *bar;
     int *status;
     const int32_t *bh, *bp, *bln;
@@ -189,54 +201,122 @@ __device__ __forceinline__ size_t operand_off(const RecParams &p, int row, int k
     return p.small ? (size_t)row * K + k : tile_off(row, k, nkb);
 }
 
-// Phase A epilogue for one thread = one batch row and a range of 8-column groups of this CTA's gate sums.
-//   out = sat16( X + sat16(rescale(sat32(acc + bh), eff_h)) )            (no peephole: final gate sum, int16)
-//   out = X + sat16(rescale(...))                                        (peephole: int32, finished in phase B)
-// X_t of the CTA's gate rows is in shared memory, [batch row][npc] int16.  Without peephole the result replaces X
-// in place and leaves through a tensor-map store; the int32 form of the peephole variant is stored directly.
-template <int G>
-__device__ __forceinline__ void phase_a_row(const RecParams &p, uint32_t taddr, int b, int n0, int g_begin, int g_end,
-                                            const int32_t *bh_s, int16_t *x_s, bool row_valid)
+// Views of what a block keeps in shared memory for its own cells (columns n = cell * G + slot of its gate rows).
+struct OwnCells {
+    int16_t *x_s;          // [x_rows][npc]   X_t, replaced in place by the gate sums
+    int16_t *ho_s;         // [x_rows][cpc]   peephole only: the output gate's recurrent term H_o (its X stays in x_s)
+    const int32_t *bh_s;   // [nc_pad]        folded bias of the recurrent accumulator
+    const int16_t *P_s;    // [nc_pad]        peephole weights (0 where a gate has none)
+    int u0;                // first cell
+    int cells;             // cells owned (even; fewer than cpc in the last block)
+};
+
+// Matmul epilogue for one batch row b and the 8-column groups [g_begin, g_end) of this block's gate sums
+// (Section 3.2.4 / 3.2.5).  Per column:
+//   H   = sat16(rescale(sat32(acc + bh), eff_h))
+//   out = sat16(X + H [+ sat16(rescale(P c^{t-1}, eff_c)) for the input and forget gates])
+// X_t is in shared memory and is replaced in place.  Without layer norm a peephole layer finishes the input and forget
+// gates here; the output gate waits for c^t: its X stays where it is and H goes to ho_s.  With layer norm and peephole
+// (LN && PEEP) nothing can be finished yet: X + H goes to global memory as int32 and the elementwise phase adds the
+// peephole terms row by row.
+// TM: accumulators come from tensor memory (taddr; warp-collective loads, so every lane runs the loop) or from
+// acc_row (int32, shared memory).  With three gates the groups are taken three at a time (24 columns = 8 cells), so
+// that the slot of every column is a compile-time constant; g_begin is then a multiple of 3.
+template <int G, bool LN, bool PEEP, bool TM>
+__device__ __forceinline__ void gate_sums_row(const RecParams &p, const OwnCells &oc, uint32_t taddr, const int32_t *acc_row,
+                                              int b, int n0, int g_begin, int g_end, const int16_t *c_row, bool row_valid)
 {
-    constexpr int NB = 2;                                    // groups per batch of tensor-memory loads
-    const bool peep = (p.flags & F_PEEPHOLE) != 0;
-    int16_t *xrow = x_s + (size_t)b * p.npc;
+    constexpr int NB = (G == 4) ? 2 : 3;                     // groups per trip of the loop
+    constexpr int NL = (G == 4) ? 2 : 1;                     // groups whose accumulators are loaded at once
+    constexpr int SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
+    int16_t *xrow = oc.x_s + (size_t)b * p.npc;
 #pragma unroll 1
     for (int gbase = g_begin; gbase < g_end; gbase += NB) {
-        uint32_t r[NB][8];
-        __syncwarp();                                        // the TMEM loads are warp-collective
+        uint32_t r[NL][8];
+        auto load_acc = [&](int first) {                     // accumulators of the groups first .. first + NL - 1 of this trip
+            if (TM) {
+                __syncwarp();                                // the TMEM loads are warp-collective
 #pragma unroll
-        for (int i = 0; i < NB; ++i)
-            if (gbase + i < g_end) ptx::tmem_ld_32x8(taddr + (uint32_t)((gbase + i) * 8), r[i]);   // warp-uniform
-        ptx::tmem_ld_wait();
-        if (!row_valid) continue;
+                for (int i = 0; i < NL; ++i)
+                    if (gbase + first + i < g_end) ptx::tmem_ld_32x8(taddr + (uint32_t)((gbase + first + i) * 8), r[i]);   // warp-uniform
+                ptx::tmem_ld_wait();
+            } else {
+#pragma unroll
+                for (int i = 0; i < NL; ++i)
+                    if (gbase + first + i < g_end) {
+                        const int4 a0 = *reinterpret_cast<const int4 *>(acc_row + (gbase + first + i) * 8);
+                        const int4 a1 = *reinterpret_cast<const int4 *>(acc_row + (gbase + first + i) * 8 + 4);
+                        r[i][0] = a0.x; r[i][1] = a0.y; r[i][2] = a0.z; r[i][3] = a0.w;
+                        r[i][4] = a1.x; r[i][5] = a1.y; r[i][6] = a1.z; r[i][7] = a1.w;
+                    }
+            }
+        };
+        if (NL == NB) {
+            load_acc(0);
+            if (TM && !row_valid) continue;
+        }
+        // c^{t-1} of the cells these columns belong to (peephole): 4 cells with four gates, 8 with three
+        const int cell0 = (gbase * 8) / G;
+        int32_t c_old[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        if (PEEP && !LN) {
+            constexpr int NC = (G == 4) ? 4 : 8;
+#pragma unroll
+            for (int k = 0; k < NC; k += 2) {
+                if (row_valid && cell0 + k < oc.cells) {
+                    const uint32_t w = *reinterpret_cast<const uint32_t *>(c_row + cell0 + k);
+                    c_old[k] = lo16(w); c_old[k + 1] = hi16(w);
+                }
+            }
+        }
 #pragma unroll
         for (int i = 0; i < NB; ++i) {
             const int grp = gbase + i;
             if (grp >= g_end) break;
+            if (NL != NB) {
+                load_acc(i);
+                if (TM && !row_valid) continue;
+            }
             const int c8 = grp * 8;
             const uint4 x4 = *reinterpret_cast<const uint4 *>(xrow + c8);
             const uint32_t xw[4] = {x4.x, x4.y, x4.z, x4.w};
-            const int4 b0 = *reinterpret_cast<const int4 *>(bh_s + c8), b1 = *reinterpret_cast<const int4 *>(bh_s + c8 + 4);
+            const int4 b0 = *reinterpret_cast<const int4 *>(oc.bh_s + c8), b1 = *reinterpret_cast<const int4 *>(oc.bh_s + c8 + 4);
             const int32_t bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-            const int ph = (G == 4) ? 0 : c8 % 3;
+            uint32_t pw[4] = {0, 0, 0, 0};
+            if (PEEP && !LN) {
+                const uint4 p4 = *reinterpret_cast<const uint4 *>(oc.P_s + c8);
+                pw[0] = p4.x; pw[1] = p4.y; pw[2] = p4.z; pw[3] = p4.w;
+            }
             int32_t o[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
-                const int gi = (G == 4) ? (j & 3) : (ph + j) % 3;
-                const int32_t acc = add_sat((int32_t)r[i][j], bb[j]);
+                const int col = i * 8 + j;                           // column inside this batch of groups
+                const int gi = (G == 4) ? (j & 3) : col % 3;         // compile-time: gbase * 8 is a multiple of G
+                const int cl = col / G;                              // cell inside this batch of groups
+                const int32_t acc = add_sat((int32_t)r[NL == NB ? i : 0][j], bb[j]);
                 const int32_t H = sat16(rescale_sel(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
                 const int32_t X = (j & 1) ? hi16(xw[j >> 1]) : lo16(xw[j >> 1]);
-                o[j] = X + H;                                        // saturated to int16 when packed (no peephole)
+                if (LN) {
+                    o[j] = X + H;                                    // saturated when packed (no peephole), or int32 as it is
+                } else if (PEEP && gi == SO) {
+                    o[j] = X;                                        // finished in phase B, once c^t exists
+                    oc.ho_s[(size_t)b * p.cpc + cell0 + cl] = (int16_t)H;
+                } else {
+                    int32_t v = X + H;
+                    if (PEEP && gi != SZ) {
+                        const int32_t P = (j & 1) ? hi16(pw[j >> 1]) : lo16(pw[j >> 1]);
+                        v += sat16(rescale_any(P * c_old[cl], p.eff_c[gi], p.f_c[gi]));
+                    }
+                    o[j] = v;                                        // saturated when packed
+                }
             }
-            if (peep) {
+            if (LN && PEEP) {
                 int32_t *dst = p.pre + (size_t)b * p.N + n0 + c8;
                 *reinterpret_cast<int4 *>(dst) = make_int4(o[0], o[1], o[2], o[3]);
                 *reinterpret_cast<int4 *>(dst + 4) = make_int4(o[4], o[5], o[6], o[7]);
-            } else {
-                *reinterpret_cast<uint4 *>(xrow + c8) = make_uint4(ptx::pack_sat_s16(o[0], o[1]), ptx::pack_sat_s16(o[2], o[3]),
-                                                                   ptx::pack_sat_s16(o[4], o[5]), ptx::pack_sat_s16(o[6], o[7]));
+                continue;
             }
+            *reinterpret_cast<uint4 *>(xrow + c8) = make_uint4(ptx::pack_sat_s16(o[0], o[1]), ptx::pack_sat_s16(o[2], o[3]),
+                                                               ptx::pack_sat_s16(o[4], o[5]), ptx::pack_sat_s16(o[6], o[7]));
         }
     }
 }
@@ -273,7 +353,94 @@ __device__ __forceinline__ void phase_c_row(const RecParams &p, uint32_t taddr, 
 }
 
 // ------------------------------------------------------------------------------------------------
-// Phase B: elementwise work on a contiguous range of the B x C cell grid.
+// Phase B without layer norm: everything after the gate sums, for the block's own cells, two adjacent cells per task.
+
+// G int16 values of two adjacent cells (cell index even): v[k][gi].  SRC: 0 shared memory (or data only this block
+// writes), 1 read-only global data, 2 global data written by other blocks this step (L2 loads)
+template <int G, int SRC>
+__device__ __forceinline__ void load_pair_i16(const int16_t *ptr, int32_t (&v)[2][4])
+{
+    if (G == 4) {
+        const uint4 *q4 = reinterpret_cast<const uint4 *>(ptr);
+        const uint4 q = SRC == 0 ? *q4 : (SRC == 1 ? __ldg(q4) : __ldcg(q4));
+        v[0][0] = lo16(q.x); v[0][1] = hi16(q.x); v[0][2] = lo16(q.y); v[0][3] = hi16(q.y);
+        v[1][0] = lo16(q.z); v[1][1] = hi16(q.z); v[1][2] = lo16(q.w); v[1][3] = hi16(q.w);
+    } else {
+        const uint32_t *w = reinterpret_cast<const uint32_t *>(ptr);
+        uint32_t a, b, c;
+        if (SRC == 0) { a = w[0]; b = w[1]; c = w[2]; }
+        else if (SRC == 1) { a = __ldg(w); b = __ldg(w + 1); c = __ldg(w + 2); }
+        else { a = __ldcg(w); b = __ldcg(w + 1); c = __ldcg(w + 2); }
+        v[0][0] = lo16(a); v[0][1] = hi16(a); v[0][2] = lo16(b);
+        v[1][0] = hi16(b); v[1][1] = lo16(c); v[1][2] = hi16(c);
+        v[0][3] = 0; v[1][3] = 0;
+    }
+}
+template <int G>
+__device__ __forceinline__ void load_pair_i32(const int32_t *ptr, int32_t (&v)[2][4])      // read-only global data
+{
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+#pragma unroll
+        for (int g = 0; g < 4; ++g) v[k][g] = g < G ? __ldg(ptr + k * G + g) : 0;
+}
+
+__device__ __forceinline__ void store_hidden_pair(const RecParams &p, int b, int u, int t, int32_t m0, int32_t m1, int8_t *h_next)
+{
+    const uint16_t v = (uint16_t)((m0 & 0xff) | ((m1 & 0xff) << 8));
+    if (p.flags & F_PROJECTION) {
+        *reinterpret_cast<uint16_t *>(p.mbuf + operand_off(p, b, u, p.C, p.kb_c)) = v;
+    } else {
+        *reinterpret_cast<uint16_t *>(h_next + operand_off(p, b, u, p.O, p.kb_h)) = v;
+        *reinterpret_cast<uint16_t *>(p.y + ((size_t)t * p.B + b) * p.O + u) = v;
+    }
+}
+
+// One pair of the block's own cells (local pair k of row b), gate sums in shared memory.
+template <int G, bool PEEP>
+__device__ __forceinline__ void own_cell_pair(const RecParams &p, const OwnCells &oc, int b, int k, int t, int8_t *h_next)
+{
+    constexpr int SI = 0, SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
+    const int ul = 2 * k, nl = ul * G;                     // local cell and column
+    const int u = oc.u0 + ul;
+    int16_t *c_ptr = p.c + (size_t)b * p.C + u;
+    int32_t a[2][4];
+    load_pair_i16<G, 0>(oc.x_s + (size_t)b * p.npc + nl, a);
+    const uint32_t cw = *reinterpret_cast<const uint32_t *>(c_ptr);
+    const int32_t c_old[2] = {lo16(cw), hi16(cw)};
+    int32_t c_new[2], m[2];
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        const int32_t f = sigmoid_q_fast(a[q][SF], 3), z = tanh_q_fast(a[q][SZ], 3);
+        int32_t i;
+        if (G == 4) i = sigmoid_q_fast(a[q][SI], 3);
+        else { i = 32768 - f; if (i > 32767) i = 32767; }          // coupled input gate, Section 3.2.9
+        c_new[q] = cell_update_fast(i, z, f, c_old[q], p.m_bits);
+        int32_t ao = a[q][SO];
+        if (PEEP) {
+            const int32_t H = oc.ho_s[(size_t)b * p.cpc + ul + q], P = oc.P_s[nl + q * G + SO];
+            ao = sat16(ao + H + sat16(rescale_any(P * c_new[q], p.eff_c[SO], p.f_c[SO])));   // Eq. 5: o sees c^t
+        }
+        m[q] = hidden_q_fast(sigmoid_q_fast(ao, 3), c_new[q], p.m_bits, p.eff_m, p.f_m, p.zp_m);
+    }
+    *reinterpret_cast<uint32_t *>(c_ptr) = pack16(c_new[0], c_new[1]);
+    store_hidden_pair(p, b, u, t, m[0], m[1], h_next);
+}
+
+// All (row, cell pair) tasks of the block, consecutive threads on consecutive pairs of a row: the gate sums of a row's
+// pairs are contiguous in shared memory.
+template <int G, bool PEEP>
+__device__ __forceinline__ void phase_b_own(const RecParams &p, const OwnCells &oc, int t, int8_t *h_next)
+{
+    const int pairs = oc.cells >> 1, total = p.B * pairs;
+    for (int i = threadIdx.x; i < total; i += RTHREADS) {
+        const int b = i / pairs, k = i - b * pairs;
+        own_cell_pair<G, PEEP>(p, oc, b, k, t, h_next);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Phase B with layer norm: elementwise work on a contiguous range of the B x C cell grid, gate sums from L2.
 
 // Warp-level part of the statistics reduction: per-gate sum / sum of squares of this warp into shared memory.
 template <int G>
@@ -306,45 +473,18 @@ __device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, const long long 
     ptx::cta_sync();
 }
 
-// G int16 values of two adjacent cells (cell index even): v[k][gi]
 template <int G>
-__device__ __forceinline__ void load_pair_i16(const int16_t *ptr, bool readonly, int32_t (&v)[2][4])
-{
-    if (G == 4) {
-        const uint4 q = readonly ? __ldg(reinterpret_cast<const uint4 *>(ptr)) : __ldcg(reinterpret_cast<const uint4 *>(ptr));
-        v[0][0] = lo16(q.x); v[0][1] = hi16(q.x); v[0][2] = lo16(q.y); v[0][3] = hi16(q.y);
-        v[1][0] = lo16(q.z); v[1][1] = hi16(q.z); v[1][2] = lo16(q.w); v[1][3] = hi16(q.w);
-    } else {
-        const uint32_t *w = reinterpret_cast<const uint32_t *>(ptr);
-        const uint32_t a = readonly ? __ldg(w) : __ldcg(w), b = readonly ? __ldg(w + 1) : __ldcg(w + 1), c = readonly ? __ldg(w + 2) : __ldcg(w + 2);
-        v[0][0] = lo16(a); v[0][1] = hi16(a); v[0][2] = lo16(b);
-        v[1][0] = hi16(b); v[1][1] = lo16(c); v[1][2] = hi16(c);
-        v[0][3] = 0; v[1][3] = 0;
-    }
-}
-template <int G>
-__device__ __forceinline__ void load_pair_i32(const int32_t *ptr, bool readonly, int32_t (&v)[2][4])
+__device__ __forceinline__ void load_pair_i32_cg(const int32_t *ptr, int32_t (&v)[2][4])   // written by other blocks this step
 {
 #pragma unroll
     for (int k = 0; k < 2; ++k)
 #pragma unroll
-        for (int g = 0; g < 4; ++g) v[k][g] = g < G ? (readonly ? __ldg(ptr + k * G + g) : __ldcg(ptr + k * G + g)) : 0;
+        for (int g = 0; g < 4; ++g) v[k][g] = g < G ? __ldcg(ptr + k * G + g) : 0;
 }
 
-__device__ __forceinline__ void store_hidden_pair(const RecParams &p, int b, int u, int t, int32_t m0, int32_t m1, int8_t *h_next)
-{
-    const uint16_t v = (uint16_t)((m0 & 0xff) | ((m1 & 0xff) << 8));
-    if (p.flags & F_PROJECTION) {
-        *reinterpret_cast<uint16_t *>(p.mbuf + operand_off(p, b, u, p.C, p.kb_c)) = v;
-    } else {
-        *reinterpret_cast<uint16_t *>(h_next + operand_off(p, b, u, p.O, p.kb_h)) = v;
-        *reinterpret_cast<uint16_t *>(p.y + ((size_t)t * p.B + b) * p.O + u) = v;
-    }
-}
-
-// Two adjacent cells (u even) of row b, every step after the gate sums (not used for layer norm + peephole).
+// Two adjacent cells (u even) of row b, every step after the gate sums (layer norm without peephole).
 template <int G, bool LN, bool PEEP>
-__device__ __forceinline__ void cell_pair(const RecParams &p, const LnRow *lr, int b, int u, int t, int8_t *h_next)
+__device__ __forceinline__ void flat_cell_pair(const RecParams &p, const LnRow *lr, int b, int u, int t, int8_t *h_next)
 {
     constexpr int SI = 0, SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
     const size_t nb = (size_t)b * p.N + (size_t)u * G;
@@ -354,8 +494,8 @@ __device__ __forceinline__ void cell_pair(const RecParams &p, const LnRow *lr, i
     const int32_t c_old[2] = {lo16(cw), hi16(cw)};
     int32_t a[2][4], P[2][4];
     if (PEEP) {
-        load_pair_i32<G>(p.pre + nb, false, a);
-        load_pair_i16<G>(p.P + nu, true, P);
+        load_pair_i32_cg<G>(p.pre + nb, a);
+        load_pair_i16<G, 1>(p.P + nu, P);
 #pragma unroll
         for (int k = 0; k < 2; ++k)
 #pragma unroll
@@ -366,11 +506,11 @@ __device__ __forceinline__ void cell_pair(const RecParams &p, const LnRow *lr, i
                 a[k][g] = sat16(v);
             }
     } else {
-        load_pair_i16<G>((const int16_t *)p.pre + nb, false, a);
+        load_pair_i16<G, 2>((const int16_t *)p.pre + nb, a);
         if (LN) {
             int32_t L[2][4], bl[2][4];
-            load_pair_i16<G>(p.L + nu, true, L);
-            load_pair_i32<G>(p.bln + nu, true, bl);
+            load_pair_i16<G, 1>(p.L + nu, L);
+            load_pair_i32<G>(p.bln + nu, bl);
 #pragma unroll
             for (int k = 0; k < 2; ++k)
 #pragma unroll
@@ -423,7 +563,7 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, in
                     for (int k = 0; k < 4; ++k) {
                         const int u = u0 + 2 * gs * k;
                         if (u < p.C) {
-                            load_pair_i16<G>(row + (size_t)u * G, false, v[k]);
+                            load_pair_i16<G, 2>(row + (size_t)u * G, v[k]);
                         } else {
 #pragma unroll
                             for (int g = 0; g < 4; ++g) { v[k][0][g] = 0; v[k][1][g] = 0; }
@@ -452,7 +592,7 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, in
         const int j1 = i1 < (re + 1) * p.C ? i1 : (re + 1) * p.C;
         for (int i = j0 + 2 * threadIdx.x; i < j1; i += 2 * RTHREADS) {
             const int b = i / p.C, u = i - b * p.C;
-            cell_pair<G, LN, PEEP>(p, ctl->ln_rows[b - rb], b, u, t, h_next);
+            flat_cell_pair<G, LN, PEEP>(p, ctl->ln_rows[b - rb], b, u, t, h_next);
         }
         if (LN) ptx::cta_sync();      // the statistics slots are reused by the next batch of rows
     }
@@ -525,22 +665,6 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
     }
 }
 
-__device__ __forceinline__ void phase_b(const RecParams &p, RecCtl *ctl, int t, int8_t *h_next, int16_t *row_s)
-{
-    const bool ln = (p.flags & F_LAYERNORM) != 0, peep = (p.flags & F_PEEPHOLE) != 0;
-    if (p.G == 4) {
-        if (ln && peep) phase_b_ln_peep<4>(p, ctl, t, h_next, row_s);
-        else if (ln) phase_b_flat<4, true, false>(p, ctl, t, h_next);
-        else if (peep) phase_b_flat<4, false, true>(p, ctl, t, h_next);
-        else phase_b_flat<4, false, false>(p, ctl, t, h_next);
-    } else {
-        if (ln && peep) phase_b_ln_peep<3>(p, ctl, t, h_next, row_s);
-        else if (ln) phase_b_flat<3, true, false>(p, ctl, t, h_next);
-        else if (peep) phase_b_flat<3, false, true>(p, ctl, t, h_next);
-        else phase_b_flat<3, false, false>(p, ctl, t, h_next);
-    }
-}
-
 // ------------------------------------------------------------------------------------------------
 // Small batch (default: B <= 4; measured crossover: from 8 rows on the tensor-core path is faster; selectable up to
 // SMALL_BATCH_MAX = 16 rows):
@@ -578,23 +702,16 @@ __device__ __forceinline__ int32_t warp_dots(const int8_t *w_row, const int8_t *
     return mine;                                   // lane b holds the dot product with batch row b
 }
 
+// recurrent accumulators of the block's gate rows into shared memory, acc_s [B][nc_pad] int32
 template <int BMAX>
-__device__ __forceinline__ void phase_a_small(const RecParams &p, int t, int cur, int n0, int n_cnt, const int8_t *R_s,
-                                              int8_t *stage_s, const int32_t *bh_s)
+__device__ __forceinline__ void phase_a_small(const RecParams &p, int cur, int n_cnt, const int8_t *R_s, int8_t *stage_s,
+                                              int32_t *acc_s)
 {
     stage_rows(stage_s, p.hbuf + (size_t)cur * p.h_stride, p.B * p.O);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const bool peep = (p.flags & F_PEEPHOLE) != 0;
     for (int n = warp; n < n_cnt; n += RTHREADS / 32) {
         const int32_t mine = warp_dots<BMAX>(R_s + (size_t)n * p.O, stage_s, p.O, lane);
-        if (lane < p.B) {
-            const int b = lane, gi = n % p.G;
-            const int32_t acc = add_sat(mine, bh_s[n]);
-            const int32_t H = sat16(rescale_sel(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
-            const int32_t X = __ldg(p.X + ((size_t)t * p.B + b) * p.N + n0 + n);
-            if (peep) p.pre[(size_t)b * p.N + n0 + n] = X + H;
-            else ((int16_t *)p.pre)[(size_t)b * p.N + n0 + n] = (int16_t)sat16(X + H);
-        }
+        if (lane < p.B) acc_s[lane * p.nc_pad + n] = mine;
     }
 }
 
@@ -702,6 +819,9 @@ __device__ __forceinline__ void ring_advance(const Ring &r, const RingPlan &pl)
     for (int s = 0; s < MAX_STAGES; ++s) r.rounds[s] += (uint32_t)pl.uses[s];
 }
 
+// One instantiation per variant (gates, layer norm, peephole): each keeps only its own epilogue and elementwise code,
+// which is what lets the register allocator fit them without spilling.
+template <int G, bool LN, bool PEEP>
 __global__ void __launch_bounds__(RTHREADS, 1)
 k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_constant__ CUtensorMap map_Wp,
                   const __grid_constant__ CUtensorMap map_X, const __grid_constant__ CUtensorMap map_pre, RecParams p)
@@ -709,54 +829,67 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const bool proj = (p.flags & F_PROJECTION) != 0;
-    // layout: [ring stages][R slice][Wproj slice][X box][row buffer][bias slice][control]
+    constexpr bool ln = LN, peep = PEEP;
+    // layout: [ring stages][R slice][Wproj slice][X box][H_o (peephole) | row buffer (layer norm + peephole)]
+    //         [per-column constants][control]
     uint8_t *ring = smem;
     uint8_t *R_s = ring + (size_t)p.stages * STAGE_BYTES;
     // R slice: npc rows per k-block.  The MMA reads nc_pad (npc rounded up to 16) rows per k-block: the up to 8 extra
     // rows are the head of the next k-block (of the next region after the last one), and their columns are never read
     uint8_t *Wp_s = R_s + (size_t)p.kb_h * p.npc * 128;
     int16_t *x_s = (int16_t *)(Wp_s + (proj ? (size_t)p.kb_c * p.pn * 128 : 0));
-    uint8_t *after_w = (uint8_t *)x_s + (((size_t)p.x_bytes + 1023) & ~(size_t)1023);
-    int16_t *row_s = (int16_t *)after_w;
-    const size_t row_bytes = ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE)) ? ((size_t)p.C * p.G + p.C) * 2 : 0;
-    int32_t *bh_s = (int32_t *)(after_w + ((row_bytes + 15) & ~(size_t)15));
-    RecCtl *ctl = (RecCtl *)(bh_s + p.nc_pad);
+    uint8_t *after_x = (uint8_t *)x_s + (((size_t)p.x_bytes + 1023) & ~(size_t)1023);
+    int16_t *ho_s = (int16_t *)after_x;
+    int16_t *row_s = (int16_t *)after_x;
+    const size_t extra = (size_t)(ln ? p.row_bytes : p.ho_bytes);
+    int32_t *bh_s = (int32_t *)(after_x + ((extra + 15) & ~(size_t)15));
+    int16_t *P_s = (int16_t *)(bh_s + p.nc_pad);
+    RecCtl *ctl = (RecCtl *)(P_s + p.nc_pad);
+    // between the matmul phases the ring is idle: at small batch the staged operand and the accumulators live there
+    int8_t *stage_s = (int8_t *)ring;                                           // small batch: staged h / m, [B][K]
+    int32_t *acc_s = (int32_t *)(ring + p.acc_off);                             // small batch: [B][nc_pad]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
     volatile int *abort_flag = &ctl->abort_flag;
     const bool has_cells = cta < p.n_cta_a;
     const bool has_ptile = proj && cta < p.n_ptiles;
-    const int n0 = cta * p.cpc * p.G;
-    int n_cnt = p.cpc * p.G;
+    const int n0 = cta * p.cpc * G;
+    int n_cnt = p.cpc * G;
     if (n0 + n_cnt > p.N) n_cnt = p.N - n0;
+    if (!has_cells) n_cnt = 0;
     const int tile_mi = has_ptile ? cta / p.npn : 0, tile_p0 = has_ptile ? (cta % p.npn) * p.pn : 0;
     const uint32_t acc_cols_a = (uint32_t)(p.MT * p.nc_pad);
     uint32_t tmem_cols = 32;
     while (tmem_cols < acc_cols_a + (uint32_t)(proj ? p.pn * p.n_issue_c : 0)) tmem_cols <<= 1;
 
+    OwnCells oc;
+    oc.x_s = x_s; oc.ho_s = ho_s; oc.bh_s = bh_s; oc.P_s = P_s;
+    oc.u0 = cta * p.cpc;
+    oc.cells = n_cnt / G;
+
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) { ptx::mbar_init(&ctl->full[s], 1); ptx::mbar_init(&ctl->empty[s], 1); ctl->rounds[s] = 0; }
         for (int i = 0; i < 2; ++i) ptx::mbar_init(&ctl->acc_full[i], 1);
-        {
-            const int nc = (p.kb_c + STAGE_KB - 1) / STAGE_KB;
-            (void)nc;
-            ptx::mbar_init(&ctl->acc_full[2], (uint32_t)(p.plan_c.n_own > 0 ? p.plan_c.n_own : 1));      // one arrival per projection issuer
-        }
+        ptx::mbar_init(&ctl->acc_full[2], (uint32_t)(p.plan_c.n_own > 0 ? p.plan_c.n_own : 1));      // one arrival per projection issuer
         ptx::mbar_init(&ctl->w_full, 1);
         ptx::mbar_init(&ctl->x_full, 1);
         ctl->abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&map_R);
         ptx::prefetch_tensormap(&map_X);
-        ptx::prefetch_tensormap(&map_pre);
+        if (ln) ptx::prefetch_tensormap(&map_pre);
         if (proj) ptx::prefetch_tensormap(&map_Wp);
     }
     if (warp == 1) {
         ptx::tmem_alloc(&ctl->tmem_base, tmem_cols);
         ptx::tmem_relinquish();
     }
-    for (int i = threadIdx.x; i < p.nc_pad; i += RTHREADS) bh_s[i] = (has_cells && i < n_cnt) ? p.bh[n0 + i] : 0;
+    for (int i = threadIdx.x; i < p.nc_pad; i += RTHREADS) {
+        const bool in = i < n_cnt;
+        bh_s[i] = in ? p.bh[n0 + i] : 0;
+        P_s[i] = (in && peep && !ln) ? p.P[n0 + i] : (int16_t)0;
+    }
     ptx::tc_fence_before();
     ptx::cta_sync();
     ptx::tc_fence_after();
@@ -799,19 +932,19 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
     unsigned epoch = 0;
     Ring rg;
     rg.base = ring; rg.rounds = ctl->rounds;
-    const int cpt_a = (p.kb_h + STAGE_KB - 1) / STAGE_KB, n_chunks_a = p.MT * cpt_a;      // recurrent matmul: chunks per batch tile
-    const int n_chunks_c = (p.kb_c + STAGE_KB - 1) / STAGE_KB;
     const int n_issue_c = p.plan_c.n_own;
     const uint32_t idesc_a = ptx::idesc_i8(128, p.nc_pad), idesc_c = ptx::idesc_i8(128, p.pn);
     const int iss = warp == 1 ? 0 : warp == 18 ? 1 : warp == 19 ? 2 : warp == 17 ? 3 : -1;      // issuer thread number of lane 0
 
-    // the CTA's box of X_t: rows [t * B, t * B + MT * 128) x its gate rows (rows past the end of X read as zero)
+    // the CTA's box of X_t: rows [t * B, t * B + x_rows) x its gate rows (rows past the end of X read as zero)
     const bool tensor_a = !p.small && has_cells;
+    int x_last_t = -1;                                             // thread 0: step of the last box requested
     auto fetch_x = [&](int t) {
         ptx::mbar_arrive_expect_tx(&ctl->x_full, p.x_bytes);
         ptx::tma_load_2d(x_s, &map_X, &ctl->x_full, n0, t * p.B);
+        x_last_t = t;
     };
-    if (tensor_a && threadIdx.x == 0) fetch_x(0);
+    if (has_cells && threadIdx.x == 0) fetch_x(0);
 
     const bool timing = p.phase_ns != nullptr && cta == 0 && threadIdx.x == 0;
     unsigned long long t_mark = timing ? globaltimer() : 0ull;
@@ -822,20 +955,33 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
             t_mark = now;
         }
     };
+    const int ngroups = n_cnt >> 3;
+    constexpr int gstep = (G == 4) ? 1 : 3;                        // groups are dealt in units of this many
 
     for (int t = 0; t < p.T; ++t) {
         const int cur = t & 1;
         int8_t *h_next = p.hbuf + (size_t)(cur ^ 1) * p.h_stride;
         const uint32_t par = (uint32_t)t & 1u;
 
-        // ================= phase A: gate sums =================
+        // ================= phase A: gate sums of the block's cells =================
         if (p.small) {
             if (has_cells) {
-                if (p.B == 1) phase_a_small<1>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
-                else if (p.B <= 2) phase_a_small<2>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
-                else if (p.B <= 4) phase_a_small<4>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
-                else if (p.B <= 8) phase_a_small<8>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
-                else phase_a_small<16>(p, t, cur, n0, n_cnt, (const int8_t *)R_s, (int8_t *)ring, bh_s);
+                if (p.B == 1) phase_a_small<1>(p, cur, n_cnt, (const int8_t *)R_s, stage_s, acc_s);
+                else if (p.B <= 2) phase_a_small<2>(p, cur, n_cnt, (const int8_t *)R_s, stage_s, acc_s);
+                else if (p.B <= 4) phase_a_small<4>(p, cur, n_cnt, (const int8_t *)R_s, stage_s, acc_s);
+                else if (p.B <= 8) phase_a_small<8>(p, cur, n_cnt, (const int8_t *)R_s, stage_s, acc_s);
+                else phase_a_small<16>(p, cur, n_cnt, (const int8_t *)R_s, stage_s, acc_s);
+                ptx::cta_sync();
+                // epilogue tasks: (batch row, unit of column groups)
+                const bool okx = wait_or_abort(&ctl->x_full, par, abort_flag);
+                const int units = ngroups / gstep;
+                if (okx)
+                    for (int i = threadIdx.x; i < p.B * units; i += RTHREADS) {
+                        const int b = i / units, gu = i - b * units;
+                        gate_sums_row<G, LN, PEEP, false>(p, oc, 0u, acc_s + (size_t)b * p.nc_pad, b, n0, gu * gstep, (gu + 1) * gstep,
+                                                          p.c + (size_t)b * p.C + oc.u0, true);
+                    }
+                if (ln) ptx::fence_proxy_async();
             }
         } else if (has_cells) {
             if (warp == 0) {
@@ -859,8 +1005,8 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
                 // 16 epilogue warps: 4 TMEM lane quarters x (batch tile, column part)
                 const int e = warp - 2, quarter = warp & 3, slot = e >> 2;
                 const int mi = slot % p.MT, part = slot / p.MT, nparts = 4 / p.MT;
-                const int ngroups = n_cnt >> 3;
-                const int g_begin = part * ngroups / nparts, g_end = (part + 1) * ngroups / nparts;
+                const int units = ngroups / gstep;
+                const int g_begin = gstep * (part * units / nparts), g_end = gstep * ((part + 1) * units / nparts);
                 const int b = mi * 128 + quarter * 32 + lane;
                 const bool probe = p.phase_ns != nullptr && cta == 0 && warp == 2 && lane == 0;
                 const unsigned long long t_in = probe ? globaltimer() : 0ull;
@@ -870,34 +1016,43 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
                     if (probe) p.phase_ns[6] += globaltimer() - t_in;      // operand load + matmul latency
                     ptx::tc_fence_after();
                     const uint32_t ta = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * p.nc_pad);
-                    if (p.G == 4) phase_a_row<4>(p, ta, b, n0, g_begin, g_end, bh_s, x_s, b < p.B);
-                    else phase_a_row<3>(p, ta, b, n0, g_begin, g_end, bh_s, x_s, b < p.B);
+                    const bool valid = b < p.B;
+                    gate_sums_row<G, LN, PEEP, true>(p, oc, ta, nullptr, b, n0, g_begin, g_end,
+                                                     p.c + (size_t)(valid ? b : 0) * p.C + oc.u0, valid);
                     ptx::tc_fence_before();
-                    ptx::fence_proxy_async();                              // the box leaves through the async proxy
+                    if (ln) ptx::fence_proxy_async();                      // the box leaves through the async proxy
                 }
               }
             }
         }
         ptx::cta_sync();
         if (tensor_a && threadIdx.x == 0) ring_advance(rg, p.plan_a);
-        if (tensor_a && threadIdx.x == 0 && !*abort_flag) {
-            if (!(p.flags & F_PEEPHOLE)) {
-                // gate sums of all batch rows x this CTA's gate rows: one store, complete before the barrier publishes it
-                ptx::tma_store_2d(&map_pre, x_s, n0, 0);
-                ptx::bulk_commit_group();
-                ptx::bulk_wait_group_all();
-                fence_proxy_async_global();
+        if (ln) {
+            // the statistics of a row need every block's cells: gate sums to L2, barrier, flat elementwise phase
+            if (has_cells && threadIdx.x == 0 && !*abort_flag) {
+                if (!peep) {
+                    // gate sums of all batch rows x this block's gate rows: one store, complete before the barrier publishes it
+                    ptx::tma_store_2d(&map_pre, x_s, n0, 0);
+                    ptx::bulk_commit_group();
+                    ptx::bulk_wait_group_all();
+                    fence_proxy_async_global();
+                }
+                if (t + 1 < p.T) fetch_x(t + 1);              // the box is free again
             }
-            if (t + 1 < p.T) fetch_x(t + 1);                               // the box is free again
+            lap(0);
+            grid_sync(p, epoch, abort_flag, false);
+            lap(1);
+            if (*abort_flag) break;
+            if (peep) phase_b_ln_peep<G>(p, ctl, t, h_next, row_s);
+            else phase_b_flat<G, true, false>(p, ctl, t, h_next);
+            ptx::cta_sync();
+        } else {
+            // same block, same cells, straight from shared memory
+            phase_b_own<G, PEEP>(p, oc, t, h_next);
+            ptx::fence_proxy_async();                        // X box and ring scratch go back to the async proxy
+            ptx::cta_sync();
+            if (has_cells && threadIdx.x == 0 && t + 1 < p.T && !*abort_flag) fetch_x(t + 1);
         }
-        lap(0);
-        grid_sync(p, epoch, abort_flag, false);
-        lap(1);
-        if (*abort_flag) break;
-
-        // ================= phase B: elementwise =================
-        phase_b(p, ctl, t, h_next, row_s);
-        ptx::cta_sync();
         lap(2);
         grid_sync(p, epoch, abort_flag, !p.small);
         lap(3);
@@ -936,8 +1091,8 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
                     if (warp >= 2 && warp < 18) {
                         // 16 epilogue warps: 4 TMEM lane quarters x 4 column parts of the tile
                         const int quarter = warp & 3, part = (warp - 2) >> 2;
-                        const int ngroups = p.pn >> 2;
-                        const int c_begin = 4 * (part * ngroups / 4), c_end = 4 * ((part + 1) * ngroups / 4);
+                        const int ngroups_c = p.pn >> 2;
+                        const int c_begin = 4 * (part * ngroups_c / 4), c_end = 4 * ((part + 1) * ngroups_c / 4);
                         if (__all_sync(0xffffffffu, wait_or_abort(&ctl->acc_full[2], par, abort_flag))) {
                             ptx::tc_fence_after();
                             const int b = tile_mi * 128 + quarter * 32 + lane;
@@ -960,7 +1115,11 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
     // ---------------- teardown ----------------
     ptx::cta_sync();
     if (*abort_flag) {
-        for (int i = 0; i < 200; ++i) __nanosleep(500);      // let copies in flight land before the CTA retires
+        // copies still in flight must land before the block's shared memory is handed on: the X box by its barrier
+        // (bounded), ring stages by a bounded pause (their barriers may be mid-phase)
+        if (threadIdx.x == 0 && x_last_t >= 0)
+            for (int i = 0; i < 2000 && !ptx::mbar_try_wait_parked(&ctl->x_full, (uint32_t)x_last_t & 1u, 1000u); ++i) {}
+        for (int i = 0; i < 200; ++i) __nanosleep(500);
         if (threadIdx.x == 0) atomicExch(p.status, 2);
     }
     ptx::cta_sync();
@@ -993,14 +1152,28 @@ size_t x_box_bytes(int MT, int npc) { return (size_t)MT * 128 * npc * 2; }
 
 size_t rec_smem_bytes(const LayerParams &p, int stages, int nc_pad, int pn, int kb_h, int kb_c, int MT, int npc)
 {
-    const bool proj = (p.flags & F_PROJECTION) != 0;
-    size_t row_bytes = ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE)) ? ((size_t)p.C * p.G + p.C) * 2 : 0;
-    row_bytes = (row_bytes + 15) & ~(size_t)15;
+    const bool proj = (p.flags & F_PROJECTION) != 0, peep = (p.flags & F_PEEPHOLE) != 0, ln = (p.flags & F_LAYERNORM) != 0;
+    // without layer norm a peephole layer keeps H_o of the block's cells, all rows; with layer norm and peephole the
+    // elementwise phase holds one row of gate sums and of new cell states
+    size_t extra = ln ? (peep ? ((size_t)p.C * p.G + p.C) * 2 : 0) : (peep ? (size_t)MT * 128 * (npc / p.G) * 2 : 0);
+    extra = (extra + 15) & ~(size_t)15;
     return 1024 + (size_t)stages * STAGE_BYTES + (size_t)kb_h * npc * 128 + (proj ? (size_t)kb_c * pn * 128 : 0) +
-           ((x_box_bytes(MT, npc) + 1023) & ~(size_t)1023) + row_bytes + (size_t)nc_pad * 4 + sizeof(RecCtl) + 64;
+           ((x_box_bytes(MT, npc) + 1023) & ~(size_t)1023) + extra + (size_t)nc_pad * 6 + sizeof(RecCtl) + 64;
 }
 
 int round_up(int v, int m) { return (v + m - 1) / m * m; }
+
+// the instantiation for a layer's variant
+const void *recurrent_kernel(const LayerParams &p)
+{
+    const bool ln = (p.flags & F_LAYERNORM) != 0, peep = (p.flags & F_PEEPHOLE) != 0;
+    if (p.G == 4) {
+        if (ln) return peep ? (const void *)k_recurrent_sm100<4, true, true> : (const void *)k_recurrent_sm100<4, true, false>;
+        return peep ? (const void *)k_recurrent_sm100<4, false, true> : (const void *)k_recurrent_sm100<4, false, false>;
+    }
+    if (ln) return peep ? (const void *)k_recurrent_sm100<3, true, true> : (const void *)k_recurrent_sm100<3, true, false>;
+    return peep ? (const void *)k_recurrent_sm100<3, false, true> : (const void *)k_recurrent_sm100<3, false, false>;
+}
 
 // contig: n_own operand tiles of `per` chunks each, one owner per tile; else n_total chunks of one tile dealt round-robin
 RingPlan make_ring_plan(int stages, int n_own, bool contig, int per, int n_total)
@@ -1084,10 +1257,10 @@ int fast_recurrent_init(FastLayer &f, const LayerParams &p, const FastScratch &s
     } else {
         f.map_Wp = f.map_R;
     }
-    if (cudaFuncSetAttribute(k_recurrent_sm100, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(recurrent_kernel(p), cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
         return QLSTM_OK;
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_recurrent_sm100, RTHREADS, f.smem) != cudaSuccess || per_sm < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, recurrent_kernel(p), RTHREADS, f.smem) != cudaSuccess || per_sm < 1)
         return QLSTM_OK;
     f.rec_ok = true;
     return QLSTM_OK;
@@ -1128,20 +1301,27 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
         rp.plan_a = make_ring_plan(f.stages, rp.MT, true, cpt_a, 0);
         rp.plan_c = make_ring_plan(f.stages, ni, false, 0, n_chunks_c);
     }
-    rp.x_bytes = (uint32_t)x_box_bytes(rp.MT, rp.npc);
-    // elementwise phase: contiguous ranges of the B x C cell grid (whole rows with layer norm + peephole)
-    if ((p.flags & F_LAYERNORM) && (p.flags & F_PEEPHOLE))
-        rp.items_per_cta = ((B + f.grid - 1) / f.grid) * p.C;
-    else
-        rp.items_per_cta = round_up((int)(((long)B * p.C + f.grid - 1) / f.grid), 8);
     rp.R = p.R; rp.Wproj = p.Wproj;
     rp.rpc = (p.O + f.grid - 1) / f.grid;
     {
+        // small batch: staged operand [16][K], then the accumulators [16][nc_pad] int32, both inside the ring
         const int maxk = p.O > p.C ? p.O : p.C;
-        const bool fits = (size_t)SMALL_BATCH_MAX * maxk <= (size_t)f.stages * STAGE_BYTES && (!(p.flags & F_PROJECTION) || rp.rpc <= f.pn);
+        const size_t stage_bytes = ((size_t)SMALL_BATCH_MAX * maxk + 1023) & ~(size_t)1023;
+        const size_t need = stage_bytes + (size_t)SMALL_BATCH_MAX * f.nc_pad * 4;
+        const bool fits = need <= (size_t)f.stages * STAGE_BYTES && (!(p.flags & F_PROJECTION) || rp.rpc <= f.pn);
         const int lim = small_batch_max < SMALL_BATCH_MAX ? small_batch_max : SMALL_BATCH_MAX;
         rp.small = (B <= lim && fits) ? 1 : 0;
+        rp.acc_off = rp.small ? (uint32_t)stage_bytes : 0u;
     }
+    // the block's box of X_t and of the gate sums: all rows of the batch (whole 128-row tiles on the tensor-core path)
+    rp.x_rows = rp.small ? B : rp.MT * 128;
+    rp.x_bytes = (uint32_t)((size_t)rp.x_rows * rp.npc * 2);
+    const bool ln = (p.flags & F_LAYERNORM) != 0, peep = (p.flags & F_PEEPHOLE) != 0;
+    rp.ho_bytes = (peep && !ln) ? (uint32_t)((size_t)rp.x_rows * f.cpc * 2) : 0u;
+    rp.row_bytes = (peep && ln) ? (uint32_t)(((size_t)p.C * p.G + p.C) * 2) : 0u;
+    // layer norm: flat elementwise phase over contiguous ranges of the B x C cell grid (whole rows with a peephole)
+    if (ln && peep) rp.items_per_cta = ((B + f.grid - 1) / f.grid) * p.C;
+    else rp.items_per_cta = round_up((int)(((long)B * p.C + f.grid - 1) / f.grid), 8);
     rp.fast_rescale_ok = 1;
     for (int g = 0; g < p.G; ++g) {
         rp.eff_h[g] = p.eff_h[g]; rp.eff_c[g] = p.eff_c[g]; rp.eff_ln[g] = p.eff_ln[g];
@@ -1174,13 +1354,14 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
         ++n_launch;
     }
 
-    // X as a tensor [T * B][N] int16 and the gate sums as [B][N] int16; a CTA's box is all batch tiles x its gate rows
+    // X as a tensor [T * B][N] int16 and (layer norm) the gate sums as [B][N] int16; a block's box is all rows of a step
+    // x its gate rows
     CUtensorMap map_X, map_pre;
-    if (!make_tensor_map_i16(&map_X, X, (uint64_t)T * B, (uint64_t)p.N, (uint32_t)rp.MT * 128, (uint32_t)rp.npc) ||
-        !make_tensor_map_i16(&map_pre, s.pre, (uint64_t)B, (uint64_t)p.N, (uint32_t)rp.MT * 128, (uint32_t)rp.npc))
+    if (!make_tensor_map_i16(&map_X, X, (uint64_t)T * B, (uint64_t)p.N, (uint32_t)rp.x_rows, (uint32_t)rp.npc) ||
+        !make_tensor_map_i16(&map_pre, s.pre, (uint64_t)B, (uint64_t)p.N, (uint32_t)rp.x_rows, (uint32_t)rp.npc))
         return QLSTM_ERR_CUDA;
     void *args[] = {(void *)&f.map_R, (void *)&f.map_Wp, (void *)&map_X, (void *)&map_pre, (void *)&rp};
-    cudaError_t e = cudaLaunchCooperativeKernel((const void *)k_recurrent_sm100, dim3(f.grid), dim3(RTHREADS), args, f.smem, st);
+    cudaError_t e = cudaLaunchCooperativeKernel(recurrent_kernel(p), dim3(f.grid), dim3(RTHREADS), args, f.smem, st);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return e == cudaErrorCooperativeLaunchTooLarge ? QLSTM_ERR_LAUNCH : QLSTM_ERR_CUDA;

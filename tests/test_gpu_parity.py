@@ -11,6 +11,7 @@ from workloads import make_workload, random_layer_stack
 pytestmark = pytest.mark.gpu
 
 SIMPLE, FAST, AUTO = 1, 2, 0
+STACK = 5            # recurrent_impl: the whole-stack kernel for small batches, forced
 
 
 def oracle(w, trace=False, x=None, h0=None, c0=None):
@@ -100,6 +101,70 @@ def test_small_batch_both_matmul_paths(B, kw):
     check_equal(run_gpu(w, impl=(FAST, FAST)), want, f"default path B={B} {kw}")
     check_equal(run_gpu(w, impl=(FAST, 3)), want, f"tcgen05 B={B} {kw}")
     check_equal(run_gpu(w, impl=(FAST, 4)), want, f"dp4a B={B} {kw}")
+
+
+# ------------------------------------------------------------------ whole-stack kernel (batch <= 4)
+
+@pytest.mark.parametrize("B", [1, 2, 3, 4])
+@pytest.mark.parametrize("kw", VARIANTS, ids=lambda k: "+".join(sorted(k)) or "basic")
+def test_stack_kernel_parity_variants(B, kw):
+    """All layers and steps in one launch, layers as a wavefront: three layers so that the wavefront is deeper than
+    one hand-over, widths that leave ragged shares to the last block of a group."""
+    w = random_layer_stack(500 + B, 3, 48, 112, 64, T=7, B=B, **kw)
+    check_equal(run_gpu(w, impl=(AUTO, STACK)), oracle(w), f"stack kernel B={B} {kw}")
+
+
+@pytest.mark.parametrize("index,kw", [(1, {}), (2, dict(batch=4, T=30)), (3, dict(batch=2, T=12)), (4, dict(batch=3, T=12)),
+                                      (5, dict(batch=1, T=24)), (5, dict(batch=4, T=8))])
+def test_stack_kernel_parity_configs(index, kw):
+    w = make_workload(index, **kw)
+    check_equal(run_gpu(w, impl=(AUTO, STACK)), oracle(w), f"stack kernel config {index} {kw}")
+
+
+@pytest.mark.parametrize("index,kw", [(1, {}), (2, dict(batch=2, T=20)), (5, dict(batch=1, T=10))])
+def test_streaming_one_step_per_call(index, kw):
+    """One time step per call, the state carried by the caller (Section 3.2.2): y, h and c of every call against
+    the oracle's trace - bit for bit, and through the default kernel selection."""
+    import paper_2101_05453_b200 as qlstm
+    w = make_workload(index, **kw)
+    want = oracle(w, trace=True)
+    tr = want[3]
+    h, c = w.initial_state()
+    with qlstm.QLSTM(w.layers, 1, w.B) as hnd:
+        for t in range(w.T):
+            y, h, c, _ = run_gpu(w, handle=hnd, x=w.x[t:t + 1], h0=h, c0=c)
+            assert np.array_equal(y[0], want[0][t]), f"y differs at step {t}"
+            off_h = off_c = 0
+            for l, q in enumerate(w.layers):
+                assert np.array_equal(c[off_c:off_c + w.B * q.n_cell].reshape(w.B, q.n_cell), tr[l]["c"][t]), (l, t)
+                assert np.array_equal(h[off_h:off_h + w.B * q.n_output].reshape(w.B, q.n_output), tr[l]["h"][t]), (l, t)
+                off_h += w.B * q.n_output
+                off_c += w.B * q.n_cell
+    check_equal((want[0], h, c), want, "state after the last call")
+
+
+def test_stack_kernel_bounded_wait_reports_timeout():
+    """Every counter of the whole-stack kernel waits for an arrival nobody makes: the waits run into their 3 ms limit,
+    all blocks leave, the status is QLSTM_ERR_TIMEOUT and the next run on the handle is correct."""
+    import paper_2101_05453_b200 as qlstm
+    w = random_layer_stack(58, 2, 32, 64, 48, projection=True, layernorm=True, T=4, B=2)
+    want = oracle(w)
+    with qlstm.QLSTM(w.layers, w.T, w.B) as hnd:
+        hnd.debug_barrier_timeout(1, 3_000_000)
+        with pytest.raises(qlstm.QlstmError) as e:
+            run_gpu(w, handle=hnd, impl=(AUTO, STACK))
+        assert e.value.code == qlstm.ERR_TIMEOUT
+        hnd.debug_barrier_timeout(0)
+        check_equal(run_gpu(w, handle=hnd, impl=(AUTO, STACK)), want, "after timeout")
+
+
+def test_stack_kernel_refuses_what_it_cannot_run():
+    import paper_2101_05453_b200 as qlstm
+    w = random_layer_stack(59, 1, 32, 64, 64, T=3, B=6)
+    with qlstm.QLSTM(w.layers, w.T, w.B) as hnd:
+        with pytest.raises(qlstm.QlstmError) as e:
+            run_gpu(w, handle=hnd, impl=(AUTO, STACK))          # batch 6 > 4
+        assert e.value.code == qlstm.ERR_DIM
 
 
 def test_trace_parity_config3_slice():
