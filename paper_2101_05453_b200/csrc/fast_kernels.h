@@ -69,13 +69,15 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
 // uses[4] of the plan for `stages` ring stages and `n_own` issuers (see RingPlan in recurrent_sm100.cu).
 // ---- whole-stack kernel for small batches (stack_small_sm100.cu): all layers and steps in one cooperative launch,
 // one group of blocks per layer, layers running as a wavefront; also the path of one-step (streaming) calls.
-constexpr int STACK_SMALL_MAX_B = 4;
+constexpr int STACK_SMALL_MAX_B = 16;
 struct StackSmall;
 int stack_small_create(const std::vector<const LayerParams *> &layers, int max_T, int max_B, int sm_count, StackSmall **out);
 void stack_small_destroy(StackSmall *s);
 bool stack_small_supported(const StackSmall *s, int T, int B);
+bool stack_small_preferred(const StackSmall *s, int T, int B);     // supported and, by measurement, the faster path
+// schedule: 0 automatic, 1 wavefront (one group of blocks per layer), 2 sequential (every layer on all blocks)
 int launch_stack_small(const StackSmall *s, const int8_t *x, int T, int B, int8_t *h, int16_t *c, int8_t *y, int *status,
-                       cudaStream_t st);
+                       int schedule, cudaStream_t st);
 void stack_small_debug_timeout(StackSmall *s, unsigned missing_arrivals, unsigned long long limit_ns);
 int stack_small_groups(const StackSmall *s, int *blocks_per_layer);     // layers, and the blocks each layer's group has
 

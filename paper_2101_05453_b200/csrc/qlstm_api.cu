@@ -369,15 +369,16 @@ int qlstm_run(qlstm_t *q, const int8_t *x_dev, int T, int B, int8_t *h_dev, int1
 
     const int nl = (int)q->layers.size();
     // small batches: the whole stack in one launch (layers as a wavefront, input projection inside the step)
-    if (!trace && (q->impl_rec == 0 || q->impl_rec == 5) && q->impl_proj != 1) {
-        if (stack_small_supported(q->stack, T, B)) {
+    if (!trace && (q->impl_rec == 0 || q->impl_rec >= 5) && q->impl_proj != 1) {
+        if (q->impl_rec == 0 ? stack_small_preferred(q->stack, T, B) : stack_small_supported(q->stack, T, B)) {
             SpanGuard g(q, st, 1);
-            int rc = launch_stack_small(q->stack, x_dev, T, B, h_dev, c_dev, y_dev, q->status, st);
+            const int schedule = q->impl_rec == 6 ? 1 : (q->impl_rec == 7 ? 2 : 0);
+            int rc = launch_stack_small(q->stack, x_dev, T, B, h_dev, c_dev, y_dev, q->status, schedule, st);
             g.done(1);
             return rc;
         }
-        if (q->impl_rec == 5) return QLSTM_ERR_DIM;
-    } else if (q->impl_rec == 5) {
+        if (q->impl_rec >= 5) return QLSTM_ERR_DIM;
+    } else if (q->impl_rec >= 5) {
         return QLSTM_ERR_ARG;
     }
     const int8_t *in = x_dev;
@@ -477,7 +478,7 @@ int qlstm_last_status(qlstm_t *q)
 
 int qlstm_set_impl(qlstm_t *q, int projection_impl, int recurrent_impl)
 {
-    if (!q || projection_impl < 0 || projection_impl > 2 || recurrent_impl < 0 || recurrent_impl > 5) return QLSTM_ERR_ARG;
+    if (!q || projection_impl < 0 || projection_impl > 2 || recurrent_impl < 0 || recurrent_impl > 7) return QLSTM_ERR_ARG;
     q->impl_proj = projection_impl;
     q->impl_rec = recurrent_impl;
     return QLSTM_OK;

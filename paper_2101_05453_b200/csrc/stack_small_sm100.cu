@@ -21,6 +21,7 @@
 //
 // Every wait is bounded by a time limit; on expiry the waiting block sets the abort word, all blocks see it at their
 // next wait and leave, and the host reports QLSTM_ERR_TIMEOUT.
+#include <algorithm>
 #include <cstring>
 #include <vector>
 
@@ -31,7 +32,7 @@ namespace ql {
 
 namespace {
 
-constexpr int SK_THREADS = 640;
+constexpr int SK_THREADS = 512;              // 128 registers per thread: the mat-vec loops keep two rows of weight loads in flight
 constexpr int SK_WARPS = SK_THREADS / 32;
 constexpr unsigned long long SK_WAIT_LIMIT_NS = 2000000000ull;     // 2 s per wait
 
@@ -67,6 +68,8 @@ struct SkCall {
     int *status;
     unsigned long long wait_limit_ns;
     unsigned missing_arrivals;     // 0; a test makes every counter wait for arrivals that never come
+    int sequential;                // schedule: 0 wavefront (one group of blocks per layer), 1 every layer on all blocks
+    int max_I, max_O, max_C_proj, max_npc;   // widest layer: sizes of the shared-memory buffers
 };
 
 __device__ __forceinline__ unsigned sk_ld_acquire(const unsigned *p)
@@ -131,13 +134,70 @@ __device__ __forceinline__ bool sk_wait(const SkCall &k, const unsigned *cnt, un
 // rows [0, nrows) of a row-major int8 matrix (K bytes per row, K a multiple of 16) times NB vectors held in shared
 // memory as [NB][K]; emit(row, b, acc) runs once per (row, b < NB) on one lane.  gs lanes share a row (a power of two
 // that divides the number of 16-byte chunks of a row, so that every lane takes the same number of chunks CPL).
-template <int NB, int CPL, class F>
+// A warp keeps the weight loads of two rows per lane in flight (R2): the loop is bound by the latency of those loads
+// and by the shared-memory reads of the vectors, which the two rows share.
+template <int NB, int CPL, bool R2, class F>
 __device__ __forceinline__ void matvec_rows_t(const int8_t *rows, int nrows, int K, int gs, const int8_t *vec_s, F emit)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int lg = lane & (gs - 1), sub = lane / gs, rpw = 32 / gs;
-    const int chunks = K >> 4;
-    const int cpl = CPL > 0 ? CPL : chunks / gs;
+    const int stride = SK_WARPS * rpw;
+    constexpr int NR = R2 ? 2 : 1;
+    for (int r0 = warp * rpw; r0 < nrows; r0 += stride * NR) {
+        int32_t acc[NR][NB];
+        uint4 w[NR][CPL];
+        bool valid[NR];
+#pragma unroll
+        for (int q = 0; q < NR; ++q) {
+            const int r = r0 + q * stride + sub;
+            valid[q] = r < nrows;
+            const uint4 *wp = reinterpret_cast<const uint4 *>(rows + (size_t)(valid[q] ? r : 0) * K) + lg;
+#pragma unroll
+            for (int j = 0; j < CPL; ++j) w[q][j] = valid[q] ? ld_stream(wp + j * gs) : make_uint4(0, 0, 0, 0);   // all loads in flight
+        }
+#pragma unroll
+        for (int q = 0; q < NR; ++q)
+#pragma unroll
+            for (int b = 0; b < NB; ++b) acc[q][b] = 0;
+        // every vector chunk is read from shared memory once and used for both rows
+#pragma unroll
+        for (int j = 0; j < CPL; ++j) {
+#pragma unroll
+            for (int b = 0; b < NB; ++b) {
+                const uint4 v = reinterpret_cast<const uint4 *>(vec_s + (size_t)b * K)[lg + j * gs];
+#pragma unroll
+                for (int q = 0; q < NR; ++q) {
+                    acc[q][b] = __dp4a((int)w[q][j].x, (int)v.x, acc[q][b]);
+                    acc[q][b] = __dp4a((int)w[q][j].y, (int)v.y, acc[q][b]);
+                    acc[q][b] = __dp4a((int)w[q][j].z, (int)v.z, acc[q][b]);
+                    acc[q][b] = __dp4a((int)w[q][j].w, (int)v.w, acc[q][b]);
+                }
+            }
+        }
+        for (int off = gs >> 1; off > 0; off >>= 1) {
+#pragma unroll
+            for (int q = 0; q < NR; ++q)
+#pragma unroll
+                for (int b = 0; b < NB; ++b) acc[q][b] += __shfl_xor_sync(0xffffffffu, acc[q][b], off);
+        }
+#pragma unroll
+        for (int q = 0; q < NR; ++q) {
+            if (valid[q]) {
+#pragma unroll
+                for (int b = 0; b < NB; ++b)
+                    if ((b & (gs - 1)) == lg) emit(r0 + q * stride + sub, b, acc[q][b]);   // the lanes of a row share out the batch rows
+            }
+        }
+    }
+}
+
+// any number of chunks per lane: one load at a time, four trips unrolled
+template <int NB, class F>
+__device__ __forceinline__ void matvec_rows_any(const int8_t *rows, int nrows, int K, int gs, const int8_t *vec_s, F emit)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lg = lane & (gs - 1), sub = lane / gs, rpw = 32 / gs;
+    const int cpl = (K >> 4) / gs;
     for (int r0 = warp * rpw; r0 < nrows; r0 += SK_WARPS * rpw) {
         const int r = r0 + sub;
         const bool valid = r < nrows;
@@ -146,33 +206,16 @@ __device__ __forceinline__ void matvec_rows_t(const int8_t *rows, int nrows, int
         for (int b = 0; b < NB; ++b) acc[b] = 0;
         if (valid) {
             const uint4 *wp = reinterpret_cast<const uint4 *>(rows + (size_t)r * K) + lg;
-            if (CPL > 0) {
-                uint4 w[CPL > 0 ? CPL : 1];
-#pragma unroll
-                for (int j = 0; j < CPL; ++j) w[j] = ld_stream(wp + j * gs);             // all loads of the row in flight
-#pragma unroll
-                for (int j = 0; j < CPL; ++j) {
-#pragma unroll
-                    for (int b = 0; b < NB; ++b) {
-                        const uint4 v = reinterpret_cast<const uint4 *>(vec_s + (size_t)b * K)[lg + j * gs];
-                        acc[b] = __dp4a((int)w[j].x, (int)v.x, acc[b]);
-                        acc[b] = __dp4a((int)w[j].y, (int)v.y, acc[b]);
-                        acc[b] = __dp4a((int)w[j].z, (int)v.z, acc[b]);
-                        acc[b] = __dp4a((int)w[j].w, (int)v.w, acc[b]);
-                    }
-                }
-            } else {
 #pragma unroll 4
-                for (int j = 0; j < cpl; ++j) {
-                    const uint4 w = ld_stream(wp + j * gs);
+            for (int j = 0; j < cpl; ++j) {
+                const uint4 w = ld_stream(wp + j * gs);
 #pragma unroll
-                    for (int b = 0; b < NB; ++b) {
-                        const uint4 v = reinterpret_cast<const uint4 *>(vec_s + (size_t)b * K)[lg + j * gs];
-                        acc[b] = __dp4a((int)w.x, (int)v.x, acc[b]);
-                        acc[b] = __dp4a((int)w.y, (int)v.y, acc[b]);
-                        acc[b] = __dp4a((int)w.z, (int)v.z, acc[b]);
-                        acc[b] = __dp4a((int)w.w, (int)v.w, acc[b]);
-                    }
+                for (int b = 0; b < NB; ++b) {
+                    const uint4 v = reinterpret_cast<const uint4 *>(vec_s + (size_t)b * K)[lg + j * gs];
+                    acc[b] = __dp4a((int)w.x, (int)v.x, acc[b]);
+                    acc[b] = __dp4a((int)w.y, (int)v.y, acc[b]);
+                    acc[b] = __dp4a((int)w.z, (int)v.z, acc[b]);
+                    acc[b] = __dp4a((int)w.w, (int)v.w, acc[b]);
                 }
             }
         }
@@ -183,7 +226,7 @@ __device__ __forceinline__ void matvec_rows_t(const int8_t *rows, int nrows, int
         if (valid) {
 #pragma unroll
             for (int b = 0; b < NB; ++b)
-                if ((b & (gs - 1)) == lg) emit(r, b, acc[b]);        // the lanes of a row share out the batch rows
+                if ((b & (gs - 1)) == lg) emit(r, b, acc[b]);
         }
     }
 }
@@ -201,12 +244,13 @@ template <int NB, class F>
 __device__ __forceinline__ void matvec_rows(const int8_t *rows, int nrows, int K, const int8_t *vec_s, F emit)
 {
     const int gs = lanes_per_row(K);
+    constexpr bool R2 = NB <= 8;             // sixteen batch rows: the accumulators of two rows would not fit in registers
     switch ((K >> 4) / gs) {
-        case 1: matvec_rows_t<NB, 1>(rows, nrows, K, gs, vec_s, emit); break;
-        case 2: matvec_rows_t<NB, 2>(rows, nrows, K, gs, vec_s, emit); break;
-        case 4: matvec_rows_t<NB, 4>(rows, nrows, K, gs, vec_s, emit); break;
-        case 5: matvec_rows_t<NB, 5>(rows, nrows, K, gs, vec_s, emit); break;
-        default: matvec_rows_t<NB, 0>(rows, nrows, K, gs, vec_s, emit); break;
+        case 1: matvec_rows_t<NB, 1, R2>(rows, nrows, K, gs, vec_s, emit); break;
+        case 2: matvec_rows_t<NB, 2, R2>(rows, nrows, K, gs, vec_s, emit); break;
+        case 4: matvec_rows_t<NB, 4, R2>(rows, nrows, K, gs, vec_s, emit); break;
+        case 5: matvec_rows_t<NB, 5, R2>(rows, nrows, K, gs, vec_s, emit); break;
+        default: matvec_rows_any<NB>(rows, nrows, K, gs, vec_s, emit); break;
     }
 }
 
@@ -227,244 +271,337 @@ __device__ __forceinline__ void stage_vec_bytes(int8_t *dst_s, const int8_t *src
     for (int i = threadIdx.x; i < NB * K; i += SK_THREADS) dst_s[i] = (i < B * K) ? src[i] : (int8_t)0;
 }
 
+// What a block does for one layer: its share of the cells and of the projection rows, and where things live.
+struct Role {
+    const SkLayer *L;              // shared memory
+    int li, rank;
+    int u0, cells, npc, n0, n_cnt; // own cells and gate rows
+    int p_lo, p_cnt;               // own projection rows
+    int16_t *c_s;                  // [NB][cpc] cell state, resident over the call
+    unsigned *cnt;                 // the layer's counters
+    const unsigned *cnt_below;     // CNT_H of the layer below, or null
+    unsigned n_below;
+    const int8_t *in_seq;          // [T][B][I]
+    int8_t *out_seq;               // [T][B][O]
+    int8_t *h_state;
+    int16_t *c_state;
+};
+
 struct SkSmem {
     int8_t *x_s, *h_s, *m_s;       // staged operands [NB][I], [NB][O], [NB][C]
-    int16_t *xs_s;                 // [NB][npc] rescaled input term
+    int16_t *xs_s, *hs_s;          // [NB][npc] rescaled input and recurrent terms
     int16_t *pre_s;                // [NB][npc] gate sums
-    int16_t *ho_s;                 // [NB][cpc] peephole: recurrent term of the output gate (its X stays in pre_s)
-    int16_t *c_s;                  // [NB][cpc] cell state of the block's cells, resident over the call
     LnRow *ln_s;                   // [NB][4]
 };
 
+// ---- the pieces of one layer-step -------------------------------------------------------------------------------
+
+// input term (Section 3.2.4, first rescale): xs = sat16(rescale(W x_t + bx, eff_x))
+template <int NB>
+__device__ __forceinline__ void input_term(const SkCall &k, const Role &r, const SkSmem &s, int t)
+{
+    const SkLayer &L = *r.L;
+    stage_vec(s.x_s, r.in_seq + (size_t)t * k.B * L.I, k.B, NB, L.I);
+    __syncthreads();
+    const int B = k.B, npc = r.npc, n0 = r.n0, G = L.G;
+    matvec_rows<NB>(L.W + (size_t)n0 * L.I, r.n_cnt, L.I, s.x_s, [&](int n, int b, int32_t acc) {
+        if (b < B) s.xs_s[b * npc + n] = (int16_t)sat16(sk_rescale(acc + L.bx[n0 + n], L.eff_x[n % G]));
+    });
+}
+
+// recurrent term: hs = sat16(rescale(sat32(R h^{t-1} + bh), eff_h)); h^{t-1} is the previous row block of the layer's
+// output sequence (the caller's h at t = 0)
+template <int NB>
+__device__ __forceinline__ void recurrent_term(const SkCall &k, const Role &r, const SkSmem &s, int t)
+{
+    const SkLayer &L = *r.L;
+    if (t == 0) stage_vec_bytes(s.h_s, r.h_state, k.B, NB, L.O);
+    else stage_vec(s.h_s, r.out_seq + (size_t)(t - 1) * k.B * L.O, k.B, NB, L.O);
+    __syncthreads();
+    const int B = k.B, npc = r.npc, n0 = r.n0, G = L.G;
+    matvec_rows<NB>(L.R + (size_t)n0 * L.O, r.n_cnt, L.O, s.h_s, [&](int n, int b, int32_t acc) {
+        if (b < B) s.hs_s[b * npc + n] = (int16_t)sat16(sk_rescale(sk_add_sat(acc, L.bh[n0 + n]), L.eff_h[n % G]));
+    });
+}
+
+// layer-norm constants of the rows for the gate slots in `slots`: the block's per-row sums go to global memory, the
+// group meets, every block adds the group's shares (integer sums: the order does not matter)
+__device__ __forceinline__ bool exchange_stats(const SkCall &k, const Role &r, const SkSmem &s, int round, unsigned slots,
+                                               unsigned *counter, unsigned target, int *abort_s)
+{
+    const SkLayer &L = *r.L;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, B = k.B, G = L.G;
+    long long *mine = L.part + ((size_t)r.rank * 2 + round) * B * 8;
+    for (int task = warp; task < B * 4; task += SK_WARPS) {
+        const int b = task >> 2, gi = task & 3;
+        if (!((slots >> gi) & 1u)) continue;
+        long long sum = 0, sq = 0;
+        for (int ul = lane; ul < r.cells; ul += 32) {
+            const int32_t v = s.pre_s[b * r.npc + ul * G + gi];
+            sum += v;
+            sq += (long long)(v * v);
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            sum += __shfl_down_sync(0xffffffffu, sum, o);
+            sq += __shfl_down_sync(0xffffffffu, sq, o);
+        }
+        if (lane == 0) { mine[task * 2] = sum; mine[task * 2 + 1] = sq; }
+    }
+    sk_arrive(counter);
+    if (!sk_wait(k, counter, target, abort_s)) return false;
+    for (int task = warp; task < B * 4; task += SK_WARPS) {
+        const int gi = task & 3;
+        if (!((slots >> gi) & 1u)) continue;
+        long long sum = 0, sq = 0;
+        for (int q = lane; q < L.n_cta; q += 32) {
+            const long long *share = L.part + ((size_t)q * 2 + round) * B * 8 + task * 2;
+            sum += __ldcg(share);
+            sq += __ldcg(share + 1);
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            sum += __shfl_down_sync(0xffffffffu, sum, o);
+            sq += __shfl_down_sync(0xffffffffu, sq, o);
+        }
+        if (lane == 0) s.ln_s[task] = make_ln_row(ln_stats(sum, sq, L.C));
+    }
+    __syncthreads();
+    return true;
+}
+
+// everything of step t after the two terms; ends with the block's arrival on the layer's step counter
+template <int NB>
+__device__ __forceinline__ bool finish_step(const SkCall &k, const Role &r, const SkSmem &s, int t, int *abort_s)
+{
+    const SkLayer &L = *r.L;
+    const int B = k.B, G = L.G, C = L.C, O = L.O, npc = r.npc, cells = r.cells, n0 = r.n0, u0 = r.u0, cpc = L.cpc;
+    const bool proj = (L.flags & F_PROJECTION) != 0, ln = (L.flags & F_LAYERNORM) != 0, peep = (L.flags & F_PEEPHOLE) != 0;
+    const int SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
+    const unsigned n_grp = (unsigned)L.n_cta;
+    __syncthreads();
+    // gate sums (Section 3.2.4 / 3.2.5): X + H (+ peephole on c^{t-1} for the input and forget gates); with a peephole the
+    // output gate's sum waits for c^t (Eq. 5)
+    for (int i = threadIdx.x; i < B * r.n_cnt; i += SK_THREADS) {
+        const int b = i / r.n_cnt, n = i - b * r.n_cnt, gi = n % G, ul = n / G;
+        int32_t v = (int32_t)s.xs_s[b * npc + n] + (int32_t)s.hs_s[b * npc + n];
+        if (peep && gi == SO) continue;
+        if (peep && gi != SZ) v += sat16(sk_rescale((int32_t)L.P[n0 + n] * r.c_s[b * cpc + ul], L.eff_c[gi]));
+        s.pre_s[b * npc + n] = (int16_t)sat16(v);
+    }
+    __syncthreads();
+    if (ln) {
+        const unsigned all = (1u << G) - 1u;
+        if (!exchange_stats(k, r, s, 0, peep ? (all & ~(1u << SO)) : all, r.cnt + CNT_A, (unsigned)(t + 1) * n_grp, abort_s)) return false;
+    }
+    // elementwise, one cell per thread
+    for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
+        const int b = i / cells, ul = i - b * cells;
+        const int nl = ul * G, n = n0 + nl;
+        const int16_t *pre = s.pre_s + b * npc + nl;
+        const LnRow *lr = s.ln_s + b * 4;
+        // input of the nonlinearity of gate slot g: the gate sum, after layer norm when the layer has it
+        auto gate_in = [&](int g) -> int32_t {
+            const int32_t v = pre[g];
+            return ln ? ln_apply_fast(v, lr[g], L.L[n + g], L.bln[n + g], L.eff_ln[g], make_fast_scale(L.eff_ln[g])) : v;
+        };
+        const int32_t f = sigmoid_q_fast(gate_in(SF), 3), z = tanh_q_fast(gate_in(SZ), 3);
+        int32_t ig;
+        if (G == 4) ig = sigmoid_q_fast(gate_in(0), 3);
+        else { ig = 32768 - f; if (ig > 32767) ig = 32767; }    // coupled input gate, Section 3.2.9
+        const int32_t c_old = r.c_s[b * cpc + ul];
+        const int32_t c_new = cell_update_fast(ig, z, f, c_old, L.m_bits);
+        r.c_s[b * cpc + ul] = (int16_t)c_new;
+        int32_t ao;
+        if (peep) {
+            ao = sat16((int32_t)s.xs_s[b * npc + nl + SO] + (int32_t)s.hs_s[b * npc + nl + SO] +
+                       sat16(sk_rescale((int32_t)L.P[n + SO] * c_new, L.eff_c[SO])));
+            if (ln) { s.pre_s[b * npc + nl + SO] = (int16_t)ao; continue; }      // waits for the row's statistics
+        } else {
+            ao = gate_in(SO);
+        }
+        const int32_t mq = hidden_q_fast(sigmoid_q_fast(ao, 3), c_new, L.m_bits, L.eff_m, make_fast_scale(L.eff_m), L.zp_m);
+        if (proj) L.m[(size_t)b * C + u0 + ul] = (int8_t)mq;
+        else r.out_seq[((size_t)t * B + b) * O + u0 + ul] = (int8_t)mq;
+    }
+    if (ln && peep) {
+        __syncthreads();
+        if (!exchange_stats(k, r, s, 1, 1u << SO, r.cnt + CNT_A2, (unsigned)(t + 1) * n_grp, abort_s)) return false;
+        for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
+            const int b = i / cells, ul = i - b * cells;
+            const int n = n0 + ul * G + SO;
+            const int32_t ao = ln_apply_fast(s.pre_s[b * npc + ul * G + SO], s.ln_s[b * 4 + SO], L.L[n], L.bln[n], L.eff_ln[SO],
+                                             make_fast_scale(L.eff_ln[SO]));
+            const int32_t mq = hidden_q_fast(sigmoid_q_fast(ao, 3), r.c_s[b * cpc + ul], L.m_bits, L.eff_m,
+                                             make_fast_scale(L.eff_m), L.zp_m);
+            if (proj) L.m[(size_t)b * C + u0 + ul] = (int8_t)mq;
+            else r.out_seq[((size_t)t * B + b) * O + u0 + ul] = (int8_t)mq;
+        }
+    }
+    // projection (Section 3.2.8): needs every m of the layer
+    if (proj) {
+        sk_arrive(r.cnt + CNT_M);
+        if (!sk_wait(k, r.cnt + CNT_M, (unsigned)(t + 1) * n_grp, abort_s)) return false;
+        stage_vec(s.m_s, L.m, B, NB, C);
+        __syncthreads();
+        const int p_lo = r.p_lo;
+        int8_t *out = r.out_seq + (size_t)t * B * O;
+        matvec_rows<NB>(L.Wproj + (size_t)p_lo * C, r.p_cnt, C, s.m_s, [&](int row, int b, int32_t acc) {
+            if (b < B) out[(size_t)b * O + p_lo + row] = (int8_t)sat8(sk_rescale(sk_add_sat(acc, L.bp[p_lo + row]), L.eff_proj) + L.zp_h);
+        });
+    }
+    // h^t is complete once every block of the group has arrived
+    sk_arrive(r.cnt + CNT_H);
+    return true;
+}
+
+__device__ __forceinline__ Role make_role(const SkCall &k, const SkLayer *Ls, int li, int rank, int16_t *c_s)
+{
+    const SkLayer &L = Ls[li];
+    Role r;
+    r.L = &L; r.li = li; r.rank = rank;
+    r.u0 = rank * L.cpc;
+    r.cells = L.C - r.u0 < L.cpc ? L.C - r.u0 : L.cpc;
+    if (r.cells < 0) r.cells = 0;
+    r.npc = L.cpc * L.G; r.n0 = r.u0 * L.G; r.n_cnt = r.cells * L.G;
+    r.p_lo = rank * L.rpc;
+    r.p_cnt = (L.flags & F_PROJECTION) ? (L.O - r.p_lo < L.rpc ? L.O - r.p_lo : L.rpc) : 0;
+    if (r.p_cnt < 0) r.p_cnt = 0;
+    r.c_s = c_s;
+    r.cnt = k.cnt + (size_t)li * CNT_PER_LAYER;
+    r.cnt_below = li > 0 ? k.cnt + (size_t)(li - 1) * CNT_PER_LAYER + CNT_H : nullptr;
+    r.n_below = li > 0 ? (unsigned)Ls[li - 1].n_cta : 0u;
+    r.in_seq = li > 0 ? Ls[li - 1].seq : k.x;
+    r.out_seq = L.seq ? L.seq : k.y;
+    r.h_state = k.h + L.h_off * k.B;
+    r.c_state = k.c + L.c_off * k.B;
+    return r;
+}
+
+// Two schedules, chosen by the host per call:
+//   wavefront   one group of blocks per layer; group l works on step t while group l + 1 works on step t - 1.  Between
+//               its arrival at the end of step t and the wait for the group, a block already computes the input term of
+//               step t + 1 (which needs the layer below, not the block's own group).
+//   sequential  every layer on all blocks, one layer after the other (calls of a few steps: there is nothing to
+//               overlap across steps, and a layer gets the whole machine's bandwidth).  Between its arrival at the end
+//               of layer l and the wait, a block already computes the recurrent term of layer l + 1 (which needs that
+//               layer's own h^{t-1}, not layer l).
 template <int NB>
 __global__ void __launch_bounds__(SK_THREADS, 1) k_stack_small(const SkLayer *__restrict__ layers, SkCall k)
 {
     extern __shared__ __align__(16) uint8_t sk_smem[];
-    __shared__ SkLayer L;
     __shared__ int abort_s;
-    const int cta = blockIdx.x;
-    // which layer this block belongs to
-    int li = -1;
-    for (int l = 0; l < k.n_layers; ++l)
-        if (cta >= layers[l].cta0 && cta < layers[l].cta0 + layers[l].n_cta) li = l;
-    if (li < 0) return;                                        // spare block: takes no part in any counter
-    if (threadIdx.x == 0) { L = layers[li]; abort_s = 0; }
+    const int cta = blockIdx.x, nl = k.n_layers, B = k.B, T = k.T;
+    // the layer descriptions, then the buffers (sized for the widest layer), then the cell states
+    SkLayer *Ls = reinterpret_cast<SkLayer *>(sk_smem);
+    for (int i = threadIdx.x; i < (int)(nl * sizeof(SkLayer) / 4); i += SK_THREADS)
+        reinterpret_cast<uint32_t *>(Ls)[i] = reinterpret_cast<const uint32_t *>(layers)[i];
+    if (threadIdx.x == 0) abort_s = 0;
     __syncthreads();
-
-    const int B = k.B, T = k.T;
-    const int G = L.G, I = L.I, C = L.C, O = L.O;
-    const bool proj = (L.flags & F_PROJECTION) != 0, ln = (L.flags & F_LAYERNORM) != 0, peep = (L.flags & F_PEEPHOLE) != 0;
-    const int SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
-    const int rank = cta - L.cta0;                             // block within the group
-    const int u0 = rank * L.cpc;
-    int cells = C - u0 < L.cpc ? C - u0 : L.cpc;
-    if (cells < 0) cells = 0;
-    const int npc = L.cpc * G, n0 = u0 * G, n_cnt = cells * G;
-    const int p_lo = rank * L.rpc;
-    int p_cnt = proj ? (O - p_lo < L.rpc ? O - p_lo : L.rpc) : 0;
-    if (p_cnt < 0) p_cnt = 0;
-
     SkSmem s;
+    int16_t *c_base;
     {
-        uint8_t *p = sk_smem;
-        s.x_s = (int8_t *)p;  p += (size_t)NB * I;
-        s.h_s = (int8_t *)p;  p += (size_t)NB * O;
-        s.m_s = (int8_t *)p;  p += proj ? (size_t)NB * C : 0;
-        s.xs_s = (int16_t *)p; p += (size_t)NB * npc * 2;
-        s.pre_s = (int16_t *)p; p += (size_t)NB * npc * 2;
-        s.ho_s = (int16_t *)p; p += (size_t)NB * L.cpc * 2;
-        s.c_s = (int16_t *)p;  p += (size_t)NB * L.cpc * 2;
-        p = (uint8_t *)(((uintptr_t)p + 15) & ~(uintptr_t)15);
-        s.ln_s = (LnRow *)p;
+        uint8_t *p = sk_smem + (((size_t)nl * sizeof(SkLayer) + 15) & ~(size_t)15);
+        s.x_s = (int8_t *)p;  p += (size_t)NB * k.max_I;
+        s.h_s = (int8_t *)p;  p += (size_t)NB * k.max_O;
+        s.m_s = (int8_t *)p;  p += (size_t)NB * k.max_C_proj;
+        s.ln_s = (LnRow *)p;  p += (size_t)NB * 4 * sizeof(LnRow);
+        s.xs_s = (int16_t *)p; p += (size_t)NB * k.max_npc * 2;
+        s.hs_s = (int16_t *)p; p += (size_t)NB * k.max_npc * 2;
+        s.pre_s = (int16_t *)p; p += (size_t)NB * k.max_npc * 2;
+        c_base = (int16_t *)p;
     }
-    unsigned *cnt = k.cnt + (size_t)li * CNT_PER_LAYER;
-    const unsigned *cnt_below = li > 0 ? k.cnt + (size_t)(li - 1) * CNT_PER_LAYER + CNT_H : nullptr;
-    const unsigned n_below = li > 0 ? (unsigned)layers[li - 1].n_cta : 0u;
-    const unsigned n_grp = (unsigned)L.n_cta;
-    const int8_t *in_seq = li > 0 ? layers[li - 1].seq : k.x;  // [T][B][I]
-    int8_t *out_seq = L.seq ? L.seq : k.y;                     // [T][B][O]
-    int8_t *h_state = k.h + L.h_off * B;
-    int16_t *c_state = k.c + L.c_off * B;
+    bool ok = true;
 
-    // cell state of the block's cells
-    for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
-        const int b = i / cells, ul = i - b * cells;
-        s.c_s[b * L.cpc + ul] = c_state[(size_t)b * C + u0 + ul];
-    }
-    __syncthreads();
-
-    // ---- input term of step t: waits for x_t from the layer below
-    auto input_term = [&](int t) -> bool {
-        if (li > 0 && !sk_wait(k, cnt_below, (unsigned)(t + 1) * n_below, &abort_s)) return false;
-        stage_vec(s.x_s, in_seq + (size_t)t * B * I, B, NB, I);
-        __syncthreads();
-        matvec_rows<NB>(L.W + (size_t)n0 * I, n_cnt, I, s.x_s, [&](int n, int b, int32_t acc) {
-            if (b < B) s.xs_s[b * npc + n] = (int16_t)sat16(sk_rescale(acc + L.bx[n0 + n], L.eff_x[n % G]));
-        });
-        return true;
-    };
-
-    // layer-norm constants of the rows for the gate slots in `slots`, from the group's shares
-    auto exchange_stats = [&](int round, unsigned slots, unsigned *counter, unsigned target) -> bool {
-        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-        long long *mine = L.part + ((size_t)rank * 2 + round) * B * 8;
-        for (int task = warp; task < B * 4; task += SK_WARPS) {
-            const int b = task >> 2, gi = task & 3;
-            if (!((slots >> gi) & 1u)) continue;
-            long long sum = 0, sq = 0;
-            for (int ul = lane; ul < cells; ul += 32) {
-                const int32_t v = s.pre_s[b * npc + ul * G + gi];
-                sum += v;
-                sq += (long long)(v * v);
-            }
-            for (int o = 16; o > 0; o >>= 1) {
-                sum += __shfl_down_sync(0xffffffffu, sum, o);
-                sq += __shfl_down_sync(0xffffffffu, sq, o);
-            }
-            if (lane == 0) { mine[task * 2] = sum; mine[task * 2 + 1] = sq; }
-        }
-        sk_arrive(counter);
-        if (!sk_wait(k, counter, target, &abort_s)) return false;
-        for (int task = warp; task < B * 4; task += SK_WARPS) {
-            const int gi = task & 3;
-            if (!((slots >> gi) & 1u)) continue;
-            long long sum = 0, sq = 0;
-            for (int r = lane; r < L.n_cta; r += 32) {
-                const long long *share = L.part + ((size_t)r * 2 + round) * B * 8 + task * 2;
-                sum += __ldcg(share);
-                sq += __ldcg(share + 1);
-            }
-            for (int o = 16; o > 0; o >>= 1) {
-                sum += __shfl_down_sync(0xffffffffu, sum, o);
-                sq += __shfl_down_sync(0xffffffffu, sq, o);
-            }
-            if (lane == 0) s.ln_s[task] = make_ln_row(ln_stats(sum, sq, C));
+    if (!k.sequential) {
+        int li = -1;
+        for (int l = 0; l < nl; ++l)
+            if (cta >= Ls[l].cta0 && cta < Ls[l].cta0 + Ls[l].n_cta) li = l;
+        if (li < 0) return;                                    // spare block: takes no part in any counter
+        const Role r = make_role(k, Ls, li, cta - Ls[li].cta0, c_base);
+        const unsigned n_grp = (unsigned)r.L->n_cta;
+        for (int i = threadIdx.x; i < B * r.cells; i += SK_THREADS) {
+            const int b = i / r.cells, ul = i - b * r.cells;
+            r.c_s[b * r.L->cpc + ul] = r.c_state[(size_t)b * r.L->C + r.u0 + ul];
         }
         __syncthreads();
-        return true;
-    };
-
-    bool ok = input_term(0);
-    for (int t = 0; t < T && ok; ++t) {
-        // ---- recurrent term: h^{t-1} is the previous row block of this layer's output (the caller's h at t = 0)
-        if (t == 0) {
-            stage_vec_bytes(s.h_s, h_state, B, NB, O);
-        } else {
-            stage_vec(s.h_s, out_seq + (size_t)(t - 1) * B * O, B, NB, O);
+        if (r.cnt_below) ok = sk_wait(k, r.cnt_below, r.n_below, &abort_s);
+        if (ok) input_term<NB>(k, r, s, 0);
+        for (int t = 0; t < T && ok; ++t) {
+            recurrent_term<NB>(k, r, s, t);
+            ok = finish_step<NB>(k, r, s, t, &abort_s);
+            if (!ok) break;
+            if (t + 1 < T) {
+                if (r.cnt_below) ok = sk_wait(k, r.cnt_below, (unsigned)(t + 2) * r.n_below, &abort_s);
+                if (!ok) break;
+                input_term<NB>(k, r, s, t + 1);
+            }
+            ok = sk_wait(k, r.cnt + CNT_H, (unsigned)(t + 1) * n_grp, &abort_s);
+        }
+        if (ok) {
+            for (int i = threadIdx.x; i < B * r.cells; i += SK_THREADS) {
+                const int b = i / r.cells, ul = i - b * r.cells;
+                r.c_state[(size_t)b * r.L->C + r.u0 + ul] = r.c_s[b * r.L->cpc + ul];
+            }
+            if (T > 0) {
+                // every block copies its share of the columns of h = the last row block of the output sequence
+                const int O = r.L->O, per = (O + r.L->n_cta - 1) / r.L->n_cta, o_lo = r.rank * per;
+                const int o_hi = o_lo + per < O ? o_lo + per : O;
+                for (int b = 0; b < B; ++b)
+                    for (int o = o_lo + (int)threadIdx.x; o < o_hi; o += SK_THREADS)
+                        r.h_state[(size_t)b * O + o] = __ldcg(r.out_seq + ((size_t)(T - 1) * B + b) * O + o);
+            }
+        }
+    } else {
+        // cell states of this block's cells of every layer
+        int c_off = 0;
+        for (int l = 0; l < nl; ++l) {
+            const Role r = make_role(k, Ls, l, cta, c_base + c_off);
+            for (int i = threadIdx.x; i < B * r.cells; i += SK_THREADS) {
+                const int b = i / r.cells, ul = i - b * r.cells;
+                r.c_s[b * r.L->cpc + ul] = r.c_state[(size_t)b * r.L->C + r.u0 + ul];
+            }
+            c_off += NB * Ls[l].cpc;
         }
         __syncthreads();
-        matvec_rows<NB>(L.R + (size_t)n0 * O, n_cnt, O, s.h_s, [&](int n, int b, int32_t acc) {
-            if (b >= B) return;
-            const int gi = n % G, ul = n / G;
-            const int32_t H = sat16(sk_rescale(sk_add_sat(acc, L.bh[n0 + n]), L.eff_h[gi]));
-            const int32_t X = s.xs_s[b * npc + n];
-            if (peep && gi == SO) {
-                s.pre_s[b * npc + n] = (int16_t)X;               // finished after the cell update (Eq. 5: o sees c^t)
-                s.ho_s[b * L.cpc + ul] = (int16_t)H;
-            } else {
-                int32_t v = X + H;
-                if (peep && gi != SZ) v += sat16(sk_rescale((int32_t)L.P[n0 + n] * s.c_s[b * L.cpc + ul], L.eff_c[gi]));
-                s.pre_s[b * npc + n] = (int16_t)sat16(v);
-            }
-        });
-        __syncthreads();
-        if (ln) {
-            const unsigned all = (1u << G) - 1u;
-            ok = exchange_stats(0, peep ? (all & ~(1u << SO)) : all, cnt + CNT_A, (unsigned)(t + 1) * n_grp);
-            if (!ok) break;
-        }
-
-        // ---- elementwise, one cell per thread
-        for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
-            const int b = i / cells, ul = i - b * cells;
-            const int nl = ul * G, n = n0 + nl;
-            const int16_t *pre = s.pre_s + b * npc + nl;
-            const LnRow *lr = s.ln_s + b * 4;
-            // input of the nonlinearity of gate slot g: the gate sum, after layer norm when the layer has it
-            auto gate_in = [&](int g) -> int32_t {
-                const int32_t v = pre[g];
-                return ln ? ln_apply_fast(v, lr[g], L.L[n + g], L.bln[n + g], L.eff_ln[g], make_fast_scale(L.eff_ln[g])) : v;
-            };
-            const int32_t f = sigmoid_q_fast(gate_in(SF), 3), z = tanh_q_fast(gate_in(SZ), 3);
-            int32_t ig;
-            if (G == 4) ig = sigmoid_q_fast(gate_in(0), 3);
-            else { ig = 32768 - f; if (ig > 32767) ig = 32767; }    // coupled input gate, Section 3.2.9
-            const int32_t c_old = s.c_s[b * L.cpc + ul];
-            const int32_t c_new = cell_update_fast(ig, z, f, c_old, L.m_bits);
-            s.c_s[b * L.cpc + ul] = (int16_t)c_new;
-            int32_t ao = peep ? (int32_t)pre[SO] : gate_in(SO);
-            if (peep) {
-                ao = sat16(ao + s.ho_s[b * L.cpc + ul] + sat16(sk_rescale((int32_t)L.P[n + SO] * c_new, L.eff_c[SO])));
-                if (ln) { s.pre_s[b * npc + nl + SO] = (int16_t)ao; continue; }      // waits for the row's statistics
-            }
-            const int32_t mq = hidden_q_fast(sigmoid_q_fast(ao, 3), c_new, L.m_bits, L.eff_m, make_fast_scale(L.eff_m), L.zp_m);
-            if (proj) L.m[(size_t)b * C + u0 + ul] = (int8_t)mq;
-            else out_seq[((size_t)t * B + b) * O + u0 + ul] = (int8_t)mq;
-        }
-        if (ln && peep) {
-            __syncthreads();
-            ok = exchange_stats(1, 1u << SO, cnt + CNT_A2, (unsigned)(t + 1) * n_grp);
-            if (!ok) break;
-            for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
-                const int b = i / cells, ul = i - b * cells;
-                const int n = n0 + ul * G + SO;
-                const int32_t ao = ln_apply_fast(s.pre_s[b * npc + ul * G + SO], s.ln_s[b * 4 + SO], L.L[n], L.bln[n], L.eff_ln[SO],
-                                                 make_fast_scale(L.eff_ln[SO]));
-                const int32_t mq = hidden_q_fast(sigmoid_q_fast(ao, 3), s.c_s[b * L.cpc + ul], L.m_bits, L.eff_m,
-                                                 make_fast_scale(L.eff_m), L.zp_m);
-                if (proj) L.m[(size_t)b * C + u0 + ul] = (int8_t)mq;
-                else out_seq[((size_t)t * B + b) * O + u0 + ul] = (int8_t)mq;
+        for (int t = 0; t < T && ok; ++t) {
+            c_off = 0;
+            for (int l = 0; l < nl && ok; ++l) {
+                const Role r = make_role(k, Ls, l, cta, c_base + c_off);
+                c_off += NB * Ls[l].cpc;
+                const unsigned n_grp = (unsigned)r.L->n_cta;
+                // this layer's own h^{t-1} (complete long ago for every layer but the last)
+                if (t > 0) ok = sk_wait(k, r.cnt + CNT_H, (unsigned)t * n_grp, &abort_s);
+                if (!ok) break;
+                recurrent_term<NB>(k, r, s, t);
+                // the layer below at this step: its arrival was the last thing this block did
+                if (r.cnt_below) ok = sk_wait(k, r.cnt_below, (unsigned)(t + 1) * r.n_below, &abort_s);
+                if (!ok) break;
+                input_term<NB>(k, r, s, t);
+                ok = finish_step<NB>(k, r, s, t, &abort_s);
             }
         }
-
-        // ---- projection (Section 3.2.8): needs every m of the layer
-        if (proj) {
-            sk_arrive(cnt + CNT_M);
-            ok = sk_wait(k, cnt + CNT_M, (unsigned)(t + 1) * n_grp, &abort_s);
-            if (!ok) break;
-            stage_vec(s.m_s, L.m, B, NB, C);
-            __syncthreads();
-            matvec_rows<NB>(L.Wproj + (size_t)p_lo * C, p_cnt, C, s.m_s, [&](int r, int b, int32_t acc) {
-                if (b >= B) return;
-                const int32_t hq = sat8(sk_rescale(sk_add_sat(acc, L.bp[p_lo + r]), L.eff_proj) + L.zp_h);
-                out_seq[((size_t)t * B + b) * O + p_lo + r] = (int8_t)hq;
-            });
+        // every layer's last step complete before the state goes back
+        for (int l = 0; l < nl && ok; ++l)
+            ok = sk_wait(k, k.cnt + (size_t)l * CNT_PER_LAYER + CNT_H, (unsigned)T * (unsigned)Ls[l].n_cta, &abort_s);
+        if (ok) {
+            c_off = 0;
+            for (int l = 0; l < nl; ++l) {
+                const Role r = make_role(k, Ls, l, cta, c_base + c_off);
+                c_off += NB * Ls[l].cpc;
+                for (int i = threadIdx.x; i < B * r.cells; i += SK_THREADS) {
+                    const int b = i / r.cells, ul = i - b * r.cells;
+                    r.c_state[(size_t)b * r.L->C + r.u0 + ul] = r.c_s[b * r.L->cpc + ul];
+                }
+                if (T > 0) {
+                    const int O = r.L->O, per = (O + r.L->n_cta - 1) / r.L->n_cta, o_lo = r.rank * per;
+                    const int o_hi = o_lo + per < O ? o_lo + per : O;
+                    for (int b = 0; b < B; ++b)
+                        for (int o = o_lo + (int)threadIdx.x; o < o_hi; o += SK_THREADS)
+                            r.h_state[(size_t)b * O + o] = __ldcg(r.out_seq + ((size_t)(T - 1) * B + b) * O + o);
+                }
+            }
         }
-        // ---- end of the step: h^t is complete once every block of the group has arrived.  The input term of the next
-        // step does not need it, so it runs between the arrival and the wait.
-        sk_arrive(cnt + CNT_H);
-        if (t + 1 < T) {
-            ok = input_term(t + 1);
-            if (!ok) break;
-        }
-        ok = sk_wait(k, cnt + CNT_H, (unsigned)(t + 1) * n_grp, &abort_s);
     }
-
-    if (!ok) {
-        if (threadIdx.x == 0) atomicExch(k.status, 2);
-        return;
-    }
-    // ---- state back to the caller: c of the block's cells; h = the last row block of the output sequence
-    for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
-        const int b = i / cells, ul = i - b * cells;
-        c_state[(size_t)b * C + u0 + ul] = s.c_s[b * L.cpc + ul];
-    }
-    if (T > 0) {
-        // every block copies the part of h that belongs to its share of the output columns
-        const int per = (O + L.n_cta - 1) / L.n_cta, o_lo = rank * per;
-        const int o_hi = o_lo + per < O ? o_lo + per : O;
-        for (int b = 0; b < B; ++b)
-            for (int o = o_lo + (int)threadIdx.x; o < o_hi; o += SK_THREADS)
-                h_state[(size_t)b * O + o] = __ldcg(out_seq + ((size_t)(T - 1) * B + b) * O + o);
-    }
-}
-
-size_t sk_smem_bytes(const LayerParams &p, int cpc, int NB)
-{
-    const bool proj = (p.flags & F_PROJECTION) != 0;
-    const size_t npc = (size_t)cpc * p.G;
-    return (size_t)NB * p.I + (size_t)NB * p.O + (proj ? (size_t)NB * p.C : 0) + 2 * (size_t)NB * npc * 2 + 2 * (size_t)NB * cpc * 2 + 16 +
-           (size_t)NB * 4 * sizeof(LnRow) + 64;
+    if (!ok && threadIdx.x == 0) atomicExch(k.status, 2);
 }
 
 }  // namespace
@@ -473,8 +610,9 @@ struct StackSmall {
     bool ok = false;
     int n_layers = 0, grid = 0, max_T = 0, max_B = 0;
     size_t smem = 0;
-    SkLayer *layers_dev = nullptr;
-    std::vector<SkLayer> layers;
+    SkLayer *plan_dev[2] = {nullptr, nullptr};     // [0] wavefront, [1] sequential
+    std::vector<SkLayer> plan[2];
+    int max_I = 0, max_O = 0, max_C_proj = 0, max_npc = 0;
     std::vector<void *> owned;
     unsigned *cnt = nullptr;       // counters + abort word
     size_t cnt_words = 0;
@@ -484,8 +622,15 @@ struct StackSmall {
 
 static const void *sk_kernel(int NB)
 {
-    return NB == 1 ? (const void *)k_stack_small<1> : NB == 2 ? (const void *)k_stack_small<2> : (const void *)k_stack_small<4>;
+    switch (NB) {
+        case 1: return (const void *)k_stack_small<1>;
+        case 2: return (const void *)k_stack_small<2>;
+        case 4: return (const void *)k_stack_small<4>;
+        case 8: return (const void *)k_stack_small<8>;
+        default: return (const void *)k_stack_small<16>;
+    }
 }
+static int sk_rows(int B) { return B <= 1 ? 1 : B <= 2 ? 2 : B <= 4 ? 4 : B <= 8 ? 8 : 16; }
 
 void stack_small_destroy(StackSmall *s)
 {
@@ -494,13 +639,24 @@ void stack_small_destroy(StackSmall *s)
     delete s;
 }
 
+// shared memory of a block for NB batch rows under both schedules
+static size_t sk_smem_bytes(const StackSmall &s, int NB)
+{
+    size_t common = (((size_t)s.n_layers * sizeof(SkLayer) + 15) & ~(size_t)15) + (size_t)NB * (s.max_I + s.max_O + s.max_C_proj) +
+                    (size_t)NB * 4 * sizeof(LnRow) + 3 * (size_t)NB * s.max_npc * 2;
+    size_t c_wave = 0, c_seq = 0;
+    for (const SkLayer &L : s.plan[0]) c_wave = std::max(c_wave, (size_t)NB * L.cpc * 2);
+    for (const SkLayer &L : s.plan[1]) c_seq += (size_t)NB * L.cpc * 2;
+    return common + std::max(c_wave, c_seq) + 64;
+}
+
 // Plans the whole-stack kernel for a handle; *out stays null when the stack does not qualify (the per-layer kernels
 // then run).  max_B beyond STACK_SMALL_MAX_B is fine: the kernel is only used for smaller batches.
 int stack_small_create(const std::vector<const LayerParams *> &lp, int max_T, int max_B, int sm_count, StackSmall **out)
 {
     *out = nullptr;
     const int n = (int)lp.size();
-    if (n < 1 || n > sm_count) return QLSTM_OK;
+    if (n < 1 || n > sm_count || n > 64) return QLSTM_OK;
     for (const LayerParams *p : lp)
         if (p->I % 16 != 0 || p->O % 16 != 0 || p->C % 16 != 0) return QLSTM_OK;
     StackSmall *s = new StackSmall();
@@ -508,12 +664,17 @@ int stack_small_create(const std::vector<const LayerParams *> &lp, int max_T, in
     s->grid = sm_count;
     s->max_T = max_T;
     s->max_B = max_B < STACK_SMALL_MAX_B ? max_B : STACK_SMALL_MAX_B;
-    const int per = sm_count / n;
     int dev = 0, max_smem = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    auto fail = [&](int rc) { stack_small_destroy(s); return rc; };
+    auto dalloc = [&](size_t bytes) -> void * {
+        void *d = nullptr;
+        if (cudaMalloc(&d, bytes ? bytes : 16) != cudaSuccess) return nullptr;
+        s->owned.push_back(d);
+        return d;
+    };
     size_t h_off = 0, c_off = 0;
-    bool fits = true;
     for (int l = 0; l < n; ++l) {
         const LayerParams &p = *lp[l];
         SkLayer L;
@@ -523,48 +684,47 @@ int stack_small_create(const std::vector<const LayerParams *> &lp, int max_T, in
         L.W = p.W; L.R = p.R; L.Wproj = p.Wproj; L.bx = p.bx; L.bh = p.bh; L.bp = p.bp; L.bln = p.bln; L.P = p.P; L.L = p.L;
         for (int g = 0; g < 4; ++g) { L.eff_x[g] = p.eff_x[g]; L.eff_h[g] = p.eff_h[g]; L.eff_c[g] = p.eff_c[g]; L.eff_ln[g] = p.eff_ln[g]; }
         L.eff_m = p.eff_m; L.eff_proj = p.eff_proj;
-        L.cta0 = l * per; L.n_cta = per;
-        L.cpc = (p.C + per - 1) / per;
-        L.rpc = (p.O + per - 1) / per;
         L.h_off = h_off; L.c_off = c_off;
         h_off += p.O; c_off += p.C;
-        const size_t need = sk_smem_bytes(p, L.cpc, STACK_SMALL_MAX_B);
-        if (need > (size_t)max_smem) fits = false;
-        if (need > s->smem) s->smem = need;
-        void *d = nullptr;
         if (l + 1 < n) {
-            if (cudaMalloc(&d, (size_t)max_T * s->max_B * p.O) != cudaSuccess) { stack_small_destroy(s); return QLSTM_ERR_NOMEM; }
-            s->owned.push_back(d);
-            L.seq = (int8_t *)d;
+            L.seq = (int8_t *)dalloc((size_t)max_T * s->max_B * p.O);
+            if (!L.seq) return fail(QLSTM_ERR_NOMEM);
         }
-        if (cudaMalloc(&d, (size_t)s->max_B * p.C) != cudaSuccess) { stack_small_destroy(s); return QLSTM_ERR_NOMEM; }
-        s->owned.push_back(d);
-        L.m = (int8_t *)d;
-        if (cudaMalloc(&d, (size_t)per * 2 * s->max_B * 8 * sizeof(long long)) != cudaSuccess) { stack_small_destroy(s); return QLSTM_ERR_NOMEM; }
-        s->owned.push_back(d);
-        L.part = (long long *)d;
-        s->layers.push_back(L);
+        L.m = (int8_t *)dalloc((size_t)s->max_B * p.C);
+        L.part = (long long *)dalloc((size_t)sm_count * 2 * s->max_B * 8 * sizeof(long long));
+        if (!L.m || !L.part) return fail(QLSTM_ERR_NOMEM);
+        for (int plan = 0; plan < 2; ++plan) {
+            const int per = plan == 0 ? sm_count / n : sm_count;
+            L.cta0 = plan == 0 ? l * per : 0;
+            L.n_cta = per;
+            L.cpc = (p.C + per - 1) / per;
+            L.rpc = (p.O + per - 1) / per;
+            s->plan[plan].push_back(L);
+            s->max_npc = std::max(s->max_npc, L.cpc * p.G);
+        }
+        s->max_I = std::max(s->max_I, p.I);
+        s->max_O = std::max(s->max_O, p.O);
+        if (p.flags & F_PROJECTION) s->max_C_proj = std::max(s->max_C_proj, p.C);
     }
-    if (!fits) { stack_small_destroy(s); return QLSTM_OK; }
+    // the largest batch whose buffers fit
+    while (s->max_B >= 1 && sk_smem_bytes(*s, sk_rows(s->max_B)) > (size_t)max_smem) s->max_B = sk_rows(s->max_B) / 2;
+    if (s->max_B < 1) return fail(QLSTM_OK);
+    s->smem = sk_smem_bytes(*s, sk_rows(s->max_B));
     s->cnt_words = (size_t)n * CNT_PER_LAYER + 16;
-    if (cudaMalloc((void **)&s->cnt, s->cnt_words * sizeof(unsigned)) != cudaSuccess) { stack_small_destroy(s); return QLSTM_ERR_NOMEM; }
-    s->owned.push_back(s->cnt);
-    if (cudaMalloc((void **)&s->layers_dev, sizeof(SkLayer) * n) != cudaSuccess) { stack_small_destroy(s); return QLSTM_ERR_NOMEM; }
-    s->owned.push_back(s->layers_dev);
-    if (cudaMemcpy(s->layers_dev, s->layers.data(), sizeof(SkLayer) * n, cudaMemcpyHostToDevice) != cudaSuccess) {
-        stack_small_destroy(s);
-        return QLSTM_ERR_CUDA;
+    s->cnt = (unsigned *)dalloc(s->cnt_words * sizeof(unsigned));
+    if (!s->cnt) return fail(QLSTM_ERR_NOMEM);
+    for (int plan = 0; plan < 2; ++plan) {
+        s->plan_dev[plan] = (SkLayer *)dalloc(sizeof(SkLayer) * n);
+        if (!s->plan_dev[plan]) return fail(QLSTM_ERR_NOMEM);
+        if (cudaMemcpy(s->plan_dev[plan], s->plan[plan].data(), sizeof(SkLayer) * n, cudaMemcpyHostToDevice) != cudaSuccess)
+            return fail(QLSTM_ERR_CUDA);
     }
-    for (int NB : {1, 2, 4}) {
-        if (cudaFuncSetAttribute(sk_kernel(NB), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s->smem) != cudaSuccess) {
-            stack_small_destroy(s);
-            return QLSTM_OK;
-        }
+    for (int NB : {1, 2, 4, 8, 16}) {
+        if (NB > sk_rows(s->max_B)) break;
+        if (cudaFuncSetAttribute(sk_kernel(NB), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)s->smem) != cudaSuccess) return fail(QLSTM_OK);
         int per_sm = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sk_kernel(NB), SK_THREADS, s->smem) != cudaSuccess || per_sm < 1) {
-            stack_small_destroy(s);
-            return QLSTM_OK;
-        }
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sk_kernel(NB), SK_THREADS, s->smem) != cudaSuccess || per_sm < 1)
+            return fail(QLSTM_OK);
     }
     s->ok = true;
     *out = s;
@@ -572,6 +732,16 @@ int stack_small_create(const std::vector<const LayerParams *> &lp, int max_T, in
 }
 
 bool stack_small_supported(const StackSmall *s, int T, int B) { return s && s->ok && B >= 1 && B <= s->max_B && T >= 1 && T <= s->max_T; }
+
+// Where the whole-stack kernel is the faster path (measured): up to 4 batch rows always (27 against 144 us per time step
+// for eight 2048-cell layers at batch 1, 26 against 38 for five 1024-cell layers at batch 4); up to 8 rows for deep
+// stacks, whose layer-after-layer cost grows with the depth while the wavefront's does not (84 against 181 us at eight
+// layers; at five layers it is about even and at 16 rows the per-layer tensor-core kernels win).
+bool stack_small_preferred(const StackSmall *s, int T, int B)
+{
+    if (!stack_small_supported(s, T, B)) return false;
+    return B <= 4 || (B <= 8 && s->n_layers >= 6);
+}
 
 void stack_small_debug_timeout(StackSmall *s, unsigned missing_arrivals, unsigned long long limit_ns)
 {
@@ -583,12 +753,14 @@ void stack_small_debug_timeout(StackSmall *s, unsigned missing_arrivals, unsigne
 int stack_small_groups(const StackSmall *s, int *blocks_per_layer)
 {
     if (!s || !s->ok) return 0;
-    if (blocks_per_layer) *blocks_per_layer = s->layers.empty() ? 0 : s->layers[0].n_cta;
+    if (blocks_per_layer) *blocks_per_layer = s->plan[0].empty() ? 0 : s->plan[0][0].n_cta;
     return s->n_layers;
 }
 
+// schedule: 0 automatic (sequential for calls of a few steps, where a wavefront has nothing to overlap), 1 wavefront,
+// 2 sequential
 int launch_stack_small(const StackSmall *s, const int8_t *x, int T, int B, int8_t *h, int16_t *c, int8_t *y, int *status,
-                       cudaStream_t st)
+                       int schedule, cudaStream_t st)
 {
     SkCall k;
     memset(&k, 0, sizeof(k));
@@ -599,11 +771,13 @@ int launch_stack_small(const StackSmall *s, const int8_t *x, int T, int B, int8_
     k.status = status;
     k.wait_limit_ns = s->dbg_limit_ns ? s->dbg_limit_ns : SK_WAIT_LIMIT_NS;
     k.missing_arrivals = s->dbg_missing;
+    // a wavefront of L layers needs about L steps to fill; below that the layers are better run one after the other
+    k.sequential = schedule == 2 || (schedule == 0 && (s->n_layers == 1 || T < s->n_layers)) ? 1 : 0;
+    k.max_I = s->max_I; k.max_O = s->max_O; k.max_C_proj = s->max_C_proj; k.max_npc = s->max_npc;
     if (cudaMemsetAsync(s->cnt, 0, s->cnt_words * sizeof(unsigned), st) != cudaSuccess) return QLSTM_ERR_CUDA;
-    const int NB = B == 1 ? 1 : (B == 2 ? 2 : 4);
-    const SkLayer *layers = s->layers_dev;
+    const SkLayer *layers = s->plan_dev[k.sequential];
     void *args[] = {(void *)&layers, (void *)&k};
-    cudaError_t e = cudaLaunchCooperativeKernel(sk_kernel(NB), dim3(s->grid), dim3(SK_THREADS), args, s->smem, st);
+    cudaError_t e = cudaLaunchCooperativeKernel(sk_kernel(sk_rows(B)), dim3(s->grid), dim3(SK_THREADS), args, s->smem, st);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return e == cudaErrorCooperativeLaunchTooLarge ? QLSTM_ERR_LAUNCH : QLSTM_ERR_CUDA;

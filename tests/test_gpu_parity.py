@@ -11,7 +11,8 @@ from workloads import make_workload, random_layer_stack
 pytestmark = pytest.mark.gpu
 
 SIMPLE, FAST, AUTO = 1, 2, 0
-STACK = 5            # recurrent_impl: the whole-stack kernel for small batches, forced
+STACK = 5            # recurrent_impl: the whole-stack kernel for small batches, forced (schedule chosen by the call's length)
+STACK_WAVEFRONT, STACK_SEQUENTIAL = 6, 7          # ... with one of its two schedules forced
 
 
 def oracle(w, trace=False, x=None, h0=None, c0=None):
@@ -105,20 +106,24 @@ def test_small_batch_both_matmul_paths(B, kw):
 
 # ------------------------------------------------------------------ whole-stack kernel (batch <= 4)
 
-@pytest.mark.parametrize("B", [1, 2, 3, 4])
+@pytest.mark.parametrize("B", [1, 2, 3, 4, 7, 16])
 @pytest.mark.parametrize("kw", VARIANTS, ids=lambda k: "+".join(sorted(k)) or "basic")
 def test_stack_kernel_parity_variants(B, kw):
-    """All layers and steps in one launch, layers as a wavefront: three layers so that the wavefront is deeper than
-    one hand-over, widths that leave ragged shares to the last block of a group."""
+    """All layers and steps in one launch: three layers so that the wavefront is deeper than one hand-over, widths that
+    leave ragged shares to the last block of a group; both schedules (one group of blocks per layer / every layer on
+    all blocks)."""
     w = random_layer_stack(500 + B, 3, 48, 112, 64, T=7, B=B, **kw)
-    check_equal(run_gpu(w, impl=(AUTO, STACK)), oracle(w), f"stack kernel B={B} {kw}")
+    want = oracle(w)
+    check_equal(run_gpu(w, impl=(AUTO, STACK_WAVEFRONT)), want, f"stack kernel, wavefront, B={B} {kw}")
+    check_equal(run_gpu(w, impl=(AUTO, STACK_SEQUENTIAL)), want, f"stack kernel, sequential, B={B} {kw}")
 
 
-@pytest.mark.parametrize("index,kw", [(1, {}), (2, dict(batch=4, T=30)), (3, dict(batch=2, T=12)), (4, dict(batch=3, T=12)),
-                                      (5, dict(batch=1, T=24)), (5, dict(batch=4, T=8))])
-def test_stack_kernel_parity_configs(index, kw):
+@pytest.mark.parametrize("index,kw", [(1, {}), (2, {}), (3, dict(batch=2, T=12)), (4, dict(batch=3, T=12)),
+                                      (5, dict(batch=1, T=24)), (5, dict(batch=4, T=8)), (5, dict(batch=8, T=12))])
+@pytest.mark.parametrize("impl", [STACK_WAVEFRONT, STACK_SEQUENTIAL])
+def test_stack_kernel_parity_configs(index, kw, impl):
     w = make_workload(index, **kw)
-    check_equal(run_gpu(w, impl=(AUTO, STACK)), oracle(w), f"stack kernel config {index} {kw}")
+    check_equal(run_gpu(w, impl=(AUTO, impl)), oracle(w), f"stack kernel config {index} {kw}")
 
 
 @pytest.mark.parametrize("index,kw", [(1, {}), (2, dict(batch=2, T=20)), (5, dict(batch=1, T=10))])
@@ -150,20 +155,21 @@ def test_stack_kernel_bounded_wait_reports_timeout():
     w = random_layer_stack(58, 2, 32, 64, 48, projection=True, layernorm=True, T=4, B=2)
     want = oracle(w)
     with qlstm.QLSTM(w.layers, w.T, w.B) as hnd:
-        hnd.debug_barrier_timeout(1, 3_000_000)
-        with pytest.raises(qlstm.QlstmError) as e:
-            run_gpu(w, handle=hnd, impl=(AUTO, STACK))
-        assert e.value.code == qlstm.ERR_TIMEOUT
-        hnd.debug_barrier_timeout(0)
-        check_equal(run_gpu(w, handle=hnd, impl=(AUTO, STACK)), want, "after timeout")
+        for impl in (STACK_WAVEFRONT, STACK_SEQUENTIAL):
+            hnd.debug_barrier_timeout(1, 3_000_000)
+            with pytest.raises(qlstm.QlstmError) as e:
+                run_gpu(w, handle=hnd, impl=(AUTO, impl))
+            assert e.value.code == qlstm.ERR_TIMEOUT
+            hnd.debug_barrier_timeout(0)
+            check_equal(run_gpu(w, handle=hnd, impl=(AUTO, impl)), want, "after timeout")
 
 
 def test_stack_kernel_refuses_what_it_cannot_run():
     import paper_2101_05453_b200 as qlstm
-    w = random_layer_stack(59, 1, 32, 64, 64, T=3, B=6)
+    w = random_layer_stack(59, 1, 32, 64, 64, T=3, B=17)
     with qlstm.QLSTM(w.layers, w.T, w.B) as hnd:
         with pytest.raises(qlstm.QlstmError) as e:
-            run_gpu(w, handle=hnd, impl=(AUTO, STACK))          # batch 6 > 4
+            run_gpu(w, handle=hnd, impl=(AUTO, STACK))          # batch 17 > 16
         assert e.value.code == qlstm.ERR_DIM
 
 
