@@ -135,6 +135,26 @@ const char *qlstm_strerror(int code);
 size_t qlstm_trace_bytes(const qlstm_t *q, int T, int B);
 
 /*
+ * Bidirectional LSTM (Section 7: uni- and bidirectional LSTMs are loops over the same cell).  Two stacks of n_layers
+ * layers read the same input: `fwd` from step 0 upwards, `bwd` from step T - 1 downwards.  Both must take the same
+ * input (n_input and zp_x of their first layers equal; n_input a multiple of 16).
+ *   y_dev DEVICE int8 out [T][B][O_fwd + O_bwd]: at step t the forward stack's h^t followed by the backward stack's
+ *         state after it has seen x_{T-1} .. x_t.  The two halves keep their own (scale, zero point); a layer stacked on
+ *         top must be quantized for an input whose two halves share one (as Table 2 does for any layer input).
+ *   h_*_dev / c_*_dev DEVICE in/out state of each direction, laid out as for qlstm_run; x_dev as for qlstm_run.
+ * qlstm_bidir_create takes HOST layer descriptions like qlstm_create and owns both stacks and the workspaces between
+ * them; errors as for qlstm_create / qlstm_run.  qlstm_bidir_last_status synchronises and reports a device-side
+ * failure of either direction.
+ */
+typedef struct qlstm_bidir qlstm_bidir_t;
+int qlstm_bidir_create(const qlstm_layer_t *fwd_layers, const qlstm_layer_t *bwd_layers, int n_layers, int max_T, int max_B,
+                       int device, qlstm_bidir_t **out);
+int qlstm_bidir_run(qlstm_bidir_t *q, const int8_t *x_dev, int T, int B, int8_t *h_fwd_dev, int16_t *c_fwd_dev,
+                    int8_t *h_bwd_dev, int16_t *c_bwd_dev, int8_t *y_dev, void *cuda_stream);
+int qlstm_bidir_last_status(qlstm_bidir_t *q);
+void qlstm_bidir_destroy(qlstm_bidir_t *q);
+
+/*
  * qlstm_layernorm_rows_static - the integer layer norm of Section 3.2.6 (mean, variance, normalise x 2^10,
  * x L + b, rescale to Q3.12; one row = one (batch row, gate) of a step) for `rows` rows at once, for callers that
  * must not allocate.  (The paper has no counterpart: this is a packaging of its layer norm

@@ -23,7 +23,10 @@ EXPORTS = ["qlstm_create", "qlstm_run", "qlstm_run_host", "qlstm_input_projectio
            "qlstm_destroy", "qlstm_strerror", "qlstm_trace_bytes", "qlstm_set_impl", "qlstm_set_profiling",
            "qlstm_get_profile", "qlstm_device_info", "qlstm_eval_activations", "qlstm_eval_layernorm_row",
            "qlstm_layernorm_rows_static", "qlstm_debug_barrier_timeout", "qlstm_debug_ring_plan",
-           "qlstm_debug_projection_plan", "qlstm_debug_mma_i8_peak", "qlstm_debug_barrier_latency"]
+           "qlstm_debug_projection_plan", "qlstm_debug_mma_i8_peak", "qlstm_debug_barrier_latency",
+           "qlstm_bidir_create", "qlstm_bidir_run", "qlstm_bidir_last_status", "qlstm_bidir_destroy",
+           "qlstm_calibrate", "qlstm_quantize_model", "qlstm_quantized_layers", "qlstm_quantized_scales",
+           "qlstm_quantized_destroy"]
 
 
 class Scale(C.Structure):
@@ -41,6 +44,17 @@ class Layer(C.Structure):
         ("eff_x", Scale * 4), ("eff_h", Scale * 4), ("eff_c", Scale * 4), ("eff_ln", Scale * 4),
         ("eff_m", Scale), ("eff_proj", Scale),
     ]
+
+
+class FloatLayer(C.Structure):
+    _fields_ = [("n_input", C.c_int32), ("n_cell", C.c_int32), ("n_output", C.c_int32), ("flags", C.c_uint32),
+                ("W", C.c_void_p * 4), ("R", C.c_void_p * 4), ("P", C.c_void_p * 4), ("L", C.c_void_p * 4),
+                ("b", C.c_void_p * 4), ("W_proj", C.c_void_p), ("b_proj", C.c_void_p)]
+
+
+class Ranges(C.Structure):
+    _fields_ = [("x_min", C.c_double), ("x_max", C.c_double), ("h_min", C.c_double), ("h_max", C.c_double),
+                ("m_min", C.c_double), ("m_max", C.c_double), ("c_absmax", C.c_double), ("g_absmax", C.c_double * 4)]
 
 
 class Profile(C.Structure):
@@ -112,6 +126,24 @@ def lib():
         L.qlstm_debug_mma_i8_peak.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double)]
         L.qlstm_debug_barrier_latency.restype = C.c_int
         L.qlstm_debug_barrier_latency.argtypes = [C.c_int, C.c_int, C.POINTER(C.c_double)]
+        L.qlstm_bidir_create.restype = C.c_int
+        L.qlstm_bidir_create.argtypes = [C.POINTER(Layer), C.POINTER(Layer), C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_void_p)]
+        L.qlstm_bidir_run.restype = C.c_int
+        L.qlstm_bidir_run.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int] + [C.c_void_p] * 6
+        L.qlstm_bidir_last_status.restype = C.c_int
+        L.qlstm_bidir_last_status.argtypes = [C.c_void_p]
+        L.qlstm_bidir_destroy.restype = None
+        L.qlstm_bidir_destroy.argtypes = [C.c_void_p]
+        L.qlstm_calibrate.restype = C.c_int
+        L.qlstm_calibrate.argtypes = [C.POINTER(FloatLayer), C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.POINTER(Ranges)]
+        L.qlstm_quantize_model.restype = C.c_int
+        L.qlstm_quantize_model.argtypes = [C.POINTER(FloatLayer), C.POINTER(Ranges), C.c_int, C.c_int, C.POINTER(C.c_void_p)]
+        L.qlstm_quantized_layers.restype = C.POINTER(Layer)
+        L.qlstm_quantized_layers.argtypes = [C.c_void_p]
+        L.qlstm_quantized_scales.restype = C.c_int
+        L.qlstm_quantized_scales.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double)]
+        L.qlstm_quantized_destroy.restype = None
+        L.qlstm_quantized_destroy.argtypes = [C.c_void_p]
         L.qlstm_layernorm_rows_static.restype = C.c_int
         L.qlstm_layernorm_rows_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p,
                                                   C.c_void_p]
@@ -252,6 +284,43 @@ class QLSTM:
         return a.value, b.value
 
 
+class BiQLSTM:
+    """Handle of a bidirectional stack (qlstm_bidir_create / qlstm_bidir_run / qlstm_bidir_destroy)."""
+
+    def __init__(self, fwd_layers: Sequence, bwd_layers: Sequence, max_T: int, max_B: int, device: int = 0):
+        assert len(fwd_layers) == len(bwd_layers)
+        keep: list = []
+        fa, ba = pack_layers(fwd_layers, keep), pack_layers(bwd_layers, keep)
+        h = C.c_void_p()
+        _check(lib().qlstm_bidir_create(fa, ba, len(fwd_layers), max_T, max_B, device, C.byref(h)), "qlstm_bidir_create")
+        self._h = h
+        self.n_output = fwd_layers[-1].n_output + bwd_layers[-1].n_output
+
+    def run(self, x, T: int, B: int, h_fwd, c_fwd, h_bwd, c_bwd, y, stream: int = 0):
+        _check(lib().qlstm_bidir_run(self._h, _dev_ptr(x), T, B, _dev_ptr(h_fwd), _dev_ptr(c_fwd), _dev_ptr(h_bwd),
+                                     _dev_ptr(c_bwd), _dev_ptr(y), stream), "qlstm_bidir_run")
+
+    def last_status(self):
+        _check(lib().qlstm_bidir_last_status(self._h), "qlstm_bidir_last_status")
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().qlstm_bidir_destroy(self._h)
+            self._h = None
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *a):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
 def eval_activations(cell_int_bits: int, sigmoid_out, tanh_out, stream: int = 0):
     """qlstm_eval_activations on two device int16 [65536] tensors."""
     _check(lib().qlstm_eval_activations(cell_int_bits, _dev_ptr(sigmoid_out), _dev_ptr(tanh_out), stream),
@@ -324,3 +393,94 @@ def barrier_latency_us(device: int = 0, n_barriers: int = 2000) -> float:
     out = C.c_double()
     _check(lib().qlstm_debug_barrier_latency(device, n_barriers, C.byref(out)), "qlstm_debug_barrier_latency")
     return out.value
+
+
+# ---- calibration and quantization on the device (include/qlstm_calib.h): marshalling only
+
+_GATES = ("i", "f", "z", "o")
+
+
+def pack_float_layers(float_layers: Sequence, keep: list):
+    """Marshals float layers (objects with the fields of workloads.float_lstm.FloatLayer) into a C array."""
+    arr = (FloatLayer * len(float_layers))()
+    for d, fl in zip(arr, float_layers):
+        d.n_input, d.n_cell, d.n_output = fl.n_input, fl.n_cell, fl.n_output
+        d.flags = (1 if fl.projection else 0) | (2 if fl.peephole else 0) | (4 if fl.layernorm else 0) | (8 if fl.cifg else 0)
+        for gi, g in enumerate(_GATES):
+            if fl.cifg and g == "i":
+                continue
+            d.W[gi] = _ptr(fl.W[g], np.float64, keep)
+            d.R[gi] = _ptr(fl.R[g], np.float64, keep)
+            d.b[gi] = _ptr(fl.b[g], np.float64, keep)
+            if fl.layernorm:
+                d.L[gi] = _ptr(fl.L[g], np.float64, keep)
+            if fl.peephole and g != "z":
+                d.P[gi] = _ptr(fl.P[g], np.float64, keep)
+        if fl.projection:
+            d.W_proj = _ptr(fl.W_proj, np.float64, keep)
+            d.b_proj = _ptr(fl.b_proj, np.float64, keep)
+    return arr
+
+
+def calibrate(float_layers: Sequence, x: np.ndarray, device: int = 0):
+    """qlstm_calibrate: float forward pass on the device; returns one dict of logged ranges per layer."""
+    keep: list = []
+    arr = pack_float_layers(float_layers, keep)
+    x = np.ascontiguousarray(x, np.float64)
+    T, B, _ = x.shape
+    out = (Ranges * len(float_layers))()
+    _check(lib().qlstm_calibrate(arr, len(float_layers), x.ctypes.data, T, B, device, out), "qlstm_calibrate")
+    return [{"x_min": r.x_min, "x_max": r.x_max, "h_min": r.h_min, "h_max": r.h_max, "m_min": r.m_min, "m_max": r.m_max,
+             "c_absmax": r.c_absmax, "g_absmax": dict(zip(_GATES, r.g_absmax))} for r in out]
+
+
+class QuantizedLayer:
+    """One layer as qlstm_quantize_model produced it: the fields of qlstm_layer_t as numpy copies, plus real scales."""
+
+
+def quantize_model(float_layers: Sequence, ranges: Sequence[dict], device: int = 0):
+    """qlstm_quantize_model: Table 2 with the reductions and roundings on the device; returns QuantizedLayer objects
+    (usable wherever a layer description is expected)."""
+    keep: list = []
+    arr = pack_float_layers(float_layers, keep)
+    rg = (Ranges * len(float_layers))()
+    for d, r in zip(rg, ranges):
+        for k in ("x_min", "x_max", "h_min", "h_max", "m_min", "m_max", "c_absmax"):
+            setattr(d, k, float(r[k]))
+        for gi, g in enumerate(_GATES):
+            d.g_absmax[gi] = float(r["g_absmax"][g])
+    h = C.c_void_p()
+    _check(lib().qlstm_quantize_model(arr, rg, len(float_layers), device, C.byref(h)), "qlstm_quantize_model")
+    try:
+        ptr = lib().qlstm_quantized_layers(h)
+        out = []
+        for l in range(len(float_layers)):
+            d = ptr[l]
+            q = QuantizedLayer()
+            q.n_input, q.n_cell, q.n_output, q.flags = d.n_input, d.n_cell, d.n_output, d.flags
+            q.cell_int_bits, q.zp_x, q.zp_m, q.zp_h = d.cell_int_bits, d.zp_x, d.zp_m, d.zp_h
+
+            def grab(addr, dtype, shape):
+                if not addr:
+                    return None
+                n = int(np.prod(shape))
+                buf = (C.c_char * (n * np.dtype(dtype).itemsize)).from_address(addr)
+                return np.frombuffer(buf, dtype=dtype).reshape(shape).copy()
+            q.W = [grab(d.W[g], np.int8, (d.n_cell, d.n_input)) for g in range(4)]
+            q.R = [grab(d.R[g], np.int8, (d.n_cell, d.n_output)) for g in range(4)]
+            q.P = [grab(d.P[g], np.int16, (d.n_cell,)) for g in range(4)]
+            q.b = [grab(d.b[g], np.int32, (d.n_cell,)) for g in range(4)]
+            q.L = [grab(d.L[g], np.int16, (d.n_cell,)) for g in range(4)]
+            q.W_proj = grab(d.W_proj, np.int8, (d.n_output, d.n_cell))
+            q.b_proj = grab(d.b_proj, np.int32, (d.n_output,))
+            for name in ("eff_x", "eff_h", "eff_c", "eff_ln"):
+                setattr(q, name, [(getattr(d, name)[g].multiplier, getattr(d, name)[g].shift) for g in range(4)])
+            q.eff_m = (d.eff_m.multiplier, d.eff_m.shift)
+            q.eff_proj = (d.eff_proj.multiplier, d.eff_proj.shift)
+            sc = (C.c_double * 4)()
+            _check(lib().qlstm_quantized_scales(h, l, sc), "qlstm_quantized_scales")
+            q.s_x, q.s_h, q.s_m, q.s_c = sc[0], sc[1], sc[2], sc[3]
+            out.append(q)
+        return out
+    finally:
+        lib().qlstm_quantized_destroy(h)
