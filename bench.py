@@ -94,17 +94,17 @@ class ClockSampler:
         return out
 
 
-# DRAM traffic of the recurrent kernel from one ncu capture (its summary is kept with the other profile summaries):
-# dram__bytes_read.sum + dram__bytes_write.sum = 176.03 + 10.54 MB for 40 steps of config 5 at batch 256; per-step
-# traffic is steady, so a launch of T steps moves T / 40 of that.  Valid only for the kernel sources the counters
-# were taken from: if they changed since, the figure is reported as null.
-NCU_RECURRENT = {"bytes": 186.57e6, "steps": 40, "config": 5, "batch": 256, "source_sha": "984460bfd146d3a8"}
+# DRAM traffic of the recurrent kernel from one ncu capture of full-size launches (three counters, one pass; its
+# summary is kept with the other profile summaries): dram__bytes_read.sum + dram__bytes_write.sum = 1268.2 + 52.8 MB
+# per launch (one layer, 300 steps) of config 5 at batch 256, against 1309.9 MB algorithmic (X read once, y written
+# once).  Valid only for the kernel sources the counters were taken from and for that launch shape: otherwise null.
+NCU_RECURRENT = {"bytes": 1321.0e6, "steps": 300, "config": 5, "batch": 256, "source_sha": "8994fd47a7cbb38f"}
 
 # DRAM traffic of the input-projection kernel from one ncu capture of a full-size launch (three counters, one pass):
-# dram__bytes_read.sum + dram__bytes_write.sum = 54.7 + 1203.9 MB at 76800 rows of config 5 (algorithmic: 49.2 MB of x,
+# dram__bytes_read.sum + dram__bytes_write.sum = 54.5 + 1203.9 MB at 76800 rows of config 5 (algorithmic: 49.2 MB of x,
 # 5.2 MB of W, 1258.3 MB of int16 output, part of which is still in L2 when the kernel ends).  Valid only for the
 # kernel sources the counters were taken from and for that launch shape: otherwise reported as null.
-NCU_PROJECTION = {"bytes": 1258.6e6, "rows": 76800, "config": 5, "source_sha": "7a742f3e6e59208d"}
+NCU_PROJECTION = {"bytes": 1258.4e6, "rows": 76800, "config": 5, "source_sha": "47d47edcf24a8e15"}
 
 # The recurrent kernel is bound by plain integer arithmetic (the fixed-point epilogues), not by its matmuls or by
 # memory.  Peak: 148 SMs x 64 int32 lanes (4 schedulers x 16-lane integer pipe) x the SM clock; a microbenchmark of
@@ -379,9 +379,9 @@ def main():
                                             ("phase_a_ms", "matmul_a_ms", "wait_a_ms", "phase_b_ms", "wait_b_ms", "phase_c_ms", "wait_c_ms")},
                 "phase_note": "separate pass with the device phase timers on (they slow the kernel: "
                               f"{1e3 * prof_phase['recurrent_ms'] / (n_l * T):.2f} us per layer-step in that pass)"}
-    if (args.config == NCU_RECURRENT["config"] and B == NCU_RECURRENT["batch"]
+    if (args.config == NCU_RECURRENT["config"] and B == NCU_RECURRENT["batch"] and T == NCU_RECURRENT["steps"]
             and recurrent_source_sha() == NCU_RECURRENT["source_sha"]):
-        roof_rec["traffic"] = NCU_RECURRENT["bytes"] * T / NCU_RECURRENT["steps"]      # bytes per launch (one layer)
+        roof_rec["traffic"] = NCU_RECURRENT["bytes"]                                     # bytes per launch (one layer)
     # algorithmic HBM bytes of the recurrent kernel per launch: X read once, y written once, state in and out
     roof_rec["algorithmic_hbm_bytes"] = rec_bytes
     dominant = roof_rec if rec_ms >= proj_ms else roof_proj
