@@ -1,4 +1,4 @@
-// Whole-stack kernel for small batches (B <= 4): every layer and every time step in ONE cooperative launch.
+// Whole-stack kernel for small batches (up to 16 rows): every layer and every time step in ONE cooperative launch.
 //
 // At batch 1..4 a layer-step is a handful of mat-vec products, far too small to fill the machine, and a stack run layer
 // after layer leaves all but one layer's worth of work idle.  Here the blocks are split into one group per layer and
