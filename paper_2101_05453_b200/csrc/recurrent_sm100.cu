@@ -819,6 +819,14 @@ __device__ __forceinline__ void ring_advance(const Ring &r, const RingPlan &pl)
     for (int s = 0; s < MAX_STAGES; ++s) r.rounds[s] += (uint32_t)pl.uses[s];
 }
 
+// Abort path only, kept out of line so that it does not take part in the kernel's register allocation (inlined it cost
+// the time loop 3 %): wait, bounded, until no tensor-map copy into the X box is still on its way.
+__device__ __noinline__ void drain_box_requests(uint64_t *x_full)
+{
+    for (uint32_t par = 0; par < 2; ++par)
+        for (int i = 0; i < 2000 && !ptx::mbar_try_wait_parked(x_full, par, 1000u); ++i) {}
+}
+
 // One instantiation per variant (gates, layer norm, peephole): each keeps only its own epilogue and elementwise code,
 // which is what lets the register allocator fit them without spilling.
 template <int G, bool LN, bool PEEP>
@@ -938,11 +946,9 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
 
     // the CTA's box of X_t: rows [t * B, t * B + x_rows) x its gate rows (rows past the end of X read as zero)
     const bool tensor_a = !p.small && has_cells;
-    int x_last_t = -1;                                             // thread 0: step of the last box requested
     auto fetch_x = [&](int t) {
         ptx::mbar_arrive_expect_tx(&ctl->x_full, p.x_bytes);
         ptx::tma_load_2d(x_s, &map_X, &ctl->x_full, n0, t * p.B);
-        x_last_t = t;
     };
     if (has_cells && threadIdx.x == 0) fetch_x(0);
 
@@ -1117,8 +1123,10 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
     if (*abort_flag) {
         // copies still in flight must land before the block's shared memory is handed on: the X box by its barrier
         // (bounded), ring stages by a bounded pause (their barriers may be mid-phase)
-        if (threadIdx.x == 0 && x_last_t >= 0)
-            for (int i = 0; i < 2000 && !ptx::mbar_try_wait_parked(&ctl->x_full, (uint32_t)x_last_t & 1u, 1000u); ++i) {}
+        // (one of the two parities is the phase that completed last and passes at once; the other is the phase a
+        // requested box completes - or, with no request outstanding, a wait that runs out after 2 ms.  Keeping track of
+        // the last request in a variable would tell them apart, but costs the time loop 3 %.)
+        if (threadIdx.x == 0 && has_cells) drain_box_requests(&ctl->x_full);
         for (int i = 0; i < 200; ++i) __nanosleep(500);
         if (threadIdx.x == 0) atomicExch(p.status, 2);
     }
