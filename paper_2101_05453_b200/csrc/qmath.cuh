@@ -39,6 +39,21 @@ QL_HD int32_t mbqm(int32_t x, Scale s)
     return p < 0 ? -(int32_t)q : (int32_t)q;
 }
 
+// Rarely taken paths of the hot loops (a scale with a left shift; a layer-norm quotient beyond 16 bits), out of line
+// on the device so that they stay out of those loops' register budget.
+#if defined(__CUDACC__)
+static __device__ __noinline__ int32_t mbqm_rare(int32_t x, Scale s) { return mbqm(x, s); }
+static __device__ __noinline__ uint64_t div_rare(uint64_t n, uint32_t d) { return n / d; }
+#endif
+QL_HD int32_t mbqm_cold(int32_t x, Scale s)
+{
+#if defined(__CUDA_ARCH__)
+    return mbqm_rare(x, s);
+#else
+    return mbqm(x, s);
+#endif
+}
+
 // The same rescale for shift <= 0 with its constants pre-computed, in 32-bit registers:
 //   round(round(|x| M / 2^31) / 2^R) = floor((2 |x| M + 2^31 + [R>0] 2^(31+R)) / 2^(32+R))
 // (nested floors collapse), i.e. the high word of one 32x32+64 multiply-add, shifted right by R.
@@ -221,7 +236,11 @@ QL_HD int64_t ln_scaled_fast(int32_t q, const LnRow &r, int32_t L, int32_t b)   
         const int32_t qp = d < 0 ? -(int32_t)qe : (int32_t)qe;
         return (int64_t)qp * L + b;                                // one 32 x 32 + 64 multiply-add
     }
+#if defined(__CUDA_ARCH__)
+    const uint64_t quo = r.sigma ? div_rare((uint64_t)ad * 1024u + half, r.sigma) : 0u;
+#else
     const uint64_t quo = r.sigma ? ((uint64_t)ad * 1024u + half) / r.sigma : 0u;
+#endif
     return (d < 0 ? -(int64_t)quo : (int64_t)quo) * (int64_t)L + (int64_t)b;
 }
 
@@ -236,7 +255,7 @@ QL_HD int32_t sat32_halves(int64_t v)              // saturate through the two 3
 QL_HD int32_t ln_apply_fast(int32_t q, const LnRow &r, int32_t L, int32_t b, Scale eff_ln, const FastScale &f_ln)
 {
     const int32_t v32 = sat32_halves(ln_scaled_fast(q, r, L, b));
-    return sat16(eff_ln.shift <= 0 ? fast_rescale(v32, f_ln) : mbqm(v32, eff_ln));
+    return sat16(eff_ln.shift <= 0 ? fast_rescale(v32, f_ln) : mbqm_cold(v32, eff_ln));
 }
 
 // ---- cell update and hidden state (Section 3.2.7) -------------------------------------------
@@ -252,7 +271,7 @@ QL_HD int32_t cell_update_fast(int32_t i, int32_t z, int32_t f, int32_t c_old, i
 QL_HD int32_t hidden_q_fast(int32_t o, int32_t c_new, int m, Scale eff_m, const FastScale &f_m, int32_t zp_m)
 {
     int32_t prod = o * tanh_q_fast(c_new, m);
-    return sat8((eff_m.shift <= 0 ? fast_rescale(prod, f_m) : mbqm(prod, eff_m)) + zp_m);
+    return sat8((eff_m.shift <= 0 ? fast_rescale(prod, f_m) : mbqm_cold(prod, eff_m)) + zp_m);
 }
 
 }  // namespace ql

@@ -168,11 +168,11 @@ __device__ __forceinline__ void grid_sync(const RecParams &p, unsigned &epoch, v
 
 __device__ __forceinline__ int32_t rescale_sel(int32_t x, const Scale &s, const FastScale &f, int fast_ok)
 {
-    return fast_ok ? fast_rescale(x, f) : mbqm(x, s);
+    return fast_ok ? fast_rescale(x, f) : mbqm_cold(x, s);
 }
 __device__ __forceinline__ int32_t rescale_any(int32_t x, const Scale &s, const FastScale &f)
 {
-    return s.shift <= 0 ? fast_rescale(x, f) : mbqm(x, s);
+    return s.shift <= 0 ? fast_rescale(x, f) : mbqm_cold(x, s);
 }
 
 // ------------------------------------------------------------------------------------------------
