@@ -75,8 +75,9 @@ int stack_small_create(const std::vector<const LayerParams *> &layers, int max_T
 void stack_small_destroy(StackSmall *s);
 bool stack_small_supported(const StackSmall *s, int T, int B);
 bool stack_small_preferred(const StackSmall *s, int T, int B);     // supported and, by measurement, the faster path
-// schedule: 0 automatic, 1 wavefront (one group of blocks per layer), 2 sequential (every layer on all blocks)
-int launch_stack_small(const StackSmall *s, const int8_t *x, int T, int B, int8_t *h, int16_t *c, int8_t *y, int *status,
+// schedule: 0 automatic, 1 wavefront (one group of blocks per layer), 2 sequential (every layer on all blocks).
+// The kernel clears the status word itself.
+int launch_stack_small(StackSmall *s, const int8_t *x, int T, int B, int8_t *h, int16_t *c, int8_t *y, int *status,
                        int schedule, cudaStream_t st);
 void stack_small_debug_timeout(StackSmall *s, unsigned missing_arrivals, unsigned long long limit_ns);
 int stack_small_groups(const StackSmall *s, int *blocks_per_layer);     // layers, and the blocks each layer's group has

@@ -365,8 +365,6 @@ int qlstm_run(qlstm_t *q, const int8_t *x_dev, int T, int B, int8_t *h_dev, int1
     q->last_stream = st;
     uint8_t *trace = (uint8_t *)trace_dev;
     if (trace && cudaMemsetAsync(trace, 0, qlstm_trace_bytes(q, T, B), st) != cudaSuccess) return QLSTM_ERR_CUDA;
-    if (cudaMemsetAsync(q->status, 0, 4 * sizeof(int), st) != cudaSuccess) return QLSTM_ERR_CUDA;
-
     const int nl = (int)q->layers.size();
     // small batches: the whole stack in one launch (layers as a wavefront, input projection inside the step)
     if (!trace && (q->impl_rec == 0 || q->impl_rec >= 5) && q->impl_proj != 1) {
@@ -381,6 +379,7 @@ int qlstm_run(qlstm_t *q, const int8_t *x_dev, int T, int B, int8_t *h_dev, int1
     } else if (q->impl_rec >= 5) {
         return QLSTM_ERR_ARG;
     }
+    if (cudaMemsetAsync(q->status, 0, 4 * sizeof(int), st) != cudaSuccess) return QLSTM_ERR_CUDA;
     const int8_t *in = x_dev;
     size_t h_off = 0, c_off = 0;
     for (int l = 0; l < nl; ++l) {

@@ -65,6 +65,8 @@ struct SkCall {
     int8_t *y;                     // [T][B][O_last]
     unsigned *cnt;                 // [n_layers][CNT_PER_LAYER] counters, zero at launch
     unsigned *abort_word;
+    unsigned *cnt_next;            // the other set of counters (and abort word): cleared by this call for the next one
+    int cnt_words;
     int *status;
     unsigned long long wait_limit_ns;
     unsigned missing_arrivals;     // 0; a test makes every counter wait for arrivals that never come
@@ -136,7 +138,7 @@ __device__ __forceinline__ bool sk_wait(const SkCall &k, const unsigned *cnt, un
 // that divides the number of 16-byte chunks of a row, so that every lane takes the same number of chunks CPL).
 // A warp keeps the weight loads of two rows per lane in flight (R2): the loop is bound by the latency of those loads
 // and by the shared-memory reads of the vectors, which the two rows share.
-template <int NB, int CPL, bool R2, class F>
+template <int NB, int CPL, bool R2, bool VG, class F>
 __device__ __forceinline__ void matvec_rows_t(const int8_t *rows, int nrows, int K, int gs, const int8_t *vec_s, F emit)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -155,16 +157,25 @@ __device__ __forceinline__ void matvec_rows_t(const int8_t *rows, int nrows, int
 #pragma unroll
             for (int j = 0; j < CPL; ++j) w[q][j] = valid[q] ? ld_stream(wp + j * gs) : make_uint4(0, 0, 0, 0);   // all loads in flight
         }
+        // VG: the vectors are read straight from global memory (L2: other blocks wrote them this step), their loads in
+        // flight together with the weights' - at one batch row this saves the round trip of staging them first
+        uint4 vg[VG ? CPL : 1][VG ? NB : 1];
+        if (VG) {
+#pragma unroll
+            for (int j = 0; j < CPL; ++j)
+#pragma unroll
+                for (int b = 0; b < NB; ++b) vg[VG ? j : 0][VG ? b : 0] = __ldcg(reinterpret_cast<const uint4 *>(vec_s + (size_t)b * K) + lg + j * gs);
+        }
 #pragma unroll
         for (int q = 0; q < NR; ++q)
 #pragma unroll
             for (int b = 0; b < NB; ++b) acc[q][b] = 0;
-        // every vector chunk is read from shared memory once and used for both rows
+        // every vector chunk is read once and used for both rows
 #pragma unroll
         for (int j = 0; j < CPL; ++j) {
 #pragma unroll
             for (int b = 0; b < NB; ++b) {
-                const uint4 v = reinterpret_cast<const uint4 *>(vec_s + (size_t)b * K)[lg + j * gs];
+                const uint4 v = VG ? vg[VG ? j : 0][VG ? b : 0] : reinterpret_cast<const uint4 *>(vec_s + (size_t)b * K)[lg + j * gs];
 #pragma unroll
                 for (int q = 0; q < NR; ++q) {
                     acc[q][b] = __dp4a((int)w[q][j].x, (int)v.x, acc[q][b]);
@@ -192,7 +203,7 @@ __device__ __forceinline__ void matvec_rows_t(const int8_t *rows, int nrows, int
 }
 
 // any number of chunks per lane: one load at a time, four trips unrolled
-template <int NB, class F>
+template <int NB, bool VG, class F>
 __device__ __forceinline__ void matvec_rows_any(const int8_t *rows, int nrows, int K, int gs, const int8_t *vec_s, F emit)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -211,7 +222,8 @@ __device__ __forceinline__ void matvec_rows_any(const int8_t *rows, int nrows, i
                 const uint4 w = ld_stream(wp + j * gs);
 #pragma unroll
                 for (int b = 0; b < NB; ++b) {
-                    const uint4 v = reinterpret_cast<const uint4 *>(vec_s + (size_t)b * K)[lg + j * gs];
+                    const uint4 *vp = reinterpret_cast<const uint4 *>(vec_s + (size_t)b * K) + lg + j * gs;
+                    const uint4 v = VG ? __ldcg(vp) : *vp;
                     acc[b] = __dp4a((int)w.x, (int)v.x, acc[b]);
                     acc[b] = __dp4a((int)w.y, (int)v.y, acc[b]);
                     acc[b] = __dp4a((int)w.z, (int)v.z, acc[b]);
@@ -240,20 +252,6 @@ __host__ __device__ inline int lanes_per_row(int K)
     return gs;
 }
 
-template <int NB, class F>
-__device__ __forceinline__ void matvec_rows(const int8_t *rows, int nrows, int K, const int8_t *vec_s, F emit)
-{
-    const int gs = lanes_per_row(K);
-    constexpr bool R2 = NB <= 8;             // sixteen batch rows: the accumulators of two rows would not fit in registers
-    switch ((K >> 4) / gs) {
-        case 1: matvec_rows_t<NB, 1, R2>(rows, nrows, K, gs, vec_s, emit); break;
-        case 2: matvec_rows_t<NB, 2, R2>(rows, nrows, K, gs, vec_s, emit); break;
-        case 4: matvec_rows_t<NB, 4, R2>(rows, nrows, K, gs, vec_s, emit); break;
-        case 5: matvec_rows_t<NB, 5, R2>(rows, nrows, K, gs, vec_s, emit); break;
-        default: matvec_rows_any<NB>(rows, nrows, K, gs, vec_s, emit); break;
-    }
-}
-
 // [B][K] bytes from global memory written by other blocks (L2 loads) into shared memory as [NB][K], rows >= B zero
 __device__ __forceinline__ void stage_vec(int8_t *dst_s, const int8_t *src, int B, int NB, int K)
 {
@@ -271,6 +269,36 @@ __device__ __forceinline__ void stage_vec_bytes(int8_t *dst_s, const int8_t *src
     for (int i = threadIdx.x; i < NB * K; i += SK_THREADS) dst_s[i] = (i < B * K) ? src[i] : (int8_t)0;
 }
 
+template <int NB, bool VG, class F>
+__device__ __forceinline__ void matvec_rows(const int8_t *rows, int nrows, int K, const int8_t *vec, F emit)
+{
+    const int gs = lanes_per_row(K);
+    constexpr bool R2 = NB <= 8;             // sixteen batch rows: the accumulators of two rows would not fit in registers
+    switch ((K >> 4) / gs) {
+        case 1: matvec_rows_t<NB, 1, R2, VG>(rows, nrows, K, gs, vec, emit); break;
+        case 2: matvec_rows_t<NB, 2, R2, VG>(rows, nrows, K, gs, vec, emit); break;
+        case 4: matvec_rows_t<NB, 4, R2, VG>(rows, nrows, K, gs, vec, emit); break;
+        case 5: matvec_rows_t<NB, 5, R2, VG>(rows, nrows, K, gs, vec, emit); break;
+        default: matvec_rows_any<NB, VG>(rows, nrows, K, gs, vec, emit); break;
+    }
+}
+
+// The B vectors of a mat-vec, [B][K] int8 in global memory.  With one batch row they are read in place (when 16-byte
+// aligned); otherwise they are staged in shared memory first, rows >= B zero.
+template <int NB, class F>
+__device__ __forceinline__ void matvec_with(const int8_t *rows, int nrows, int K, const int8_t *vec_g, int B, int8_t *stage_s,
+                                            bool written_by_other_blocks, F emit)
+{
+    if (NB == 1 && (((uintptr_t)vec_g) & 15) == 0) {
+        matvec_rows<NB, true>(rows, nrows, K, vec_g, emit);
+        return;
+    }
+    if (written_by_other_blocks) stage_vec(stage_s, vec_g, B, NB, K);
+    else stage_vec_bytes(stage_s, vec_g, B, NB, K);
+    __syncthreads();
+    matvec_rows<NB, false>(rows, nrows, K, stage_s, emit);
+}
+
 // What a block does for one layer: its share of the cells and of the projection rows, and where things live.
 struct Role {
     const SkLayer *L;              // shared memory
@@ -278,6 +306,10 @@ struct Role {
     int u0, cells, npc, n0, n_cnt; // own cells and gate rows
     int p_lo, p_cnt;               // own projection rows
     int16_t *c_s;                  // [NB][cpc] cell state, resident over the call
+    // per-row constants of the block's own rows, copied to shared memory once (a global load inside every epilogue
+    // would be one more round trip in each step's chain): indexed by the local gate row / projection row
+    const int32_t *bx, *bh, *bln, *bp;
+    const int16_t *Lw, *Pw;
     unsigned *cnt;                 // the layer's counters
     const unsigned *cnt_below;     // CNT_H of the layer below, or null
     unsigned n_below;
@@ -301,11 +333,9 @@ template <int NB>
 __device__ __forceinline__ void input_term(const SkCall &k, const Role &r, const SkSmem &s, int t)
 {
     const SkLayer &L = *r.L;
-    stage_vec(s.x_s, r.in_seq + (size_t)t * k.B * L.I, k.B, NB, L.I);
-    __syncthreads();
     const int B = k.B, npc = r.npc, n0 = r.n0, G = L.G;
-    matvec_rows<NB>(L.W + (size_t)n0 * L.I, r.n_cnt, L.I, s.x_s, [&](int n, int b, int32_t acc) {
-        if (b < B) s.xs_s[b * npc + n] = (int16_t)sat16(sk_rescale(acc + L.bx[n0 + n], L.eff_x[n % G]));
+    matvec_with<NB>(L.W + (size_t)n0 * L.I, r.n_cnt, L.I, r.in_seq + (size_t)t * B * L.I, B, s.x_s, true, [&](int n, int b, int32_t acc) {
+        if (b < B) s.xs_s[b * npc + n] = (int16_t)sat16(sk_rescale(acc + r.bx[n], L.eff_x[n % G]));
     });
 }
 
@@ -315,12 +345,10 @@ template <int NB>
 __device__ __forceinline__ void recurrent_term(const SkCall &k, const Role &r, const SkSmem &s, int t)
 {
     const SkLayer &L = *r.L;
-    if (t == 0) stage_vec_bytes(s.h_s, r.h_state, k.B, NB, L.O);
-    else stage_vec(s.h_s, r.out_seq + (size_t)(t - 1) * k.B * L.O, k.B, NB, L.O);
-    __syncthreads();
     const int B = k.B, npc = r.npc, n0 = r.n0, G = L.G;
-    matvec_rows<NB>(L.R + (size_t)n0 * L.O, r.n_cnt, L.O, s.h_s, [&](int n, int b, int32_t acc) {
-        if (b < B) s.hs_s[b * npc + n] = (int16_t)sat16(sk_rescale(sk_add_sat(acc, L.bh[n0 + n]), L.eff_h[n % G]));
+    const int8_t *h_prev = t == 0 ? r.h_state : r.out_seq + (size_t)(t - 1) * B * L.O;
+    matvec_with<NB>(L.R + (size_t)n0 * L.O, r.n_cnt, L.O, h_prev, B, s.h_s, t != 0, [&](int n, int b, int32_t acc) {
+        if (b < B) s.hs_s[b * npc + n] = (int16_t)sat16(sk_rescale(sk_add_sat(acc, r.bh[n]), L.eff_h[n % G]));
     });
 }
 
@@ -384,7 +412,7 @@ __device__ __forceinline__ bool finish_step(const SkCall &k, const Role &r, cons
         const int b = i / r.n_cnt, n = i - b * r.n_cnt, gi = n % G, ul = n / G;
         int32_t v = (int32_t)s.xs_s[b * npc + n] + (int32_t)s.hs_s[b * npc + n];
         if (peep && gi == SO) continue;
-        if (peep && gi != SZ) v += sat16(sk_rescale((int32_t)L.P[n0 + n] * r.c_s[b * cpc + ul], L.eff_c[gi]));
+        if (peep && gi != SZ) v += sat16(sk_rescale((int32_t)r.Pw[n] * r.c_s[b * cpc + ul], L.eff_c[gi]));
         s.pre_s[b * npc + n] = (int16_t)sat16(v);
     }
     __syncthreads();
@@ -392,60 +420,107 @@ __device__ __forceinline__ bool finish_step(const SkCall &k, const Role &r, cons
         const unsigned all = (1u << G) - 1u;
         if (!exchange_stats(k, r, s, 0, peep ? (all & ~(1u << SO)) : all, r.cnt + CNT_A, (unsigned)(t + 1) * n_grp, abort_s)) return false;
     }
-    // elementwise, one cell per thread
-    for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
-        const int b = i / cells, ul = i - b * cells;
-        const int nl = ul * G, n = n0 + nl;
-        const int16_t *pre = s.pre_s + b * npc + nl;
-        const LnRow *lr = s.ln_s + b * 4;
-        // input of the nonlinearity of gate slot g: the gate sum, after layer norm when the layer has it
-        auto gate_in = [&](int g) -> int32_t {
-            const int32_t v = pre[g];
-            return ln ? ln_apply_fast(v, lr[g], L.L[n + g], L.bln[n + g], L.eff_ln[g], make_fast_scale(L.eff_ln[g])) : v;
+    const bool quad = B * cells * 4 <= SK_THREADS;
+    if (quad) {
+        // Few cells (one or two batch rows): four lanes per cell, one gate each, so that the cell's five nonlinearities
+        // are not one thread's serial chain.  Lane j takes gate slot j (layer norm + sigmoid / tanh), the group exchanges
+        // the gate values with shuffles, every lane forms c^t, then the output gate's lane and the update gate's lane
+        // compute sigmoid(o) and tanh(c^t) side by side and lane 0 forms the hidden state.
+        const int task_i = threadIdx.x >> 2, j = threadIdx.x & 3, base = (threadIdx.x & 31) & ~3;
+        const bool task = task_i < B * cells;
+        const int b = task ? task_i / cells : 0, ul = task ? task_i - b * cells : 0;
+        const int nl = ul * G;
+        const bool mine = task && j < G;                           // this lane has a gate
+        auto gate_in_of = [&](int g) -> int32_t {
+            const int32_t v = s.pre_s[b * npc + nl + g];
+            return ln ? ln_apply_fast(v, s.ln_s[b * 4 + g], r.Lw[nl + g], r.bln[nl + g], L.eff_ln[g], make_fast_scale(L.eff_ln[g])) : v;
         };
-        const int32_t f = sigmoid_q_fast(gate_in(SF), 3), z = tanh_q_fast(gate_in(SZ), 3);
-        int32_t ig;
-        if (G == 4) ig = sigmoid_q_fast(gate_in(0), 3);
-        else { ig = 32768 - f; if (ig > 32767) ig = 32767; }    // coupled input gate, Section 3.2.9
-        const int32_t c_old = r.c_s[b * cpc + ul];
-        const int32_t c_new = cell_update_fast(ig, z, f, c_old, L.m_bits);
-        r.c_s[b * cpc + ul] = (int16_t)c_new;
-        int32_t ao;
-        if (peep) {
-            ao = sat16((int32_t)s.xs_s[b * npc + nl + SO] + (int32_t)s.hs_s[b * npc + nl + SO] +
-                       sat16(sk_rescale((int32_t)L.P[n + SO] * c_new, L.eff_c[SO])));
-            if (ln) { s.pre_s[b * npc + nl + SO] = (int16_t)ao; continue; }      // waits for the row's statistics
-        } else {
-            ao = gate_in(SO);
+        int32_t val = 0;
+        if (mine && !(peep && j == SO)) {
+            const int32_t v = gate_in_of(j);
+            val = (j == SZ) ? tanh_q_fast(v, 3) : sigmoid_q_fast(v, 3);
         }
-        const int32_t mq = hidden_q_fast(sigmoid_q_fast(ao, 3), c_new, L.m_bits, L.eff_m, make_fast_scale(L.eff_m), L.zp_m);
-        if (proj) L.m[(size_t)b * C + u0 + ul] = (int8_t)mq;
-        else r.out_seq[((size_t)t * B + b) * O + u0 + ul] = (int8_t)mq;
-    }
-    if (ln && peep) {
-        __syncthreads();
-        if (!exchange_stats(k, r, s, 1, 1u << SO, r.cnt + CNT_A2, (unsigned)(t + 1) * n_grp, abort_s)) return false;
-        for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
-            const int b = i / cells, ul = i - b * cells;
-            const int n = n0 + ul * G + SO;
-            const int32_t ao = ln_apply_fast(s.pre_s[b * npc + ul * G + SO], s.ln_s[b * 4 + SO], L.L[n], L.bln[n], L.eff_ln[SO],
-                                             make_fast_scale(L.eff_ln[SO]));
-            const int32_t mq = hidden_q_fast(sigmoid_q_fast(ao, 3), r.c_s[b * cpc + ul], L.m_bits, L.eff_m,
-                                             make_fast_scale(L.eff_m), L.zp_m);
+        const int32_t f = __shfl_sync(0xffffffffu, val, base + SF), z = __shfl_sync(0xffffffffu, val, base + SZ);
+        int32_t ig = __shfl_sync(0xffffffffu, val, base);
+        int32_t o = __shfl_sync(0xffffffffu, val, base + SO);
+        if (G != 4) { ig = 32768 - f; if (ig > 32767) ig = 32767; }  // coupled input gate, Section 3.2.9
+        const int32_t c_old = task ? r.c_s[b * cpc + ul] : 0;
+        const int32_t c_new = cell_update_fast(ig, z, f, c_old, L.m_bits);
+        __syncwarp();
+        if (task && j == 0) r.c_s[b * cpc + ul] = (int16_t)c_new;
+        if (peep && task && j == SO) {
+            const int32_t ao = sat16((int32_t)s.xs_s[b * npc + nl + SO] + (int32_t)s.hs_s[b * npc + nl + SO] +
+                                     sat16(sk_rescale((int32_t)r.Pw[nl + SO] * c_new, L.eff_c[SO])));
+            if (ln) s.pre_s[b * npc + nl + SO] = (int16_t)ao;     // waits for the row's statistics
+            else val = sigmoid_q_fast(ao, 3);
+        }
+        if (ln && peep) {
+            __syncthreads();
+            if (!exchange_stats(k, r, s, 1, 1u << SO, r.cnt + CNT_A2, (unsigned)(t + 1) * n_grp, abort_s)) return false;
+            if (task && j == SO) val = sigmoid_q_fast(gate_in_of(SO), 3);
+        }
+        if (peep) o = __shfl_sync(0xffffffffu, val, base + SO);
+        int32_t tc = (task && j == SZ) ? tanh_q_fast(c_new, L.m_bits) : 0;
+        tc = __shfl_sync(0xffffffffu, tc, base + SZ);
+        if (task && j == 0) {
+            const int32_t mq = sat8(sk_rescale(o * tc, L.eff_m) + L.zp_m);              // Section 3.2.7
             if (proj) L.m[(size_t)b * C + u0 + ul] = (int8_t)mq;
             else r.out_seq[((size_t)t * B + b) * O + u0 + ul] = (int8_t)mq;
+        }
+    } else {
+        // elementwise, one cell per thread
+        for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
+            const int b = i / cells, ul = i - b * cells;
+            const int nl = ul * G;
+            const int16_t *pre = s.pre_s + b * npc + nl;
+            const LnRow *lr = s.ln_s + b * 4;
+            // input of the nonlinearity of gate slot g: the gate sum, after layer norm when the layer has it
+            auto gate_in = [&](int g) -> int32_t {
+                const int32_t v = pre[g];
+                return ln ? ln_apply_fast(v, lr[g], r.Lw[nl + g], r.bln[nl + g], L.eff_ln[g], make_fast_scale(L.eff_ln[g])) : v;
+            };
+            const int32_t f = sigmoid_q_fast(gate_in(SF), 3), z = tanh_q_fast(gate_in(SZ), 3);
+            int32_t ig;
+            if (G == 4) ig = sigmoid_q_fast(gate_in(0), 3);
+            else { ig = 32768 - f; if (ig > 32767) ig = 32767; }    // coupled input gate, Section 3.2.9
+            const int32_t c_old = r.c_s[b * cpc + ul];
+            const int32_t c_new = cell_update_fast(ig, z, f, c_old, L.m_bits);
+            r.c_s[b * cpc + ul] = (int16_t)c_new;
+            int32_t ao;
+            if (peep) {
+                ao = sat16((int32_t)s.xs_s[b * npc + nl + SO] + (int32_t)s.hs_s[b * npc + nl + SO] +
+                           sat16(sk_rescale((int32_t)r.Pw[nl + SO] * c_new, L.eff_c[SO])));
+                if (ln) { s.pre_s[b * npc + nl + SO] = (int16_t)ao; continue; }      // waits for the row's statistics
+            } else {
+                ao = gate_in(SO);
+            }
+            const int32_t mq = hidden_q_fast(sigmoid_q_fast(ao, 3), c_new, L.m_bits, L.eff_m, make_fast_scale(L.eff_m), L.zp_m);
+            if (proj) L.m[(size_t)b * C + u0 + ul] = (int8_t)mq;
+            else r.out_seq[((size_t)t * B + b) * O + u0 + ul] = (int8_t)mq;
+        }
+        if (ln && peep) {
+            __syncthreads();
+            if (!exchange_stats(k, r, s, 1, 1u << SO, r.cnt + CNT_A2, (unsigned)(t + 1) * n_grp, abort_s)) return false;
+            for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
+                const int b = i / cells, ul = i - b * cells;
+                const int n = n0 + ul * G + SO;
+                const int32_t ao = ln_apply_fast(s.pre_s[b * npc + ul * G + SO], s.ln_s[b * 4 + SO], r.Lw[n], r.bln[n], L.eff_ln[SO],
+                                                 make_fast_scale(L.eff_ln[SO]));
+                const int32_t mq = hidden_q_fast(sigmoid_q_fast(ao, 3), r.c_s[b * cpc + ul], L.m_bits, L.eff_m,
+                                                 make_fast_scale(L.eff_m), L.zp_m);
+                if (proj) L.m[(size_t)b * C + u0 + ul] = (int8_t)mq;
+                else r.out_seq[((size_t)t * B + b) * O + u0 + ul] = (int8_t)mq;
+            }
         }
     }
     // projection (Section 3.2.8): needs every m of the layer
     if (proj) {
         sk_arrive(r.cnt + CNT_M);
         if (!sk_wait(k, r.cnt + CNT_M, (unsigned)(t + 1) * n_grp, abort_s)) return false;
-        stage_vec(s.m_s, L.m, B, NB, C);
-        __syncthreads();
         const int p_lo = r.p_lo;
         int8_t *out = r.out_seq + (size_t)t * B * O;
-        matvec_rows<NB>(L.Wproj + (size_t)p_lo * C, r.p_cnt, C, s.m_s, [&](int row, int b, int32_t acc) {
-            if (b < B) out[(size_t)b * O + p_lo + row] = (int8_t)sat8(sk_rescale(sk_add_sat(acc, L.bp[p_lo + row]), L.eff_proj) + L.zp_h);
+        matvec_with<NB>(L.Wproj + (size_t)p_lo * C, r.p_cnt, C, L.m, B, s.m_s, true, [&](int row, int b, int32_t acc) {
+            if (b < B) out[(size_t)b * O + p_lo + row] = (int8_t)sat8(sk_rescale(sk_add_sat(acc, r.bp[row]), L.eff_proj) + L.zp_h);
         });
     }
     // h^t is complete once every block of the group has arrived
@@ -453,7 +528,18 @@ __device__ __forceinline__ bool finish_step(const SkCall &k, const Role &r, cons
     return true;
 }
 
-__device__ __forceinline__ Role make_role(const SkCall &k, const SkLayer *Ls, int li, int rank, int16_t *c_s)
+// bytes a role keeps resident in shared memory: cell state [NB][cpc] int16, then bx, bh, bln [npc] int32, bp [rpc] int32,
+// L, P [npc] int16
+__host__ __device__ inline size_t role_bytes(int NB, int cpc, int G, int rpc)
+{
+    const size_t npc = (size_t)cpc * G;
+    return (((size_t)NB * cpc * 2 + 15) & ~(size_t)15) + npc * 12 + (((size_t)rpc * 4 + 15) & ~(size_t)15) + ((npc * 4 + 15) & ~(size_t)15);
+}
+
+// calls of at least this many steps keep the per-row constants of a block's rows in shared memory
+constexpr int SK_RESIDENT_MIN_T = 4;
+
+__device__ __forceinline__ Role make_role(const SkCall &k, const SkLayer *Ls, int li, int rank, uint8_t *region, int NB)
 {
     const SkLayer &L = Ls[li];
     Role r;
@@ -465,7 +551,24 @@ __device__ __forceinline__ Role make_role(const SkCall &k, const SkLayer *Ls, in
     r.p_lo = rank * L.rpc;
     r.p_cnt = (L.flags & F_PROJECTION) ? (L.O - r.p_lo < L.rpc ? L.O - r.p_lo : L.rpc) : 0;
     if (r.p_cnt < 0) r.p_cnt = 0;
-    r.c_s = c_s;
+    {
+        uint8_t *p = region;
+        r.c_s = (int16_t *)p;  p += ((size_t)NB * L.cpc * 2 + 15) & ~(size_t)15;
+        if (k.T >= SK_RESIDENT_MIN_T) {
+            r.bx = (const int32_t *)p;  p += (size_t)r.npc * 4;
+            r.bh = (const int32_t *)p;  p += (size_t)r.npc * 4;
+            r.bln = (const int32_t *)p; p += (size_t)r.npc * 4;
+            r.bp = (const int32_t *)p;  p += ((size_t)L.rpc * 4 + 15) & ~(size_t)15;
+            r.Lw = (const int16_t *)p;  p += (size_t)r.npc * 2;
+            r.Pw = (const int16_t *)p;
+        } else {                                               // a call of a few steps reads them where they are
+            r.bx = L.bx + r.n0; r.bh = L.bh + r.n0;
+            r.bln = L.bln ? L.bln + r.n0 : nullptr;
+            r.bp = L.bp ? L.bp + r.p_lo : nullptr;
+            r.Lw = L.L ? L.L + r.n0 : nullptr;
+            r.Pw = L.P ? L.P + r.n0 : nullptr;
+        }
+    }
     r.cnt = k.cnt + (size_t)li * CNT_PER_LAYER;
     r.cnt_below = li > 0 ? k.cnt + (size_t)(li - 1) * CNT_PER_LAYER + CNT_H : nullptr;
     r.n_below = li > 0 ? (unsigned)Ls[li - 1].n_cta : 0u;
@@ -474,6 +577,22 @@ __device__ __forceinline__ Role make_role(const SkCall &k, const SkLayer *Ls, in
     r.h_state = k.h + L.h_off * k.B;
     r.c_state = k.c + L.c_off * k.B;
     return r;
+}
+
+// all threads: the per-row constants of a role's own rows into its shared-memory region
+__device__ __forceinline__ void load_role_consts(const Role &r)
+{
+    const SkLayer &L = *r.L;
+    if (r.bx == L.bx + r.n0) return;                           // not resident for this call
+    const bool ln = (L.flags & F_LAYERNORM) != 0, peep = (L.flags & F_PEEPHOLE) != 0;
+    for (int n = threadIdx.x; n < r.n_cnt; n += SK_THREADS) {
+        const_cast<int32_t *>(r.bx)[n] = L.bx[r.n0 + n];
+        const_cast<int32_t *>(r.bh)[n] = L.bh[r.n0 + n];
+        const_cast<int32_t *>(r.bln)[n] = ln ? L.bln[r.n0 + n] : 0;
+        const_cast<int16_t *>(r.Lw)[n] = ln ? L.L[r.n0 + n] : (int16_t)0;
+        const_cast<int16_t *>(r.Pw)[n] = peep ? L.P[r.n0 + n] : (int16_t)0;
+    }
+    for (int q = threadIdx.x; q < r.p_cnt; q += SK_THREADS) const_cast<int32_t *>(r.bp)[q] = L.bp[r.p_lo + q];
 }
 
 // Two schedules, chosen by the host per call:
@@ -495,9 +614,15 @@ __global__ void __launch_bounds__(SK_THREADS, 1) k_stack_small(const SkLayer *__
     for (int i = threadIdx.x; i < (int)(nl * sizeof(SkLayer) / 4); i += SK_THREADS)
         reinterpret_cast<uint32_t *>(Ls)[i] = reinterpret_cast<const uint32_t *>(layers)[i];
     if (threadIdx.x == 0) abort_s = 0;
+    if (cta == 0) {
+        // calls alternate between two sets of counters; nothing in this call touches the other one, so it is cleared here
+        // for the next call (no memset launch per call: a one-step call is only a hundred-odd microseconds long)
+        for (int i = threadIdx.x; i < k.cnt_words; i += SK_THREADS) k.cnt_next[i] = 0u;
+        if (threadIdx.x == 0) *k.status = 0;
+    }
     __syncthreads();
     SkSmem s;
-    int16_t *c_base;
+    uint8_t *c_base;                                           // resident regions of the roles
     {
         uint8_t *p = sk_smem + (((size_t)nl * sizeof(SkLayer) + 15) & ~(size_t)15);
         s.x_s = (int8_t *)p;  p += (size_t)NB * k.max_I;
@@ -507,7 +632,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) k_stack_small(const SkLayer *__
         s.xs_s = (int16_t *)p; p += (size_t)NB * k.max_npc * 2;
         s.hs_s = (int16_t *)p; p += (size_t)NB * k.max_npc * 2;
         s.pre_s = (int16_t *)p; p += (size_t)NB * k.max_npc * 2;
-        c_base = (int16_t *)p;
+        c_base = (uint8_t *)(((uintptr_t)p + 15) & ~(uintptr_t)15);
     }
     bool ok = true;
 
@@ -516,7 +641,8 @@ __global__ void __launch_bounds__(SK_THREADS, 1) k_stack_small(const SkLayer *__
         for (int l = 0; l < nl; ++l)
             if (cta >= Ls[l].cta0 && cta < Ls[l].cta0 + Ls[l].n_cta) li = l;
         if (li < 0) return;                                    // spare block: takes no part in any counter
-        const Role r = make_role(k, Ls, li, cta - Ls[li].cta0, c_base);
+        const Role r = make_role(k, Ls, li, cta - Ls[li].cta0, c_base, NB);
+        load_role_consts(r);
         const unsigned n_grp = (unsigned)r.L->n_cta;
         for (int i = threadIdx.x; i < B * r.cells; i += SK_THREADS) {
             const int b = i / r.cells, ul = i - b * r.cells;
@@ -552,21 +678,22 @@ __global__ void __launch_bounds__(SK_THREADS, 1) k_stack_small(const SkLayer *__
         }
     } else {
         // cell states of this block's cells of every layer
-        int c_off = 0;
+        size_t c_off = 0;
         for (int l = 0; l < nl; ++l) {
-            const Role r = make_role(k, Ls, l, cta, c_base + c_off);
+            const Role r = make_role(k, Ls, l, cta, c_base + c_off, NB);
+            load_role_consts(r);
             for (int i = threadIdx.x; i < B * r.cells; i += SK_THREADS) {
                 const int b = i / r.cells, ul = i - b * r.cells;
                 r.c_s[b * r.L->cpc + ul] = r.c_state[(size_t)b * r.L->C + r.u0 + ul];
             }
-            c_off += NB * Ls[l].cpc;
+            c_off += role_bytes(NB, Ls[l].cpc, Ls[l].G, Ls[l].rpc);
         }
         __syncthreads();
         for (int t = 0; t < T && ok; ++t) {
             c_off = 0;
             for (int l = 0; l < nl && ok; ++l) {
-                const Role r = make_role(k, Ls, l, cta, c_base + c_off);
-                c_off += NB * Ls[l].cpc;
+                const Role r = make_role(k, Ls, l, cta, c_base + c_off, NB);
+                c_off += role_bytes(NB, Ls[l].cpc, Ls[l].G, Ls[l].rpc);
                 const unsigned n_grp = (unsigned)r.L->n_cta;
                 // this layer's own h^{t-1} (complete long ago for every layer but the last)
                 if (t > 0) ok = sk_wait(k, r.cnt + CNT_H, (unsigned)t * n_grp, &abort_s);
@@ -585,8 +712,8 @@ __global__ void __launch_bounds__(SK_THREADS, 1) k_stack_small(const SkLayer *__
         if (ok) {
             c_off = 0;
             for (int l = 0; l < nl; ++l) {
-                const Role r = make_role(k, Ls, l, cta, c_base + c_off);
-                c_off += NB * Ls[l].cpc;
+                const Role r = make_role(k, Ls, l, cta, c_base + c_off, NB);
+                c_off += role_bytes(NB, Ls[l].cpc, Ls[l].G, Ls[l].rpc);
                 for (int i = threadIdx.x; i < B * r.cells; i += SK_THREADS) {
                     const int b = i / r.cells, ul = i - b * r.cells;
                     r.c_state[(size_t)b * r.L->C + r.u0 + ul] = r.c_s[b * r.L->cpc + ul];
@@ -614,8 +741,9 @@ struct StackSmall {
     std::vector<SkLayer> plan[2];
     int max_I = 0, max_O = 0, max_C_proj = 0, max_npc = 0;
     std::vector<void *> owned;
-    unsigned *cnt = nullptr;       // counters + abort word
-    size_t cnt_words = 0;
+    unsigned *cnt = nullptr;       // two sets of counters + abort word, used by alternate calls
+    size_t cnt_words = 0;          // words of one set
+    unsigned calls = 0;
     unsigned dbg_missing = 0;
     unsigned long long dbg_limit_ns = 0;
 };
@@ -645,9 +773,9 @@ static size_t sk_smem_bytes(const StackSmall &s, int NB)
     size_t common = (((size_t)s.n_layers * sizeof(SkLayer) + 15) & ~(size_t)15) + (size_t)NB * (s.max_I + s.max_O + s.max_C_proj) +
                     (size_t)NB * 4 * sizeof(LnRow) + 3 * (size_t)NB * s.max_npc * 2;
     size_t c_wave = 0, c_seq = 0;
-    for (const SkLayer &L : s.plan[0]) c_wave = std::max(c_wave, (size_t)NB * L.cpc * 2);
-    for (const SkLayer &L : s.plan[1]) c_seq += (size_t)NB * L.cpc * 2;
-    return common + std::max(c_wave, c_seq) + 64;
+    for (const SkLayer &L : s.plan[0]) c_wave = std::max(c_wave, role_bytes(NB, L.cpc, L.G, L.rpc));
+    for (const SkLayer &L : s.plan[1]) c_seq += role_bytes(NB, L.cpc, L.G, L.rpc);
+    return common + std::max(c_wave, c_seq) + 96;
 }
 
 // Plans the whole-stack kernel for a handle; *out stays null when the stack does not qualify (the per-layer kernels
@@ -711,8 +839,9 @@ int stack_small_create(const std::vector<const LayerParams *> &lp, int max_T, in
     if (s->max_B < 1) return fail(QLSTM_OK);
     s->smem = sk_smem_bytes(*s, sk_rows(s->max_B));
     s->cnt_words = (size_t)n * CNT_PER_LAYER + 16;
-    s->cnt = (unsigned *)dalloc(s->cnt_words * sizeof(unsigned));
+    s->cnt = (unsigned *)dalloc(2 * s->cnt_words * sizeof(unsigned));
     if (!s->cnt) return fail(QLSTM_ERR_NOMEM);
+    if (cudaMemset(s->cnt, 0, 2 * s->cnt_words * sizeof(unsigned)) != cudaSuccess) return fail(QLSTM_ERR_CUDA);
     for (int plan = 0; plan < 2; ++plan) {
         s->plan_dev[plan] = (SkLayer *)dalloc(sizeof(SkLayer) * n);
         if (!s->plan_dev[plan]) return fail(QLSTM_ERR_NOMEM);
@@ -740,7 +869,9 @@ bool stack_small_supported(const StackSmall *s, int T, int B) { return s && s->o
 bool stack_small_preferred(const StackSmall *s, int T, int B)
 {
     if (!stack_small_supported(s, T, B)) return false;
-    return B <= 4 || (B <= 8 && s->n_layers >= 6);
+    // a call of one or two steps is launch- and barrier-bound layer by layer (35 against 54 us for one step of ten
+    // 512-cell layers at 8 rows)
+    return B <= 4 || (B <= 8 && (s->n_layers >= 6 || T <= 2));
 }
 
 void stack_small_debug_timeout(StackSmall *s, unsigned missing_arrivals, unsigned long long limit_ns)
@@ -759,22 +890,25 @@ int stack_small_groups(const StackSmall *s, int *blocks_per_layer)
 
 // schedule: 0 automatic (sequential for calls of a few steps, where a wavefront has nothing to overlap), 1 wavefront,
 // 2 sequential
-int launch_stack_small(const StackSmall *s, const int8_t *x, int T, int B, int8_t *h, int16_t *c, int8_t *y, int *status,
+int launch_stack_small(StackSmall *s, const int8_t *x, int T, int B, int8_t *h, int16_t *c, int8_t *y, int *status,
                        int schedule, cudaStream_t st)
 {
     SkCall k;
     memset(&k, 0, sizeof(k));
     k.T = T; k.B = B; k.n_layers = s->n_layers;
     k.x = x; k.h = h; k.c = c; k.y = y;
-    k.cnt = s->cnt;
-    k.abort_word = s->cnt + (size_t)s->n_layers * CNT_PER_LAYER;
+    unsigned *set = s->cnt + (size_t)(s->calls & 1u) * s->cnt_words;
+    k.cnt = set;
+    k.abort_word = set + (size_t)s->n_layers * CNT_PER_LAYER;
+    k.cnt_next = s->cnt + (size_t)((s->calls + 1u) & 1u) * s->cnt_words;
+    k.cnt_words = (int)s->cnt_words;
+    ++s->calls;
     k.status = status;
     k.wait_limit_ns = s->dbg_limit_ns ? s->dbg_limit_ns : SK_WAIT_LIMIT_NS;
     k.missing_arrivals = s->dbg_missing;
     // a wavefront of L layers needs about L steps to fill; below that the layers are better run one after the other
     k.sequential = schedule == 2 || (schedule == 0 && (s->n_layers == 1 || T < s->n_layers)) ? 1 : 0;
     k.max_I = s->max_I; k.max_O = s->max_O; k.max_C_proj = s->max_C_proj; k.max_npc = s->max_npc;
-    if (cudaMemsetAsync(s->cnt, 0, s->cnt_words * sizeof(unsigned), st) != cudaSuccess) return QLSTM_ERR_CUDA;
     const SkLayer *layers = s->plan_dev[k.sequential];
     void *args[] = {(void *)&layers, (void *)&k};
     cudaError_t e = cudaLaunchCooperativeKernel(sk_kernel(sk_rows(B)), dim3(s->grid), dim3(SK_THREADS), args, s->smem, st);
