@@ -81,6 +81,24 @@ int qlstm_get_profile(qlstm_t *q, qlstm_profile_t *out, int reset);
  *     n <= 8191.
  */
 int qlstm_eval_activations(int cell_int_bits, int16_t *sigmoid_dev, int16_t *tanh_dev, void *cuda_stream);
+/*
+ * The persistent recurrent kernel memoises the nonlinearities of Section 3.2.1: at qlstm_create the definition is
+ * evaluated once over the whole int16 domain and packed into per-layer tables (plain uint16, or one 32-bit word per four
+ * inputs), which the kernel copies into shared memory before every elementwise phase.
+ *   qlstm_eval_activation_tables builds the tables of a layer whose cell state has cell_int_bits integer bits exactly as
+ *     qlstm_create does for a kernel with max_bytes (<= 131072) of idle shared memory, and looks every int16 input up with
+ *     the kernel's own lookup code: sigmoid_dev (Q3.12 in), tanh_gate_dev (Q3.12 in), tanh_cell_dev (Q_{m.15-m} in,
+ *     m = cell_int_bits): DEVICE int16 [65536], entry x + 32768.  layout_out7 (HOST) = { bytes of the tables, byte offset
+ *     of the gate tanh, of the cell tanh, last |x| with an entry of its own for the two, format of the cell tanh
+ *     (0 shared with the gate's, 1 packed, 2 plain), format of the sigmoid (0 plain, 1 packed) }; bytes = 0 means that
+ *     the tables do not fit or that the definition failed a check the formats rely on (the outputs are then untouched;
+ *     such a layer keeps the arithmetic).  Synchronises the stream.
+ *   qlstm_debug_activation_tables(q, 0) makes the kernel evaluate the definition instead (1 restores the default); it
+ *     returns the number of layers that hold tables, or a negative qlstm_error.
+ */
+int qlstm_eval_activation_tables(int cell_int_bits, int max_bytes, int16_t *sigmoid_dev, int16_t *tanh_gate_dev,
+                                 int16_t *tanh_cell_dev, int *layout_out7, void *cuda_stream);
+int qlstm_debug_activation_tables(qlstm_t *q, int enable);
 int qlstm_eval_layernorm_row(const int16_t *q_dev, int n, const int16_t *L_dev, const int32_t *b_dev,
                              qlstm_scale_t eff_ln, int16_t *out_dev, void *cuda_stream);
 

@@ -22,6 +22,7 @@ IMPL_AUTO, IMPL_SIMPLE, IMPL_FAST = 0, 1, 2
 EXPORTS = ["qlstm_create", "qlstm_run", "qlstm_run_host", "qlstm_input_projection", "qlstm_last_status",
            "qlstm_destroy", "qlstm_strerror", "qlstm_trace_bytes", "qlstm_set_impl", "qlstm_set_profiling",
            "qlstm_get_profile", "qlstm_device_info", "qlstm_eval_activations", "qlstm_eval_layernorm_row",
+           "qlstm_eval_activation_tables", "qlstm_debug_activation_tables",
            "qlstm_layernorm_rows_static", "qlstm_debug_barrier_timeout", "qlstm_debug_ring_plan",
            "qlstm_debug_projection_plan", "qlstm_debug_mma_i8_peak", "qlstm_debug_barrier_latency",
            "qlstm_bidir_create", "qlstm_bidir_run", "qlstm_bidir_last_status", "qlstm_bidir_destroy",
@@ -113,6 +114,11 @@ def lib():
         L.qlstm_device_info.argtypes = [C.c_void_p, C.POINTER(C.c_int), C.POINTER(C.c_int)]
         L.qlstm_eval_activations.restype = C.c_int
         L.qlstm_eval_activations.argtypes = [C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.qlstm_eval_activation_tables.restype = C.c_int
+        L.qlstm_eval_activation_tables.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_int),
+                                                   C.c_void_p]
+        L.qlstm_debug_activation_tables.restype = C.c_int
+        L.qlstm_debug_activation_tables.argtypes = [C.c_void_p, C.c_int]
         L.qlstm_eval_layernorm_row.restype = C.c_int
         L.qlstm_eval_layernorm_row.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, Scale, C.c_void_p, C.c_void_p]
         L.qlstm_debug_barrier_timeout.restype = C.c_int
@@ -266,6 +272,12 @@ class QLSTM:
     def set_impl(self, projection: int = IMPL_AUTO, recurrent: int = IMPL_AUTO):
         _check(lib().qlstm_set_impl(self._h, projection, recurrent), "qlstm_set_impl")
 
+    def activation_tables(self, enable: bool = True) -> int:
+        """Memoised sigmoid / tanh in the persistent kernel on (default) or off; returns the layers that hold tables."""
+        n = lib().qlstm_debug_activation_tables(self._h, 1 if enable else 0)
+        _check(min(n, 0), "qlstm_debug_activation_tables")
+        return n
+
     def set_profiling(self, level: int):
         """0 off, 1 per-kernel event times, 2 also the device phase timers (which slow the kernel they time)."""
         _check(lib().qlstm_set_profiling(self._h, int(level)), "qlstm_set_profiling")
@@ -325,6 +337,14 @@ def eval_activations(cell_int_bits: int, sigmoid_out, tanh_out, stream: int = 0)
     """qlstm_eval_activations on two device int16 [65536] tensors."""
     _check(lib().qlstm_eval_activations(cell_int_bits, _dev_ptr(sigmoid_out), _dev_ptr(tanh_out), stream),
            "qlstm_eval_activations")
+
+
+def eval_activation_tables(cell_int_bits: int, max_bytes: int, sigmoid_out, tanh_gate_out, tanh_cell_out, stream: int = 0):
+    """qlstm_eval_activation_tables on three device int16 [65536] tensors; returns the seven layout numbers."""
+    lay = (C.c_int * 7)()
+    _check(lib().qlstm_eval_activation_tables(cell_int_bits, max_bytes, _dev_ptr(sigmoid_out), _dev_ptr(tanh_gate_out),
+                                              _dev_ptr(tanh_cell_out), lay, stream), "qlstm_eval_activation_tables")
+    return list(lay)
 
 
 def eval_layernorm_row(q, n: int, L, b, eff_ln, out, stream: int = 0):

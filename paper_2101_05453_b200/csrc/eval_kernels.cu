@@ -5,6 +5,7 @@
 
 #include "../../include/qlstm.h"
 #include "../../include/qlstm_debug.h"
+#include "act_table.cuh"
 #include "qmath.cuh"
 
 namespace ql {
@@ -37,9 +38,51 @@ __global__ void k_eval_layernorm_row(const int16_t *q, int n, const int16_t *L, 
     for (int i = threadIdx.x; i < n; i += blockDim.x) out[i] = (int16_t)ln_apply_fast(q[i], row, L[i], b[i], eff, f);
 }
 
+// The memoised nonlinearities through the lookup code of the recurrent kernel: the blob is copied into shared memory
+// as that kernel's bulk copy does, then every int16 input is looked up.
+__global__ void k_eval_activation_tables(const uint8_t *blob, ActTabLayout lay, int16_t *sig, int16_t *tz, int16_t *tc)
+{
+    extern __shared__ __align__(16) uint8_t tab_s[];
+    for (uint32_t i = threadIdx.x; i < lay.bytes / 16; i += blockDim.x)
+        reinterpret_cast<uint4 *>(tab_s)[i] = reinterpret_cast<const uint4 *>(blob)[i];
+    __syncthreads();
+    const ActTabs at = make_act_tabs((uint32_t)__cvta_generic_to_shared(tab_s), lay);
+    for (int i = threadIdx.x; i < 65536; i += blockDim.x) {
+        const int32_t x = i - 32768;
+        sig[i] = (int16_t)tab_sigmoid(at, x);
+        tz[i] = (int16_t)tab_tanh_gate(at, x);
+        tc[i] = (int16_t)tab_tanh_cell(at, x);
+    }
+}
+
 }  // namespace ql
 
 extern "C" {
+
+int qlstm_eval_activation_tables(int cell_int_bits, int max_bytes, int16_t *sigmoid_dev, int16_t *tanh_gate_dev,
+                                 int16_t *tanh_cell_dev, int *layout_out7, void *cuda_stream)
+{
+    if (cell_int_bits < 0 || cell_int_bits > 15 || max_bytes < 0 || max_bytes > 128 * 1024 || !sigmoid_dev || !tanh_gate_dev ||
+        !tanh_cell_dev || !layout_out7)
+        return QLSTM_ERR_ARG;
+    int *layout_out6 = layout_out7;
+    uint8_t *blob = nullptr;
+    ql::ActTabLayout lay;
+    if (!ql::act_tables_build(cell_int_bits, (size_t)max_bytes, &blob, &lay)) return QLSTM_ERR_CUDA;
+    layout_out6[0] = (int)lay.bytes; layout_out6[1] = (int)lay.tz_off; layout_out6[2] = (int)lay.tc_off;
+    layout_out6[3] = lay.tz_amax; layout_out6[4] = lay.tc_amax; layout_out6[5] = lay.tc_mode; layout_out7[6] = lay.sig_packed;
+    if (!blob) return QLSTM_OK;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    int rc = QLSTM_OK;
+    if (cudaFuncSetAttribute(ql::k_eval_activation_tables, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)lay.bytes) != cudaSuccess)
+        rc = QLSTM_ERR_CUDA;
+    if (rc == QLSTM_OK) {
+        ql::k_eval_activation_tables<<<1, 1024, lay.bytes, st>>>(blob, lay, sigmoid_dev, tanh_gate_dev, tanh_cell_dev);
+        if (cudaGetLastError() != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) rc = QLSTM_ERR_CUDA;
+    }
+    cudaFree(blob);
+    return rc;
+}
 
 int qlstm_eval_activations(int cell_int_bits, int16_t *sigmoid_dev, int16_t *tanh_dev, void *cuda_stream)
 {

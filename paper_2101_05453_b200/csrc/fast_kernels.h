@@ -6,6 +6,7 @@
 
 #include <vector>
 
+#include "act_table.cuh"
 #include "qlstm_internal.h"
 
 namespace ql {
@@ -41,6 +42,10 @@ struct FastLayer {
     int n_issue_c = 1;           // projection MMA issuers, each with its own partial accumulator
     size_t smem = 0;
     CUtensorMap map_R, map_Wp;   // resident weight slices; the streamed operands h, m use plain bulk copies
+    // memoised sigmoid / tanh of the elementwise phase (act_table.cuh): device blob and its layout; null: arithmetic path
+    uint8_t *act_tab = nullptr;
+    ActTabLayout act_lay = {0, 0, 0, 0, 0, 0, 0};
+    bool dbg_no_tables = false;  // test hook: keep the arithmetic path although the tables exist
     // test hook: make every grid barrier expect `dbg_barrier_extra` arrivals that never come, with a short wait limit
     unsigned dbg_barrier_extra = 0;
     unsigned long long dbg_spin_limit_ns = 0;

@@ -495,6 +495,17 @@ int qlstm_debug_barrier_timeout(qlstm_t *q, int missing_arrivals, unsigned long 
     return QLSTM_OK;
 }
 
+int qlstm_debug_activation_tables(qlstm_t *q, int enable)
+{
+    if (!q) return QLSTM_ERR_ARG;
+    int n = 0;
+    for (auto &L : q->layers) {
+        L.fast.dbg_no_tables = enable == 0;
+        if (L.fast.act_tab) ++n;
+    }
+    return n;
+}
+
 int qlstm_set_profiling(qlstm_t *q, int level)
 {
     if (!q) return QLSTM_ERR_ARG;

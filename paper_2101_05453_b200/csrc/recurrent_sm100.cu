@@ -31,6 +31,7 @@
 
 #include "../../include/qlstm.h"
 #include "../../include/qlstm_debug.h"
+#include "act_table.cuh"
 #include "fast_kernels.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
@@ -94,11 +95,13 @@ struct RecParams {
     int gate_slot[4];             // canonical gate -> slot, -1 if absent
     unsigned long long spin_limit_ns;   // bound of one grid-barrier wait
     unsigned barrier_extra;             // 0; a test sets it to make the barrier wait for an arrival that never comes
+    const uint8_t *tab;           // memoised sigmoid / tanh tables of this layer (act_table.cuh), copied into the idle ring
+    ActTabLayout tab_lay;         // before every elementwise phase; used by the instantiations with TAB only
     unsigned long long *phase_ns; // null, or 6 accumulators: work and barrier wait of phases A, B, C (CTA 0)
 };
 
 struct RecCtl {
-    uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[3], w_full, x_full;
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[3], w_full, x_full, tab_full;
     uint32_t tmem_base;
     uint32_t rounds[MAX_STAGES];
     int abort_flag;
@@ -396,9 +399,34 @@ __device__ __forceinline__ void store_hidden_pair(const RecParams &p, int b, int
     }
 }
 
+// The nonlinearities of the elementwise phase: the fixed-point definition, or its memoised values (TAB).
+template <bool TAB>
+__device__ __forceinline__ int32_t gate_sigmoid(const ActTabs &at, int32_t x)
+{
+    if constexpr (TAB) return tab_sigmoid(at, x);
+    else return sigmoid_q_fast(x, 3);
+}
+template <bool TAB>
+__device__ __forceinline__ int32_t gate_tanh(const ActTabs &at, int32_t x)
+{
+    if constexpr (TAB) return tab_tanh_gate(at, x);
+    else return tanh_q_fast(x, 3);
+}
+template <bool TAB>
+__device__ __forceinline__ int32_t hidden_of(const RecParams &p, const ActTabs &at, int32_t o, int32_t c_new)
+{
+    if constexpr (TAB) {
+        const int32_t prod = o * tab_tanh_cell(at, c_new);
+        return sat8((p.eff_m.shift <= 0 ? fast_rescale(prod, p.f_m) : mbqm_cold(prod, p.eff_m)) + p.zp_m);
+    } else {
+        return hidden_q_fast(o, c_new, p.m_bits, p.eff_m, p.f_m, p.zp_m);
+    }
+}
+
 // One pair of the block's own cells (local pair k of row b), gate sums in shared memory.
-template <int G, bool PEEP>
-__device__ __forceinline__ void own_cell_pair(const RecParams &p, const OwnCells &oc, int b, int k, int t, int8_t *h_next)
+template <int G, bool PEEP, bool TAB>
+__device__ __forceinline__ void own_cell_pair(const RecParams &p, const OwnCells &oc, const ActTabs &at, int b, int k, int t,
+                                              int8_t *h_next)
 {
     constexpr int SI = 0, SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
     const int ul = 2 * k, nl = ul * G;                     // local cell and column
@@ -411,9 +439,9 @@ __device__ __forceinline__ void own_cell_pair(const RecParams &p, const OwnCells
     int32_t c_new[2], m[2];
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
-        const int32_t f = sigmoid_q_fast(a[q][SF], 3), z = tanh_q_fast(a[q][SZ], 3);
+        const int32_t f = gate_sigmoid<TAB>(at, a[q][SF]), z = gate_tanh<TAB>(at, a[q][SZ]);
         int32_t i;
-        if (G == 4) i = sigmoid_q_fast(a[q][SI], 3);
+        if (G == 4) i = gate_sigmoid<TAB>(at, a[q][SI]);
         else { i = 32768 - f; if (i > 32767) i = 32767; }          // coupled input gate, Section 3.2.9
         c_new[q] = cell_update_fast(i, z, f, c_old[q], p.m_bits);
         int32_t ao = a[q][SO];
@@ -421,7 +449,7 @@ __device__ __forceinline__ void own_cell_pair(const RecParams &p, const OwnCells
             const int32_t H = oc.ho_s[(size_t)b * p.cpc + ul + q], P = oc.P_s[nl + q * G + SO];
             ao = sat16(ao + H + sat16(rescale_any(P * c_new[q], p.eff_c[SO], p.f_c[SO])));   // Eq. 5: o sees c^t
         }
-        m[q] = hidden_q_fast(sigmoid_q_fast(ao, 3), c_new[q], p.m_bits, p.eff_m, p.f_m, p.zp_m);
+        m[q] = hidden_of<TAB>(p, at, gate_sigmoid<TAB>(at, ao), c_new[q]);
     }
     *reinterpret_cast<uint32_t *>(c_ptr) = pack16(c_new[0], c_new[1]);
     store_hidden_pair(p, b, u, t, m[0], m[1], h_next);
@@ -429,13 +457,13 @@ __device__ __forceinline__ void own_cell_pair(const RecParams &p, const OwnCells
 
 // All (row, cell pair) tasks of the block, consecutive threads on consecutive pairs of a row: the gate sums of a row's
 // pairs are contiguous in shared memory.
-template <int G, bool PEEP>
-__device__ __forceinline__ void phase_b_own(const RecParams &p, const OwnCells &oc, int t, int8_t *h_next)
+template <int G, bool PEEP, bool TAB>
+__device__ __forceinline__ void phase_b_own(const RecParams &p, const OwnCells &oc, const ActTabs &at, int t, int8_t *h_next)
 {
     const int pairs = oc.cells >> 1, total = p.B * pairs;
     for (int i = threadIdx.x; i < total; i += RTHREADS) {
         const int b = i / pairs, k = i - b * pairs;
-        own_cell_pair<G, PEEP>(p, oc, b, k, t, h_next);
+        own_cell_pair<G, PEEP, TAB>(p, oc, at, b, k, t, h_next);
     }
 }
 
@@ -483,8 +511,9 @@ __device__ __forceinline__ void load_pair_i32_cg(const int32_t *ptr, int32_t (&v
 }
 
 // Two adjacent cells (u even) of row b, every step after the gate sums (layer norm without peephole).
-template <int G, bool LN, bool PEEP>
-__device__ __forceinline__ void flat_cell_pair(const RecParams &p, const LnRow *lr, int b, int u, int t, int8_t *h_next)
+template <int G, bool LN, bool PEEP, bool TAB>
+__device__ __forceinline__ void flat_cell_pair(const RecParams &p, const ActTabs &at, const LnRow *lr, int b, int u, int t,
+                                               int8_t *h_next)
 {
     constexpr int SI = 0, SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
     const size_t nb = (size_t)b * p.N + (size_t)u * G;
@@ -520,22 +549,22 @@ __device__ __forceinline__ void flat_cell_pair(const RecParams &p, const LnRow *
     int32_t c_new[2], m[2];
 #pragma unroll
     for (int k = 0; k < 2; ++k) {
-        const int32_t f = sigmoid_q_fast(a[k][SF], 3), z = tanh_q_fast(a[k][SZ], 3);
+        const int32_t f = gate_sigmoid<TAB>(at, a[k][SF]), z = gate_tanh<TAB>(at, a[k][SZ]);
         int32_t i;
-        if (G == 4) i = sigmoid_q_fast(a[k][SI], 3);
+        if (G == 4) i = gate_sigmoid<TAB>(at, a[k][SI]);
         else { i = 32768 - f; if (i > 32767) i = 32767; }          // coupled input gate, Section 3.2.9
         c_new[k] = cell_update_fast(i, z, f, c_old[k], p.m_bits);
         int32_t ao = a[k][SO];
         if (PEEP) ao = sat16(ao + sat16(rescale_any(P[k][SO] * c_new[k], p.eff_c[SO], p.f_c[SO])));
-        const int32_t o = sigmoid_q_fast(ao, 3);
-        m[k] = hidden_q_fast(o, c_new[k], p.m_bits, p.eff_m, p.f_m, p.zp_m);
+        const int32_t o = gate_sigmoid<TAB>(at, ao);
+        m[k] = hidden_of<TAB>(p, at, o, c_new[k]);
     }
     *reinterpret_cast<uint32_t *>(c_ptr) = pack16(c_new[0], c_new[1]);
     store_hidden_pair(p, b, u, t, m[0], m[1], h_next);
 }
 
-template <int G, bool LN, bool PEEP>
-__device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, int t, int8_t *h_next)
+template <int G, bool LN, bool PEEP, bool TAB>
+__device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, const ActTabs &at, int t, int8_t *h_next)
 {
     const int total = p.B * p.C;
     const int i0 = blockIdx.x * p.items_per_cta;
@@ -592,7 +621,7 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, in
         const int j1 = i1 < (re + 1) * p.C ? i1 : (re + 1) * p.C;
         for (int i = j0 + 2 * threadIdx.x; i < j1; i += 2 * RTHREADS) {
             const int b = i / p.C, u = i - b * p.C;
-            flat_cell_pair<G, LN, PEEP>(p, ctl->ln_rows[b - rb], b, u, t, h_next);
+            flat_cell_pair<G, LN, PEEP, TAB>(p, at, ctl->ln_rows[b - rb], b, u, t, h_next);
         }
         if (LN) ptx::cta_sync();      // the statistics slots are reused by the next batch of rows
     }
@@ -600,8 +629,9 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, in
 
 // Layer norm with peephole: the gate sums need their peephole term before the statistics, and the output
 // gate's statistics need c^t of the whole row, so a row is processed by one CTA in three passes.
-template <int G>
-__device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl, int t, int8_t *h_next, int16_t *row_s)
+template <int G, bool TAB>
+__device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl, const ActTabs &at, int t, int8_t *h_next,
+                                                int16_t *row_s)
 {
     constexpr int SI = 0, SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
     const int rows_per_cta = p.items_per_cta / p.C;
@@ -635,9 +665,9 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
 #pragma unroll
             for (int g = 0; g < G; ++g)
                 if (g != SO) a[g] = ln_apply_fast(pre_s[nb + g], lr[g], __ldg(p.L + nb + g), __ldg(p.bln + nb + g), p.eff_ln[g], p.f_ln[g]);
-            const int32_t f = sigmoid_q_fast(a[SF], 3), z = tanh_q_fast(a[SZ], 3);
+            const int32_t f = gate_sigmoid<TAB>(at, a[SF]), z = gate_tanh<TAB>(at, a[SZ]);
             int32_t i;
-            if (G == 4) i = sigmoid_q_fast(a[SI], 3);
+            if (G == 4) i = gate_sigmoid<TAB>(at, a[SI]);
             else { i = 32768 - f; if (i > 32767) i = 32767; }
             const int32_t c_new = cell_update_fast(i, z, f, c_row[u], p.m_bits);
             c_row[u] = (int16_t)c_new;
@@ -652,8 +682,8 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
         for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
             const int n = u * G + SO;
             const int32_t ao = ln_apply_fast(pre_s[n], lr[SO], __ldg(p.L + n), __ldg(p.bln + n), p.eff_ln[SO], p.f_ln[SO]);
-            const int32_t o = sigmoid_q_fast(ao, 3);
-            const int32_t m = hidden_q_fast(o, cnew_s[u], p.m_bits, p.eff_m, p.f_m, p.zp_m);
+            const int32_t o = gate_sigmoid<TAB>(at, ao);
+            const int32_t m = hidden_of<TAB>(p, at, o, cnew_s[u]);
             if (p.flags & F_PROJECTION) {
                 p.mbuf[operand_off(p, b, u, p.C, p.kb_c)] = (int8_t)m;
             } else {
@@ -829,7 +859,7 @@ __device__ __noinline__ void drain_box_requests(uint64_t *x_full)
 
 // One instantiation per variant (gates, layer norm, peephole): each keeps only its own epilogue and elementwise code,
 // which is what lets the register allocator fit them without spilling.
-template <int G, bool LN, bool PEEP>
+template <int G, bool LN, bool PEEP, bool TAB>
 __global__ void __launch_bounds__(RTHREADS, 1)
 k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_constant__ CUtensorMap map_Wp,
                   const __grid_constant__ CUtensorMap map_X, const __grid_constant__ CUtensorMap map_pre, RecParams p)
@@ -882,6 +912,7 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
         ptx::mbar_init(&ctl->acc_full[2], (uint32_t)(p.plan_c.n_own > 0 ? p.plan_c.n_own : 1));      // one arrival per projection issuer
         ptx::mbar_init(&ctl->w_full, 1);
         ptx::mbar_init(&ctl->x_full, 1);
+        ptx::mbar_init(&ctl->tab_full, 1);
         ctl->abort_flag = 0;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&map_R);
@@ -963,6 +994,13 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
     };
     const int ngroups = n_cnt >> 3;
     constexpr int gstep = (G == 4) ? 1 : 3;                        // groups are dealt in units of this many
+    // TAB: the tables of the nonlinearities are copied into the ring when the recurrent matmul has drained it, read by
+    // the elementwise phase, and overwritten by the projection's operand after the next grid barrier
+    const ActTabs at = make_act_tabs(ptx::smem_u32(ring), p.tab_lay);
+    auto fetch_tables = [&]() {
+        ptx::mbar_arrive_expect_tx(&ctl->tab_full, p.tab_lay.bytes);
+        ptx::bulk_load_1d(ring, p.tab, p.tab_lay.bytes, &ctl->tab_full);
+    };
 
     for (int t = 0; t < p.T; ++t) {
         const int cur = t & 1;
@@ -994,6 +1032,12 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
                 if (lane == 0) {
                     fence_proxy_async_global();
                     ring_produce(ctl, rg, p.plan_a, true, p.kb_h, p.hbuf + (size_t)cur * p.h_stride, abort_flag);
+                    if (TAB) {
+                        // every MMA of this step has read its ring stages once the accumulators are complete
+                        bool drained = true;
+                        for (int mi = 0; mi < p.MT; ++mi) drained = drained && wait_or_abort(&ctl->acc_full[mi], par, abort_flag);
+                        if (drained) fetch_tables();
+                    }
                 }
                 __syncwarp();
             } else {
@@ -1031,6 +1075,7 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
               }
             }
         }
+        if (TAB && !has_cells && ln && threadIdx.x == 0) fetch_tables();     // no matmul here: the ring is idle already
         ptx::cta_sync();
         if (tensor_a && threadIdx.x == 0) ring_advance(rg, p.plan_a);
         if (ln) {
@@ -1049,12 +1094,14 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
             grid_sync(p, epoch, abort_flag, false);
             lap(1);
             if (*abort_flag) break;
-            if (peep) phase_b_ln_peep<G>(p, ctl, t, h_next, row_s);
-            else phase_b_flat<G, true, false>(p, ctl, t, h_next);
+            // (a wait that runs out sets the abort flag: the next barrier ends the time loop)
+            if (TAB && !wait_or_abort(&ctl->tab_full, par, abort_flag)) {}
+            else if (peep) phase_b_ln_peep<G, TAB>(p, ctl, at, t, h_next, row_s);
+            else phase_b_flat<G, true, false, TAB>(p, ctl, at, t, h_next);
             ptx::cta_sync();
         } else {
             // same block, same cells, straight from shared memory
-            phase_b_own<G, PEEP>(p, oc, t, h_next);
+            if (!TAB || !has_cells || wait_or_abort(&ctl->tab_full, par, abort_flag)) phase_b_own<G, PEEP, TAB>(p, oc, at, t, h_next);
             ptx::fence_proxy_async();                        // X box and ring scratch go back to the async proxy
             ptx::cta_sync();
             if (has_cells && threadIdx.x == 0 && t + 1 < p.T && !*abort_flag) fetch_x(t + 1);
@@ -1171,17 +1218,19 @@ size_t rec_smem_bytes(const LayerParams &p, int stages, int nc_pad, int pn, int 
 
 int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
-// the instantiation for a layer's variant
-const void *recurrent_kernel(const LayerParams &p)
+// the instantiation for a layer's variant; tab: with the memoised nonlinearities
+template <bool TAB>
+const void *recurrent_kernel_of(const LayerParams &p)
 {
     const bool ln = (p.flags & F_LAYERNORM) != 0, peep = (p.flags & F_PEEPHOLE) != 0;
     if (p.G == 4) {
-        if (ln) return peep ? (const void *)k_recurrent_sm100<4, true, true> : (const void *)k_recurrent_sm100<4, true, false>;
-        return peep ? (const void *)k_recurrent_sm100<4, false, true> : (const void *)k_recurrent_sm100<4, false, false>;
+        if (ln) return peep ? (const void *)k_recurrent_sm100<4, true, true, TAB> : (const void *)k_recurrent_sm100<4, true, false, TAB>;
+        return peep ? (const void *)k_recurrent_sm100<4, false, true, TAB> : (const void *)k_recurrent_sm100<4, false, false, TAB>;
     }
-    if (ln) return peep ? (const void *)k_recurrent_sm100<3, true, true> : (const void *)k_recurrent_sm100<3, true, false>;
-    return peep ? (const void *)k_recurrent_sm100<3, false, true> : (const void *)k_recurrent_sm100<3, false, false>;
+    if (ln) return peep ? (const void *)k_recurrent_sm100<3, true, true, TAB> : (const void *)k_recurrent_sm100<3, true, false, TAB>;
+    return peep ? (const void *)k_recurrent_sm100<3, false, true, TAB> : (const void *)k_recurrent_sm100<3, false, false, TAB>;
 }
+const void *recurrent_kernel(const LayerParams &p, bool tab) { return tab ? recurrent_kernel_of<true>(p) : recurrent_kernel_of<false>(p); }
 
 // contig: n_own operand tiles of `per` chunks each, one owner per tile; else n_total chunks of one tile dealt round-robin
 RingPlan make_ring_plan(int stages, int n_own, bool contig, int per, int n_total)
@@ -1265,11 +1314,16 @@ int fast_recurrent_init(FastLayer &f, const LayerParams &p, const FastScratch &s
     } else {
         f.map_Wp = f.map_R;
     }
-    if (cudaFuncSetAttribute(recurrent_kernel(p), cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
-        return QLSTM_OK;
-    int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, recurrent_kernel(p), RTHREADS, f.smem) != cudaSuccess || per_sm < 1)
-        return QLSTM_OK;
+    for (int tab = 0; tab < 2; ++tab) {
+        int per_sm = 0;
+        if (cudaFuncSetAttribute(recurrent_kernel(p, tab != 0), cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
+            return QLSTM_OK;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, recurrent_kernel(p, tab != 0), RTHREADS, f.smem) != cudaSuccess ||
+            per_sm < 1)
+            return QLSTM_OK;
+    }
+    // memoised nonlinearities, if their tables fit into the ring (they live there between the matmul phases)
+    if (!act_tables_build(p.m_bits, (size_t)f.stages * STAGE_BYTES, &f.act_tab, &f.act_lay)) return QLSTM_ERR_CUDA;
     f.rec_ok = true;
     return QLSTM_OK;
 }
@@ -1282,7 +1336,12 @@ int fast_layer_init(FastLayer &f, const LayerParams &p, const FastScratch &s, in
     return fast_recurrent_init(f, p, s, max_B);
 }
 
-void fast_layer_destroy(FastLayer &) {}
+void fast_layer_destroy(FastLayer &f)
+{
+    if (f.act_tab) cudaFree(f.act_tab);
+    f.act_tab = nullptr;
+    f.act_lay = ActTabLayout{0, 0, 0, 0, 0, 0, 0};
+}
 
 bool fast_recurrent_supported(const FastLayer &f, const LayerParams &, int B) { return f.rec_ok && B <= 256; }
 
@@ -1342,6 +1401,9 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     rp.f_proj = make_fast_scale(p.eff_proj);
     rp.f_m = make_fast_scale(p.eff_m);
     rp.phase_ns = phase_ns;
+    const bool tab = f.act_tab != nullptr && !rp.small && !f.dbg_no_tables;
+    rp.tab = tab ? f.act_tab : nullptr;
+    rp.tab_lay = f.act_lay;
     rp.spin_limit_ns = f.dbg_spin_limit_ns ? f.dbg_spin_limit_ns : SPIN_LIMIT_NS;
     rp.barrier_extra = f.dbg_barrier_extra;
     if (p.eff_proj.shift > 0) rp.fast_rescale_ok = 0;
@@ -1369,7 +1431,7 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
         !make_tensor_map_i16(&map_pre, s.pre, (uint64_t)B, (uint64_t)p.N, (uint32_t)rp.x_rows, (uint32_t)rp.npc))
         return QLSTM_ERR_CUDA;
     void *args[] = {(void *)&f.map_R, (void *)&f.map_Wp, (void *)&map_X, (void *)&map_pre, (void *)&rp};
-    cudaError_t e = cudaLaunchCooperativeKernel(recurrent_kernel(p), dim3(f.grid), dim3(RTHREADS), args, f.smem, st);
+    cudaError_t e = cudaLaunchCooperativeKernel(recurrent_kernel(p, tab), dim3(f.grid), dim3(RTHREADS), args, f.smem, st);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return e == cudaErrorCooperativeLaunchTooLarge ? QLSTM_ERR_LAUNCH : QLSTM_ERR_CUDA;

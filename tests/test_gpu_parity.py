@@ -469,6 +469,67 @@ def test_device_activations_exhaustive(m):
     assert np.array_equal(tnh.cpu().numpy().astype(np.int32), R.tanh_all(m))
 
 
+@pytest.mark.parametrize("m,room", [(0, 128), (1, 128), (2, 128), (2, 96), (3, 128), (3, 64), (4, 128), (5, 128), (5, 96),
+                                    (6, 128), (9, 128), (15, 128)])
+def test_device_activation_tables_exhaustive(m, room):
+    """The memoised nonlinearities of the persistent kernel (tables built as at create time for `room` KB of idle shared
+    memory, the kernel's own lookup code) on every int16 input against the oracle: sigmoid and tanh of the gates
+    (Q3.12), tanh of a Q_{m.15-m} cell."""
+    import torch
+    from paper_2101_05453_b200 import binding
+    out = [torch.full((65536,), 12345, dtype=torch.int16, device="cuda") for _ in range(3)]
+    lay = binding.eval_activation_tables(m, room * 1024, *out, stream=torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    nbytes, tz_off, tc_off, tz_amax, tc_amax, tc_mode, sig_packed = lay
+    assert 0 < nbytes <= room * 1024 and nbytes % 16 == 0, lay         # the definition passes the formats' checks
+    assert tz_off % 16 == 0 and tc_off % 16 == 0
+    assert tc_mode == (0 if m == 3 else (1 if m < 3 else 2)), lay      # steps of 2^m fit the 5-bit offsets up to m = 3
+    assert sig_packed == (1 if room < 128 else 0), lay                 # the plain sigmoid table alone is 64 KB
+    assert 0 < tz_amax <= 32768 and 0 < tc_amax <= 32768
+    sig, tz, tc = (o.cpu().numpy().astype(np.int32) for o in out)
+    assert np.array_equal(sig, R.sigmoid_all(3))
+    assert np.array_equal(tz, R.tanh_all(3))
+    assert np.array_equal(tc, R.tanh_all(m))
+
+
+def test_device_activation_tables_that_do_not_fit():
+    import torch
+    from paper_2101_05453_b200 import binding
+    out = [torch.full((65536,), 12345, dtype=torch.int16, device="cuda") for _ in range(3)]
+    lay = binding.eval_activation_tables(2, 48 * 1024, *out, stream=torch.cuda.current_stream().cuda_stream)
+    assert lay[0] == 0
+    assert all(int(o.min()) == 12345 and int(o.max()) == 12345 for o in out)
+
+
+@pytest.mark.parametrize("idx,B", [(5, 256), (5, 40), (4, 64), (3, 32), (2, 8)])
+def test_tables_and_arithmetic_agree(idx, B):
+    """The same call with the memoised nonlinearities and with the definition evaluated in the kernel: identical
+    outputs and state, both equal to the oracle (which the other parity tests compare the default path with)."""
+    import torch
+    import paper_2101_05453_b200 as qlstm
+    T = 6
+    w = make_workload(idx, batch=B, T=T)
+    O = w.layers[-1].n_output
+    dev = torch.device("cuda:0")
+    q = qlstm.QLSTM(w.layers, T, B, device=0)
+    q.set_impl(2, 2)
+    res = []
+    for enable in (True, False):
+        n_tab = q.activation_tables(enable)
+        assert n_tab == len(w.layers)                 # every layer of these configurations has room for its tables
+        h0, c0 = w.initial_state()
+        h, c = torch.from_numpy(h0).to(dev), torch.from_numpy(c0).to(dev)
+        y = torch.zeros((T, B, O), dtype=torch.int8, device=dev)
+        q.run(torch.from_numpy(w.x).to(dev), T, B, h, c, y)
+        torch.cuda.synchronize()
+        q.last_status()
+        res.append((y.cpu().numpy(), h.cpu().numpy(), c.cpu().numpy()))
+    q.close()
+    check_equal(res[0], res[1], f"config {idx} batch {B}: tables against arithmetic")
+    if B <= 64:
+        check_equal(res[0], oracle(w), f"config {idx} batch {B}: tables against the oracle")
+
+
 @pytest.mark.parametrize("seed", range(10))
 def test_device_layernorm_rows(seed):
     import torch
