@@ -37,4 +37,11 @@ int32_t qmh_hidden_fast(int32_t o, int32_t c, int m, int32_t mult, int32_t shift
     return ql::hidden_q_fast(o, c, m, sc, ql::make_fast_scale(sc), zp);
 }
 uint64_t qmh_isqrt(uint64_t v) { return ql::isqrt64(v); }
+uint64_t qmh_isqrt_from_f32(uint64_t v) { return ql::isqrt_from_f32(v); }
+uint64_t qmh_div_by_magic(uint64_t x, uint32_t n) { return ql::div_by_magic(x, ql::make_div_magic(n)); }
+void qmh_ln_stats(int64_t sum, int64_t sumsq, int n, int fast, int64_t *mean_sigma)
+{
+    ql::LnStats s = fast ? ql::ln_stats_fast(sum, sumsq, ql::make_div_magic((uint32_t)n)) : ql::ln_stats(sum, sumsq, n);
+    mean_sigma[0] = s.mean; mean_sigma[1] = s.sigma;
+}
 }

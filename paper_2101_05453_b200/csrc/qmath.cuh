@@ -207,6 +207,60 @@ QL_HD LnStats ln_stats(int64_t sum, int64_t sumsq, int n)
     return s;
 }
 
+// The same statistics without a hardware-less 64-bit division or an fp64 square root on the way (in the kernels one
+// thread per (row, gate) computes them while the whole block waits): the divisor n is fixed per layer, so x / n is the
+// high half of x * ceil(2^64 / n), exact for x < 2^50 and n < 2^14; the square root starts from an fp32 estimate.
+// Requires n < 2^14 and |q| <= 2^15 (then sum 2^10 < 2^39 and sumsq < 2^44).
+struct DivMagic { uint64_t m; uint32_t n; };
+
+QL_HD DivMagic make_div_magic(uint32_t n)
+{
+    DivMagic d;
+    d.n = n;
+    d.m = n > 1 ? ~(uint64_t)0 / n + 1 : 0;          // floor((2^64 - 1) / n) + 1 = floor(2^64 / n) + 1 unless n divides 2^64,
+                                                     // where it is 2^64 / n exactly: both are valid multipliers
+    return d;
+}
+
+QL_HD uint64_t umul64hi_hd(uint64_t a, uint64_t b)
+{
+#if defined(__CUDA_ARCH__)
+    return __umul64hi(a, b);
+#else
+    return (uint64_t)(((unsigned __int128)a * b) >> 64);
+#endif
+}
+
+QL_HD uint64_t div_by_magic(uint64_t x, const DivMagic &d) { return d.n > 1 ? umul64hi_hd(x, d.m) : x; }   // x < 2^50
+
+QL_HD uint64_t isqrt_from_f32(uint64_t v)           // floor(sqrt(v)), v < 2^52
+{
+#if defined(__CUDA_ARCH__)
+    uint64_t r = (uint64_t)__fsqrt_rn((float)v);
+#else
+    uint64_t r = (uint64_t)__builtin_sqrtf((float)v);
+#endif
+    while (r * r > v) --r;
+    while ((r + 1) * (r + 1) <= v) ++r;
+    return r;
+}
+
+QL_HD LnStats ln_stats_fast(int64_t sum, int64_t sumsq, const DivMagic &d)
+{
+    LnStats s;
+    const uint64_t half = d.n >> 1;
+    const uint64_t as = (uint64_t)(sum < 0 ? -sum : sum) * 1024u;
+    const int64_t am = (int64_t)div_by_magic(as + half, d);
+    s.mean = sum < 0 ? -am : am;
+    // round(sumsq 2^20 / n) = floor(sumsq / n) 2^20 + floor(((sumsq mod n) 2^20 + n / 2) / n)
+    const uint64_t q1 = div_by_magic((uint64_t)sumsq, d);
+    const uint64_t r1 = (uint64_t)sumsq - q1 * d.n;
+    const uint64_t msq = (q1 << 20) + div_by_magic((r1 << 20) + half, d);
+    const int64_t var = (int64_t)msq - s.mean * s.mean;
+    s.sigma = (int64_t)isqrt_from_f32(var > 0 ? (uint64_t)var : 0);
+    return s;
+}
+
 // One element: q' = round(2^10 (2^10 q - mean) / sigma); out = sat16(rescale(sat32(q' L + b), eff_ln)).
 // Per (row, gate) constants: mean, sigma and the fp32 reciprocal of sigma for the quotient estimate.
 struct LnRow { int32_t mean; uint32_t sigma; float inv_sigma; };
@@ -220,31 +274,40 @@ QL_HD LnRow make_ln_row(LnStats s)
     return r;
 }
 
-// q' = round(2^10 (2^10 q - mean) / sigma), exact.  Quotients below 2^16 (|z-score| < 64) take the fp32
+// q' = round(2^10 (2^10 q - mean) / sigma), exact.  Quotients up to 2^16 (|z-score| <= 64) take the fp32
 // estimate (biased low: q' or q' - 1) and one remainder test modulo 2^32; anything larger - a tiny sigma
-// against a large deviation - takes the plain 64-bit division.
-QL_HD int64_t ln_scaled_fast(int32_t q, const LnRow &r, int32_t L, int32_t b)   // q' * L + b
+// against a large deviation - takes the plain 64-bit division.  fast: the quotient fits 17 bits, so that its product
+// with an int16 weight fits an int32.
+QL_HD int64_t ln_quotient_core(int32_t q, const LnRow &r, bool &fast)
 {
     const int32_t d = 1024 * q - r.mean;
     const uint32_t ad = (uint32_t)(d < 0 ? -d : d);
     const uint32_t half = r.sigma >> 1;
     const float est = fma_rn(fma_rn((float)ad, 1024.0f, (float)half), r.inv_sigma, -0.05f);
-    if (est < 65536.0f) {
+    fast = est < 65536.0f;
+    if (fast) {
+#if defined(__CUDA_ARCH__)
+        uint32_t qe = __float2uint_rz(est);                        // a negative estimate (ad = 0) converts to 0
+#else
         uint32_t qe = est > 0.0f ? (uint32_t)est : 0u;
+#endif
         const uint32_t rem = (ad << 10) + half - qe * r.sigma;     // in [0, 2 sigma), exact modulo 2^32
         qe += (rem >= r.sigma && r.sigma != 0u) ? 1u : 0u;
-        const int32_t qp = d < 0 ? -(int32_t)qe : (int32_t)qe;
-        return (int64_t)qp * L + b;                                // one 32 x 32 + 64 multiply-add
+        return d < 0 ? -(int32_t)qe : (int32_t)qe;
     }
 #if defined(__CUDA_ARCH__)
     const uint64_t quo = r.sigma ? div_rare((uint64_t)ad * 1024u + half, r.sigma) : 0u;
 #else
     const uint64_t quo = r.sigma ? ((uint64_t)ad * 1024u + half) / r.sigma : 0u;
 #endif
-    return (d < 0 ? -(int64_t)quo : (int64_t)quo) * (int64_t)L + (int64_t)b;
+    return d < 0 ? -(int64_t)quo : (int64_t)quo;
 }
 
-QL_HD int64_t ln_quotient_fast(int32_t q, const LnRow &r) { return ln_scaled_fast(q, r, 1, 0); }
+QL_HD int64_t ln_quotient_fast(int32_t q, const LnRow &r)
+{
+    bool fast;
+    return ln_quotient_core(q, r, fast);
+}
 
 QL_HD int32_t sat32_halves(int64_t v)              // saturate through the two 32-bit halves
 {
@@ -252,9 +315,30 @@ QL_HD int32_t sat32_halves(int64_t v)              // saturate through the two 3
     return hi == (lo >> 31) ? lo : (int32_t)(0x7fffffff ^ (hi >> 31));
 }
 
+QL_HD int32_t add_sat_s32(int32_t a, int32_t b)
+{
+#if defined(__CUDA_ARCH__)
+    int32_t d;
+    asm("add.sat.s32 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+#else
+    return sat32((int64_t)a + b);
+#endif
+}
+
+// sat32(q' L + b): in 32 bits on the fast path (|q'| <= 2^16 and -2^15 <= L < 2^15: the product is exact, the sum
+// saturates), in 64 bits otherwise
+QL_HD int32_t ln_scaled_sat32(int32_t q, const LnRow &r, int32_t L, int32_t b)
+{
+    bool fast;
+    const int64_t qp = ln_quotient_core(q, r, fast);
+    if (fast) return add_sat_s32((int32_t)qp * L, b);
+    return sat32_halves(qp * (int64_t)L + (int64_t)b);
+}
+
 QL_HD int32_t ln_apply_fast(int32_t q, const LnRow &r, int32_t L, int32_t b, Scale eff_ln, const FastScale &f_ln)
 {
-    const int32_t v32 = sat32_halves(ln_scaled_fast(q, r, L, b));
+    const int32_t v32 = ln_scaled_sat32(q, r, L, b);
     return sat16(eff_ln.shift <= 0 ? fast_rescale(v32, f_ln) : mbqm_cold(v32, eff_ln));
 }
 

@@ -95,6 +95,7 @@ struct RecParams {
     int gate_slot[4];             // canonical gate -> slot, -1 if absent
     unsigned long long spin_limit_ns;   // bound of one grid-barrier wait
     unsigned barrier_extra;             // 0; a test sets it to make the barrier wait for an arrival that never comes
+    DivMagic div_c;               // division by C (layer-norm statistics) as a multiplication
     const uint8_t *tab;           // memoised sigmoid / tanh tables of this layer (act_table.cuh), copied into the idle ring
     ActTabLayout tab_lay;         // before every elementwise phase; used by the instantiations with TAB only
     unsigned long long *phase_ns; // null, or 6 accumulators: work and barrier wait of phases A, B, C (CTA 0)
@@ -379,6 +380,28 @@ __device__ __forceinline__ void load_pair_i16(const int16_t *ptr, int32_t (&v)[2
         v[0][3] = 0; v[1][3] = 0;
     }
 }
+// The same pair from global data written by other blocks this step, as loaded (so that several loads can be in flight
+// before the first is unpacked), and its unpacking.
+template <int G>
+__device__ __forceinline__ uint4 load_pair_raw(const int16_t *ptr)
+{
+    if (G == 4) return __ldcg(reinterpret_cast<const uint4 *>(ptr));
+    const uint32_t *w = reinterpret_cast<const uint32_t *>(ptr);
+    return make_uint4(__ldcg(w), __ldcg(w + 1), __ldcg(w + 2), 0u);
+}
+template <int G>
+__device__ __forceinline__ void unpack_pair(const uint4 &q, int32_t (&v)[2][4])
+{
+    if (G == 4) {
+        v[0][0] = lo16(q.x); v[0][1] = hi16(q.x); v[0][2] = lo16(q.y); v[0][3] = hi16(q.y);
+        v[1][0] = lo16(q.z); v[1][1] = hi16(q.z); v[1][2] = lo16(q.w); v[1][3] = hi16(q.w);
+    } else {
+        v[0][0] = lo16(q.x); v[0][1] = hi16(q.x); v[0][2] = lo16(q.y);
+        v[1][0] = hi16(q.y); v[1][1] = lo16(q.z); v[1][2] = hi16(q.z);
+        v[0][3] = 0; v[1][3] = 0;
+    }
+}
+
 template <int G>
 __device__ __forceinline__ void load_pair_i32(const int32_t *ptr, int32_t (&v)[2][4])      // read-only global data
 {
@@ -488,15 +511,15 @@ __device__ __forceinline__ void warp_reduce_stats(RecCtl *ctl, const long long (
 
 // Block-wide reduction (all warps contribute to one row) into ctl->ln_rows[slot][*].
 template <int G>
-__device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, const long long (&sum)[4], const long long (&sq)[4], int n,
-                                                   int slot)
+__device__ __forceinline__ void block_reduce_stats(RecCtl *ctl, const long long (&sum)[4], const long long (&sq)[4],
+                                                   const DivMagic &div_n, int slot)
 {
     warp_reduce_stats<G>(ctl, sum, sq);
     ptx::cta_sync();
     if (threadIdx.x < G) {
         long long a = 0, b = 0;
         for (int w = 0; w < RTHREADS / 32; ++w) { a += ctl->red_sum[w][threadIdx.x]; b += ctl->red_sq[w][threadIdx.x]; }
-        ctl->ln_rows[slot][threadIdx.x] = make_ln_row(ln_stats(a, b, n));
+        ctl->ln_rows[slot][threadIdx.x] = make_ln_row(ln_stats_fast(a, b, div_n));
     }
     ptx::cta_sync();
 }
@@ -584,27 +607,25 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, co
             if (r < nrows) {
                 const int16_t *row = (const int16_t *)p.pre + (size_t)(rb + r) * p.N;
                 const int tig = (warp - r * wpr) * 32 + lane, gs = wpr * 32;
-                // four independent loads in flight per thread: the row comes from L2, and one load per trip would
-                // pay its latency C / (2 gs) times in a row
-                for (int u0 = 2 * tig; u0 < p.C; u0 += 8 * gs) {
-                    int32_t v[4][2][4];
+                // eight independent loads in flight per thread, kept packed until all are issued: the row comes from
+                // L2, and every trip of this loop pays that latency once
+                for (int u0 = 2 * tig; u0 < p.C; u0 += 16 * gs) {
+                    uint4 raw[8];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
+                    for (int k = 0; k < 8; ++k) {
                         const int u = u0 + 2 * gs * k;
-                        if (u < p.C) {
-                            load_pair_i16<G, 2>(row + (size_t)u * G, v[k]);
-                        } else {
-#pragma unroll
-                            for (int g = 0; g < 4; ++g) { v[k][0][g] = 0; v[k][1][g] = 0; }
-                        }
+                        raw[k] = u < p.C ? load_pair_raw<G>(row + (size_t)u * G) : make_uint4(0u, 0u, 0u, 0u);
                     }
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
+                    for (int k = 0; k < 8; ++k) {
+                        int32_t v[2][4];
+                        unpack_pair<G>(raw[k], v);
 #pragma unroll
                         for (int g = 0; g < G; ++g) {
-                            sum[g] += v[k][0][g] + v[k][1][g];
-                            sq[g] += (long long)(v[k][0][g] * v[k][0][g]) + (long long)(v[k][1][g] * v[k][1][g]);
+                            sum[g] += v[0][g] + v[1][g];
+                            sq[g] += (long long)(v[0][g] * v[0][g]) + (long long)(v[1][g] * v[1][g]);
                         }
+                    }
                 }
             }
             warp_reduce_stats<G>(ctl, sum, sq);
@@ -613,15 +634,21 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, co
                 const int rr = threadIdx.x >> 2, g = threadIdx.x & 3;
                 long long a = 0, b = 0;
                 for (int w = rr * wpr; w < (rr + 1) * wpr; ++w) { a += ctl->red_sum[w][g]; b += ctl->red_sq[w][g]; }
-                ctl->ln_rows[rr][g] = make_ln_row(ln_stats(a, b, p.C));
+                ctl->ln_rows[rr][g] = make_ln_row(ln_stats_fast(a, b, p.div_c));
             }
             ptx::cta_sync();
         }
         const int j0 = i0 > rb * p.C ? i0 : rb * p.C;
         const int j1 = i1 < (re + 1) * p.C ? i1 : (re + 1) * p.C;
-        for (int i = j0 + 2 * threadIdx.x; i < j1; i += 2 * RTHREADS) {
-            const int b = i / p.C, u = i - b * p.C;
+        // (row, cell) of a thread's tasks: one division for the first, then steps of 2 RTHREADS cells
+        constexpr int step = 2 * RTHREADS;
+        const int sb = step / p.C, su = step - sb * p.C;
+        int i = j0 + 2 * (int)threadIdx.x;
+        int b = i / p.C, u = i - b * p.C;
+        for (; i < j1; i += step) {
             flat_cell_pair<G, LN, PEEP, TAB>(p, at, ctl->ln_rows[b - rb], b, u, t, h_next);
+            b += sb; u += su;
+            if (u >= p.C) { u -= p.C; ++b; }
         }
         if (LN) ptx::cta_sync();      // the statistics slots are reused by the next batch of rows
     }
@@ -657,7 +684,7 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
                 sq[g] += (long long)(v * v);
             }
         }
-        block_reduce_stats<G>(ctl, sum, sq, p.C, 0);
+        block_reduce_stats<G>(ctl, sum, sq, p.div_c, 0);
         long long sum_o[4] = {0, 0, 0, 0}, sq_o[4] = {0, 0, 0, 0};
         for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
             const int nb = u * G;
@@ -678,7 +705,7 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
             sq_o[SO] += (long long)(v * v);
         }
         ptx::cta_sync();              // statistics of i, f, z are consumed; their slots are reused for o
-        block_reduce_stats<G>(ctl, sum_o, sq_o, p.C, 0);
+        block_reduce_stats<G>(ctl, sum_o, sq_o, p.div_c, 0);
         for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
             const int n = u * G + SO;
             const int32_t ao = ln_apply_fast(pre_s[n], lr[SO], __ldg(p.L + n), __ldg(p.bln + n), p.eff_ln[SO], p.f_ln[SO]);
@@ -1354,6 +1381,7 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     rp.T = T; rp.B = B; rp.MT = (B + 127) / 128; rp.Bpad = s.Bpad;
     rp.h_stride = (size_t)s.Bpad * f.kb_h * 128;
     rp.C = p.C; rp.O = p.O; rp.G = p.G; rp.N = p.N;
+    rp.div_c = make_div_magic((uint32_t)p.C);
     rp.flags = p.flags; rp.m_bits = p.m_bits; rp.zp_m = p.zp_m; rp.zp_h = p.zp_h;
     rp.cpc = f.cpc; rp.n_cta_a = f.n_cta_a; rp.nc_pad = f.nc_pad;
     rp.pn = f.pn; rp.npn = f.npn; rp.n_ptiles = rp.MT * f.npn;

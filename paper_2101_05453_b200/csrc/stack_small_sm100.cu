@@ -42,6 +42,7 @@ enum { CNT_A = 0, CNT_A2 = 1, CNT_M = 2, CNT_H = 3, CNT_PER_LAYER = 16 };      /
 
 struct SkLayer {
     int I, C, O, G, N;
+    DivMagic div_c;                // division by C (layer-norm statistics) as a multiplication
     uint32_t flags;
     int m_bits, zp_m, zp_h;
     const int8_t *W, *R, *Wproj;
@@ -390,7 +391,7 @@ __device__ __forceinline__ bool exchange_stats(const SkCall &k, const Role &r, c
             sum += __shfl_down_sync(0xffffffffu, sum, o);
             sq += __shfl_down_sync(0xffffffffu, sq, o);
         }
-        if (lane == 0) s.ln_s[task] = make_ln_row(ln_stats(sum, sq, L.C));
+        if (lane == 0) s.ln_s[task] = make_ln_row(ln_stats_fast(sum, sq, L.div_c));
     }
     __syncthreads();
     return true;
@@ -808,6 +809,7 @@ int stack_small_create(const std::vector<const LayerParams *> &lp, int max_T, in
         SkLayer L;
         memset(&L, 0, sizeof(L));
         L.I = p.I; L.C = p.C; L.O = p.O; L.G = p.G; L.N = p.N;
+        L.div_c = make_div_magic((uint32_t)p.C);
         L.flags = p.flags; L.m_bits = p.m_bits; L.zp_m = p.zp_m; L.zp_h = p.zp_h;
         L.W = p.W; L.R = p.R; L.Wproj = p.Wproj; L.bx = p.bx; L.bh = p.bh; L.bp = p.bp; L.bln = p.bln; L.P = p.P; L.L = p.L;
         for (int g = 0; g < 4; ++g) { L.eff_x[g] = p.eff_x[g]; L.eff_h[g] = p.eff_h[g]; L.eff_c[g] = p.eff_c[g]; L.eff_ln[g] = p.eff_ln[g]; }

@@ -23,6 +23,12 @@ def H():
     lib.qmh_mbqm.argtypes = [C.c_int32] * 3
     lib.qmh_isqrt.restype = C.c_uint64
     lib.qmh_isqrt.argtypes = [C.c_uint64]
+    lib.qmh_isqrt_from_f32.restype = C.c_uint64
+    lib.qmh_isqrt_from_f32.argtypes = [C.c_uint64]
+    lib.qmh_div_by_magic.restype = C.c_uint64
+    lib.qmh_div_by_magic.argtypes = [C.c_uint64, C.c_uint32]
+    lib.qmh_ln_stats.restype = None
+    lib.qmh_ln_stats.argtypes = [C.c_int64, C.c_int64, C.c_int, C.c_int, C.POINTER(C.c_int64)]
     return lib
 
 
@@ -202,3 +208,57 @@ def test_fast_layernorm_against_fp64_layer_norm(H):
     qf = q.astype(float)
     want = (qf - qf.mean()) / qf.std() * (L * s_L) + b * (s_L * 2.0 ** -10)
     assert np.abs(out / 4096.0 - want).max() <= 3e-3             # q' is on a 2^-10 grid: about 1e-3 per unit of L
+
+
+def test_division_by_fixed_divisor_and_fp32_seeded_root(H):
+    """The statistics' division by the row length as a multiplication (exact below 2^50 for lengths below 2^14) and
+    the integer square root from an fp32 estimate, against Python integers."""
+    rng = np.random.default_rng(41)
+    for n in [1, 2, 3, 7, 16, 48, 640, 1000, 1024, 2048, 4095, 4096, 8191, 16383]:
+        xs = [0, 1, n - 1, n, n + 1, 2 ** 50 - 1, 2 ** 50 - n, (2 ** 50 - 1) // n * n, (2 ** 50 - 1) // n * n - 1]
+        xs += [int(v) for v in rng.integers(0, 2 ** 50, 300)] + [int(v) * n for v in rng.integers(0, 2 ** 36, 100)]
+        xs += [int(v) * n - 1 for v in rng.integers(1, 2 ** 36, 100)]
+        for x in xs:
+            assert H.qmh_div_by_magic(x, n) == x // n, (x, n)
+    vs = [0, 1, 2, 3, 4, 2 ** 52 - 1, 2 ** 50, 2 ** 50 - 1] + [int(v) for v in rng.integers(0, 2 ** 52, 2000)]
+    for r in [1, 2, 4095, 4096, 2 ** 24 - 1, 2 ** 24, 2 ** 24 + 1, 2 ** 25 - 1, 2 ** 25, 2 ** 26 - 1, 33554431, 47453132]:
+        vs += [r * r - 1, r * r, r * r + 1, r * r + r, r * r + 2 * r]
+    for v in vs:
+        assert H.qmh_isqrt_from_f32(v) == math.isqrt(v), v
+
+
+def test_fast_statistics_equal_the_plain_ones_and_the_definition(H):
+    """ln_stats_fast (no 64-bit division, no fp64 root) against ln_stats and against the definition in Python integers
+    (Section 3.2.6): mean = round(2^10 sum / n), sigma = floor(sqrt(round(2^20 sumsq / n) - mean^2))."""
+    rng = np.random.default_rng(42)
+
+    def rdiv(a, b):
+        q = (abs(a) + b // 2) // b
+        return -q if a < 0 else q
+
+    out_f, out_p = (C.c_int64 * 2)(), (C.c_int64 * 2)()
+    cases = []
+    for n in [1, 2, 16, 48, 640, 1024, 2048, 3000, 8191]:
+        for kind in range(40):
+            if kind == 0:
+                q = np.full(n, 32767)
+            elif kind == 1:
+                q = np.full(n, -32768)
+            elif kind == 2:
+                q = np.where(np.arange(n) % 2 == 0, 32767, -32768)
+            elif kind == 3:
+                q = np.zeros(n, dtype=np.int64); q[0] = -32768
+            elif kind == 4:
+                q = np.full(n, 123)
+            else:
+                q = rng.integers(-32768, 32768, n) // int(rng.integers(1, 3000))
+            q = q.astype(np.int64)
+            cases.append((int(q.sum()), int((q * q).sum()), n))
+    for s, s2, n in cases:
+        H.qmh_ln_stats(s, s2, n, 1, out_f)
+        H.qmh_ln_stats(s, s2, n, 0, out_p)
+        mean = rdiv(s * 1024, n)
+        var = rdiv(s2 * 1048576, n) - mean * mean
+        sigma = math.isqrt(max(var, 0))
+        assert (out_f[0], out_f[1]) == (mean, sigma), (s, s2, n)
+        assert (out_p[0], out_p[1]) == (mean, sigma), (s, s2, n)
