@@ -494,18 +494,20 @@ __device__ __forceinline__ void phase_b_own(const RecParams &p, const OwnCells &
 // Phase B with layer norm: elementwise work on a contiguous range of the B x C cell grid, gate sums from L2.
 
 // Warp-level part of the statistics reduction: per-gate sum / sum of squares of this warp into shared memory.
+// The warp-wide adds are the hardware's 32-bit integer reduction (one instruction per value, where a shuffle tree is
+// ten per 64-bit value and the shuffle unit issues one per clock for the whole SM): a thread's sum of at most a row of
+// int16 values fits 32 bits as it is; its sum of squares (below 2^44) goes as its low 20 bits and the rest.
 template <int G>
 __device__ __forceinline__ void warp_reduce_stats(RecCtl *ctl, const long long (&sum)[4], const long long (&sq)[4])
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 #pragma unroll
     for (int g = 0; g < G; ++g) {
-        long long a = sum[g], b = sq[g];
-        for (int o = 16; o > 0; o >>= 1) {
-            a += __shfl_down_sync(0xffffffffu, a, o);
-            b += __shfl_down_sync(0xffffffffu, b, o);
-        }
-        if (lane == 0) { ctl->red_sum[warp][g] = a; ctl->red_sq[warp][g] = b; }
+        const int a = __reduce_add_sync(0xffffffffu, (int)sum[g]);
+        const unsigned long long q = (unsigned long long)sq[g];
+        const unsigned lo = __reduce_add_sync(0xffffffffu, (unsigned)(q & 0xfffffu));
+        const unsigned hi = __reduce_add_sync(0xffffffffu, (unsigned)(q >> 20));
+        if (lane == 0) { ctl->red_sum[warp][g] = a; ctl->red_sq[warp][g] = (long long)(((unsigned long long)hi << 20) + lo); }
     }
 }
 
