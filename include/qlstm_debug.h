@@ -18,7 +18,7 @@ extern "C" {
  * (one thread per output, one launch per phase), 2 = fast kernels (tensor-core projection,
  * persistent recurrent kernel); 2 fails with QLSTM_ERR_DIM at run time if a shape is unsupported.
  * recurrent_impl 2 always runs layer after layer (projection launch + persistent kernel per layer), where 0 takes the
- * whole-stack kernel at batch <= 4 (<= 8 for stacks of six or more layers); 3 = like 2 but with the tensor-core matmuls even at batch <= 4, where 2 uses dp4a
+ * whole-stack kernel at small batches (up to 4 rows; up to 8 for stacks of two or more layers; up to 16 for four or more); 3 = like 2 but with the tensor-core matmuls even at batch <= 4, where 2 uses dp4a
  * mat-vecs; 4 = like 2 but with the dp4a mat-vecs up to batch 16 (the crossover is a measured default, not a limit);
  * 5 = the whole-stack kernel or QLSTM_ERR_DIM (batch > 16, or a dimension that is not a multiple of 16), with its
  * schedule chosen from the call's length; 6 = the same with the wavefront schedule (one group of blocks per layer)

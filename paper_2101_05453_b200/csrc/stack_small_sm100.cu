@@ -134,6 +134,56 @@ __device__ __forceinline__ bool sk_wait(const SkCall &k, const unsigned *cnt, un
     return *abort_s == 0;
 }
 
+// Sums of NB values per lane over the gs lanes that share a row.  While a lane still holds more than one value a round
+// halves what it keeps - it sends the half it gives up and adds the half it receives - so the rounds cost
+// NB/2 + NB/4 + ... shuffles instead of NB each (the shuffle unit issues one per clock for the whole SM, and at 8 or 16
+// batch rows it was the busiest unit of the mat-vecs).  Afterwards acc[0 .. cnt) of a lane with `emitter` set hold the
+// sums of the batch rows b0 .. b0 + cnt - 1.
+template <int NB, int S>
+__device__ __forceinline__ void group_reduce_round(int32_t (&acc)[NB], int off, int lg, int &b0, bool &emitter)
+{
+    constexpr int CNT = (NB >> S) >= 1 ? (NB >> S) : 1;
+    if (off < 1) return;
+    if constexpr (CNT > 1) {
+        const bool up = (lg & off) != 0;
+#pragma unroll
+        for (int i = 0; i < CNT / 2; ++i) {
+            const int32_t keep = up ? acc[i + CNT / 2] : acc[i], give = up ? acc[i] : acc[i + CNT / 2];
+            acc[i] = keep + __shfl_xor_sync(0xffffffffu, give, off);
+        }
+        if (up) b0 += CNT / 2;
+    } else {
+        acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], off);
+        if (lg & off) emitter = false;               // every lane of the pair holds the sum: one of them emits it
+    }
+}
+template <int NB>
+__device__ __forceinline__ int group_reduce(int32_t (&acc)[NB], int gs, int lg, int &b0, bool &emitter)
+{
+    b0 = 0;
+    if constexpr (NB <= 2) {                         // too few values to share out: the plain butterfly, lane b emits row b
+        for (int off = gs >> 1; off > 0; off >>= 1) {
+#pragma unroll
+            for (int b = 0; b < NB; ++b) acc[b] += __shfl_xor_sync(0xffffffffu, acc[b], off);
+        }
+        if (NB == 2 && gs > 1) {
+            if (lg == 1) { acc[0] = acc[NB - 1]; b0 = 1; }
+            emitter = lg < 2;
+            return 1;
+        }
+        emitter = lg == 0;
+        return NB;
+    }
+    emitter = true;
+    group_reduce_round<NB, 0>(acc, gs >> 1, lg, b0, emitter);
+    group_reduce_round<NB, 1>(acc, gs >> 2, lg, b0, emitter);
+    group_reduce_round<NB, 2>(acc, gs >> 3, lg, b0, emitter);
+    group_reduce_round<NB, 3>(acc, gs >> 4, lg, b0, emitter);
+    group_reduce_round<NB, 4>(acc, gs >> 5, lg, b0, emitter);
+    const int cnt = NB / gs;                         // gs and NB are powers of two
+    return cnt >= 1 ? cnt : 1;
+}
+
 // rows [0, nrows) of a row-major int8 matrix (K bytes per row, K a multiple of 16) times NB vectors held in shared
 // memory as [NB][K]; emit(row, b, acc) runs once per (row, b < NB) on one lane.  gs lanes share a row (a power of two
 // that divides the number of 16-byte chunks of a row, so that every lane takes the same number of chunks CPL).
@@ -186,18 +236,15 @@ __device__ __forceinline__ void matvec_rows_t(const int8_t *rows, int nrows, int
                 }
             }
         }
-        for (int off = gs >> 1; off > 0; off >>= 1) {
-#pragma unroll
-            for (int q = 0; q < NR; ++q)
-#pragma unroll
-                for (int b = 0; b < NB; ++b) acc[q][b] += __shfl_xor_sync(0xffffffffu, acc[q][b], off);
-        }
 #pragma unroll
         for (int q = 0; q < NR; ++q) {
-            if (valid[q]) {
+            int b0;
+            bool emitter;
+            const int cnt = group_reduce<NB>(acc[q], gs, lg, b0, emitter);      // the lanes of a row share out the batch rows
+            if (valid[q] && emitter) {
 #pragma unroll
-                for (int b = 0; b < NB; ++b)
-                    if ((b & (gs - 1)) == lg) emit(r0 + q * stride + sub, b, acc[q][b]);   // the lanes of a row share out the batch rows
+                for (int i = 0; i < NB; ++i)
+                    if (i < cnt) emit(r0 + q * stride + sub, b0 + i, acc[q][i]);
             }
         }
     }
@@ -232,14 +279,13 @@ __device__ __forceinline__ void matvec_rows_any(const int8_t *rows, int nrows, i
                 }
             }
         }
-        for (int off = gs >> 1; off > 0; off >>= 1) {
+        int b0;
+        bool emitter;
+        const int cnt = group_reduce<NB>(acc, gs, lg, b0, emitter);
+        if (valid && emitter) {
 #pragma unroll
-            for (int b = 0; b < NB; ++b) acc[b] += __shfl_xor_sync(0xffffffffu, acc[b], off);
-        }
-        if (valid) {
-#pragma unroll
-            for (int b = 0; b < NB; ++b)
-                if ((b & (gs - 1)) == lg) emit(r, b, acc[b]);
+            for (int i = 0; i < NB; ++i)
+                if (i < cnt) emit(r, b0 + i, acc[i]);
         }
     }
 }
@@ -402,7 +448,7 @@ template <int NB>
 __device__ __forceinline__ bool finish_step(const SkCall &k, const Role &r, const SkSmem &s, int t, int *abort_s)
 {
     const SkLayer &L = *r.L;
-    const int B = k.B, G = L.G, C = L.C, O = L.O, npc = r.npc, cells = r.cells, n0 = r.n0, u0 = r.u0, cpc = L.cpc;
+    const int B = k.B, G = L.G, C = L.C, O = L.O, npc = r.npc, cells = r.cells, u0 = r.u0, cpc = L.cpc;
     const bool proj = (L.flags & F_PROJECTION) != 0, ln = (L.flags & F_LAYERNORM) != 0, peep = (L.flags & F_PEEPHOLE) != 0;
     const int SF = (G == 4) ? 1 : 0, SZ = SF + 1, SO = SF + 2;
     const unsigned n_grp = (unsigned)L.n_cta;
@@ -504,7 +550,7 @@ __device__ __forceinline__ bool finish_step(const SkCall &k, const Role &r, cons
             if (!exchange_stats(k, r, s, 1, 1u << SO, r.cnt + CNT_A2, (unsigned)(t + 1) * n_grp, abort_s)) return false;
             for (int i = threadIdx.x; i < B * cells; i += SK_THREADS) {
                 const int b = i / cells, ul = i - b * cells;
-                const int n = n0 + ul * G + SO;
+                const int n = ul * G + SO;                     // index into the block's own rows
                 const int32_t ao = ln_apply_fast(s.pre_s[b * npc + ul * G + SO], s.ln_s[b * 4 + SO], r.Lw[n], r.bln[n], L.eff_ln[SO],
                                                  make_fast_scale(L.eff_ln[SO]));
                 const int32_t mq = hidden_q_fast(sigmoid_q_fast(ao, 3), r.c_s[b * cpc + ul], L.m_bits, L.eff_m,
@@ -864,16 +910,19 @@ int stack_small_create(const std::vector<const LayerParams *> &lp, int max_T, in
 
 bool stack_small_supported(const StackSmall *s, int T, int B) { return s && s->ok && B >= 1 && B <= s->max_B && T >= 1 && T <= s->max_T; }
 
-// Where the whole-stack kernel is the faster path (measured): up to 4 batch rows always (27 against 144 us per time step
-// for eight 2048-cell layers at batch 1, 26 against 38 for five 1024-cell layers at batch 4); up to 8 rows for deep
-// stacks, whose layer-after-layer cost grows with the depth while the wavefront's does not (84 against 181 us at eight
-// layers; at five layers it is about even and at 16 rows the per-layer tensor-core kernels win).
+// Where the whole-stack kernel is the faster path (measured, us per time step of the whole stack, this kernel against
+// layer after layer): the wavefront's step costs one layer-step whatever the depth, the per-layer kernels' cost grows
+// with it.  Eight 2048-cell layers: 26 / 127 at batch 1, 59 / 157 at 8, 107 / 158 at 16; five 1024-cell layers: 17 / 32
+// at batch 4, 23 / 39 at 8, 33 / 39 at 16; two 256-cell layers: 6 / 10 at batch 2, 8.5 / 11 at 8; a single 2048-cell
+// layer (nothing to overlap): 27 / 28 at batch 4, 39 / 27 at 8, 54 / 27 at 16.
 bool stack_small_preferred(const StackSmall *s, int T, int B)
 {
     if (!stack_small_supported(s, T, B)) return false;
-    // a call of one or two steps is launch- and barrier-bound layer by layer (35 against 54 us for one step of ten
-    // 512-cell layers at 8 rows)
-    return B <= 4 || (B <= 8 && (s->n_layers >= 6 || T <= 2));
+    if (B <= 4) return true;
+    // a call of one or two steps is launch- and barrier-bound layer by layer (33 against 54 us for one step of two
+    // 256-cell layers at 8 rows)
+    if (B <= 8 && (s->n_layers >= 2 || T <= 2)) return true;
+    return s->n_layers >= 4;                             // 9 to 16 rows: measured for five and eight layers only
 }
 
 void stack_small_debug_timeout(StackSmall *s, unsigned missing_arrivals, unsigned long long limit_ns)

@@ -104,7 +104,7 @@ def test_small_batch_both_matmul_paths(B, kw):
     check_equal(run_gpu(w, impl=(FAST, 4)), want, f"dp4a B={B} {kw}")
 
 
-# ------------------------------------------------------------------ whole-stack kernel (batch <= 4)
+# ------------------------------------------------------------------ whole-stack kernel (batch <= 16)
 
 @pytest.mark.parametrize("B", [1, 2, 3, 4, 7, 16])
 @pytest.mark.parametrize("kw", VARIANTS, ids=lambda k: "+".join(sorted(k)) or "basic")
@@ -119,7 +119,10 @@ def test_stack_kernel_parity_variants(B, kw):
 
 
 @pytest.mark.parametrize("index,kw", [(1, {}), (2, {}), (3, dict(batch=2, T=12)), (4, dict(batch=3, T=12)),
-                                      (5, dict(batch=1, T=24)), (5, dict(batch=4, T=8)), (5, dict(batch=8, T=12))])
+                                      (5, dict(batch=1, T=24)), (5, dict(batch=4, T=8)), (5, dict(batch=8, T=12)),
+                                      # one cell per thread instead of four lanes per cell (batch x cells of a block above
+                                      # 128), with layer norm + peephole and its second statistics exchange
+                                      (3, dict(batch=16, T=6)), (3, dict(batch=8, T=3)), (4, dict(batch=16, T=6))])
 @pytest.mark.parametrize("impl", [STACK_WAVEFRONT, STACK_SEQUENTIAL])
 def test_stack_kernel_parity_configs(index, kw, impl):
     w = make_workload(index, **kw)
