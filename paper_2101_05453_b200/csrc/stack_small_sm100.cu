@@ -399,6 +399,18 @@ __device__ __forceinline__ void recurrent_term(const SkCall &k, const Role &r, c
     });
 }
 
+// Warp-wide sums of the layer-norm statistics with the 32-bit hardware reduction (one instruction, where a shuffle
+// tree of a 64-bit value is ten): a sum of at most a row of int16 values fits 32 bits on every lane and in total; a sum
+// of squares (non-negative, below 2^44 in total) goes as its low 20 bits and the rest.  Every lane gets the result.
+__device__ __forceinline__ long long warp_sum_small(long long v) { return (long long)__reduce_add_sync(0xffffffffu, (int)v); }
+__device__ __forceinline__ long long warp_sum_nonneg(long long v)
+{
+    const unsigned long long q = (unsigned long long)v;
+    const unsigned lo = __reduce_add_sync(0xffffffffu, (unsigned)(q & 0xfffffu));
+    const unsigned hi = __reduce_add_sync(0xffffffffu, (unsigned)(q >> 20));
+    return (long long)(((unsigned long long)hi << 20) + lo);
+}
+
 // layer-norm constants of the rows for the gate slots in `slots`: the block's per-row sums go to global memory, the
 // group meets, every block adds the group's shares (integer sums: the order does not matter)
 __device__ __forceinline__ bool exchange_stats(const SkCall &k, const Role &r, const SkSmem &s, int round, unsigned slots,
@@ -416,10 +428,8 @@ __device__ __forceinline__ bool exchange_stats(const SkCall &k, const Role &r, c
             sum += v;
             sq += (long long)(v * v);
         }
-        for (int o = 16; o > 0; o >>= 1) {
-            sum += __shfl_down_sync(0xffffffffu, sum, o);
-            sq += __shfl_down_sync(0xffffffffu, sq, o);
-        }
+        sum = warp_sum_small(sum);
+        sq = warp_sum_nonneg(sq);
         if (lane == 0) { mine[task * 2] = sum; mine[task * 2 + 1] = sq; }
     }
     sk_arrive(counter);
@@ -433,10 +443,8 @@ __device__ __forceinline__ bool exchange_stats(const SkCall &k, const Role &r, c
             sum += __ldcg(share);
             sq += __ldcg(share + 1);
         }
-        for (int o = 16; o > 0; o >>= 1) {
-            sum += __shfl_down_sync(0xffffffffu, sum, o);
-            sq += __shfl_down_sync(0xffffffffu, sq, o);
-        }
+        sum = warp_sum_small(sum);
+        sq = warp_sum_nonneg(sq);
         if (lane == 0) s.ln_s[task] = make_ln_row(ln_stats_fast(sum, sq, L.div_c));
     }
     __syncthreads();
@@ -922,7 +930,9 @@ bool stack_small_preferred(const StackSmall *s, int T, int B)
     // a call of one or two steps is launch- and barrier-bound layer by layer (33 against 54 us for one step of two
     // 256-cell layers at 8 rows)
     if (B <= 8 && (s->n_layers >= 2 || T <= 2)) return true;
-    return s->n_layers >= 4;                             // 9 to 16 rows: measured for five and eight layers only
+    // 9 to 16 rows: measured for five and eight layers only, and only where the wavefront has steps to overlap (one
+    // step per call at 16 rows: 448 against 375 us for the eight layers, 139 against 167 for the five)
+    return s->n_layers >= 4 && T >= s->n_layers;
 }
 
 void stack_small_debug_timeout(StackSmall *s, unsigned missing_arrivals, unsigned long long limit_ns)
