@@ -93,8 +93,10 @@ int qlstm_eval_activations(int cell_int_bits, int16_t *sigmoid_dev, int16_t *tan
  *     (0 shared with the gate's, 1 packed, 2 plain), format of the sigmoid (0 plain, 1 packed) }; bytes = 0 means that
  *     the tables do not fit or that the definition failed a check the formats rely on (the outputs are then untouched;
  *     such a layer keeps the arithmetic).  Synchronises the stream.
- *   qlstm_debug_activation_tables(q, 0) makes the kernel evaluate the definition instead (1 restores the default); it
- *     returns the number of layers that hold tables, or a negative qlstm_error.
+ *   qlstm_debug_activation_tables(q, 0) makes the kernel evaluate the definition instead (1 restores the default); 2
+ *     selects the kernel's general instantiation, the one a layer gets when one of its scales has a left shift
+ *     (shift > 0), which otherwise only such layers reach.  Returns the number of layers that hold tables, or a
+ *     negative qlstm_error.
  */
 int qlstm_eval_activation_tables(int cell_int_bits, int max_bytes, int16_t *sigmoid_dev, int16_t *tanh_gate_dev,
                                  int16_t *tanh_cell_dev, int *layout_out7, void *cuda_stream);

@@ -272,9 +272,10 @@ class QLSTM:
     def set_impl(self, projection: int = IMPL_AUTO, recurrent: int = IMPL_AUTO):
         _check(lib().qlstm_set_impl(self._h, projection, recurrent), "qlstm_set_impl")
 
-    def activation_tables(self, enable: bool = True) -> int:
-        """Memoised sigmoid / tanh in the persistent kernel on (default) or off; returns the layers that hold tables."""
-        n = lib().qlstm_debug_activation_tables(self._h, 1 if enable else 0)
+    def activation_tables(self, enable=True) -> int:
+        """Memoised sigmoid / tanh in the persistent kernel on (default) or off; 2: the kernel's general instantiation
+        (scales with a left shift allowed, no tables).  Returns the number of layers that hold tables."""
+        n = lib().qlstm_debug_activation_tables(self._h, int(enable))
         _check(min(n, 0), "qlstm_debug_activation_tables")
         return n
 

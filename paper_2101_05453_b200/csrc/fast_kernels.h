@@ -46,6 +46,7 @@ struct FastLayer {
     uint8_t *act_tab = nullptr;
     ActTabLayout act_lay = {0, 0, 0, 0, 0, 0, 0};
     bool dbg_no_tables = false;  // test hook: keep the arithmetic path although the tables exist
+    bool dbg_general_kernel = false;   // test hook: the instantiation that accepts scales with a left shift
     // test hook: make every grid barrier expect `dbg_barrier_extra` arrivals that never come, with a short wait limit
     unsigned dbg_barrier_extra = 0;
     unsigned long long dbg_spin_limit_ns = 0;

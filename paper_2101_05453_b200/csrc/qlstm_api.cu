@@ -497,10 +497,11 @@ int qlstm_debug_barrier_timeout(qlstm_t *q, int missing_arrivals, unsigned long 
 
 int qlstm_debug_activation_tables(qlstm_t *q, int enable)
 {
-    if (!q) return QLSTM_ERR_ARG;
+    if (!q || enable < 0 || enable > 2) return QLSTM_ERR_ARG;
     int n = 0;
     for (auto &L : q->layers) {
         L.fast.dbg_no_tables = enable == 0;
+        L.fast.dbg_general_kernel = enable == 2;
         if (L.fast.act_tab) ++n;
     }
     return n;

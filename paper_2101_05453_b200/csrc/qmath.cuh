@@ -342,6 +342,13 @@ QL_HD int32_t ln_apply_fast(int32_t q, const LnRow &r, int32_t L, int32_t b, Sca
     return sat16(eff_ln.shift <= 0 ? fast_rescale(v32, f_ln) : mbqm_cold(v32, eff_ln));
 }
 
+// The same for a scale known to shift right (eff_ln.shift <= 0): no rarely taken call in the caller's loop, which the
+// instruction scheduler does not move work across.
+QL_HD int32_t ln_apply_noshift(int32_t q, const LnRow &r, int32_t L, int32_t b, const FastScale &f_ln)
+{
+    return sat16(fast_rescale(ln_scaled_sat32(q, r, L, b), f_ln));
+}
+
 // ---- cell update and hidden state (Section 3.2.7) -------------------------------------------
 
 // x / 2^e for |x| <= 2^30 and 1 <= e <= 30, ties away from zero, in 32 bits

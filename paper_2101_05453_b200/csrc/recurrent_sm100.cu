@@ -170,13 +170,26 @@ __device__ __forceinline__ void grid_sync(const RecParams &p, unsigned &epoch, v
     ptx::cta_sync();
 }
 
+// FS: every scale of the layer shifts right (the usual case; decided per launch), so the rescale is the multiply-add
+// form alone.  Otherwise each use chooses, and the form with a left shift is an out-of-line call: a call in an unrolled
+// loop keeps the scheduler from interleaving the loop's independent chains (5 % of the step time at batch 256).
+template <bool FS>
 __device__ __forceinline__ int32_t rescale_sel(int32_t x, const Scale &s, const FastScale &f, int fast_ok)
 {
-    return fast_ok ? fast_rescale(x, f) : mbqm_cold(x, s);
+    if constexpr (FS) return fast_rescale(x, f);
+    else return fast_ok ? fast_rescale(x, f) : mbqm_cold(x, s);
 }
+template <bool FS>
 __device__ __forceinline__ int32_t rescale_any(int32_t x, const Scale &s, const FastScale &f)
 {
-    return s.shift <= 0 ? fast_rescale(x, f) : mbqm_cold(x, s);
+    if constexpr (FS) return fast_rescale(x, f);
+    else return s.shift <= 0 ? fast_rescale(x, f) : mbqm_cold(x, s);
+}
+template <bool FS>
+__device__ __forceinline__ int32_t ln_apply_sel(int32_t q, const LnRow &r, int32_t L, int32_t b, const Scale &eff, const FastScale &f)
+{
+    if constexpr (FS) return ln_apply_noshift(q, r, L, b, f);
+    else return ln_apply_fast(q, r, L, b, eff, f);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -226,7 +239,7 @@ struct OwnCells {
 // TM: accumulators come from tensor memory (taddr; warp-collective loads, so every lane runs the loop) or from
 // acc_row (int32, shared memory).  With three gates the groups are taken three at a time (24 columns = 8 cells), so
 // that the slot of every column is a compile-time constant; g_begin is then a multiple of 3.
-template <int G, bool LN, bool PEEP, bool TM>
+template <int G, bool LN, bool PEEP, bool TM, bool FS>
 __device__ __forceinline__ void gate_sums_row(const RecParams &p, const OwnCells &oc, uint32_t taddr, const int32_t *acc_row,
                                               int b, int n0, int g_begin, int g_end, const int16_t *c_row, bool row_valid)
 {
@@ -297,7 +310,7 @@ __device__ __forceinline__ void gate_sums_row(const RecParams &p, const OwnCells
                 const int gi = (G == 4) ? (j & 3) : col % 3;         // compile-time: gbase * 8 is a multiple of G
                 const int cl = col / G;                              // cell inside this batch of groups
                 const int32_t acc = add_sat((int32_t)r[NL == NB ? i : 0][j], bb[j]);
-                const int32_t H = sat16(rescale_sel(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
+                const int32_t H = sat16(rescale_sel<FS>(acc, p.eff_h[gi], p.f_h[gi], p.fast_rescale_ok));
                 const int32_t X = (j & 1) ? hi16(xw[j >> 1]) : lo16(xw[j >> 1]);
                 if (LN) {
                     o[j] = X + H;                                    // saturated when packed (no peephole), or int32 as it is
@@ -308,7 +321,7 @@ __device__ __forceinline__ void gate_sums_row(const RecParams &p, const OwnCells
                     int32_t v = X + H;
                     if (PEEP && gi != SZ) {
                         const int32_t P = (j & 1) ? hi16(pw[j >> 1]) : lo16(pw[j >> 1]);
-                        v += sat16(rescale_any(P * c_old[cl], p.eff_c[gi], p.f_c[gi]));
+                        v += sat16(rescale_any<FS>(P * c_old[cl], p.eff_c[gi], p.f_c[gi]));
                     }
                     o[j] = v;                                        // saturated when packed
                 }
@@ -327,6 +340,7 @@ __device__ __forceinline__ void gate_sums_row(const RecParams &p, const OwnCells
 
 // Phase C epilogue for one thread = one batch row and the columns [c_begin, c_end) of the projection tile, four at
 // a time: sum of the issuers' partial accumulators + folded bias (saturating) -> rescale -> + zp_h -> int8.
+template <bool FS>
 __device__ __forceinline__ void phase_c_row(const RecParams &p, uint32_t taddr, int n_acc, int b, int t, int p0, int c_begin,
                                             int c_end, int8_t *h_next, bool row_valid)
 {
@@ -348,7 +362,7 @@ __device__ __forceinline__ void phase_c_row(const RecParams &p, uint32_t taddr, 
             for (int a = 1; a < 4; ++a)
                 if (a < n_acc) sum += (int32_t)r[a][j];      // partial sums of the other issuers (exact in int32)
             const int32_t acc = add_sat(sum, bb[j]);
-            const int32_t hq = sat8(rescale_sel(acc, p.eff_proj, p.f_proj, p.fast_rescale_ok) + p.zp_h);
+            const int32_t hq = sat8(rescale_sel<FS>(acc, p.eff_proj, p.f_proj, p.fast_rescale_ok) + p.zp_h);
             w |= (uint32_t)(hq & 0xff) << (8 * j);
         }
         *reinterpret_cast<uint32_t *>(h_next + tile_off(b, p0 + col, p.kb_h)) = w;
@@ -435,19 +449,17 @@ __device__ __forceinline__ int32_t gate_tanh(const ActTabs &at, int32_t x)
     if constexpr (TAB) return tab_tanh_gate(at, x);
     else return tanh_q_fast(x, 3);
 }
-template <bool TAB>
+template <bool TAB, bool FS>
 __device__ __forceinline__ int32_t hidden_of(const RecParams &p, const ActTabs &at, int32_t o, int32_t c_new)
 {
-    if constexpr (TAB) {
-        const int32_t prod = o * tab_tanh_cell(at, c_new);
-        return sat8((p.eff_m.shift <= 0 ? fast_rescale(prod, p.f_m) : mbqm_cold(prod, p.eff_m)) + p.zp_m);
-    } else {
-        return hidden_q_fast(o, c_new, p.m_bits, p.eff_m, p.f_m, p.zp_m);
-    }
+    int32_t tc;
+    if constexpr (TAB) tc = tab_tanh_cell(at, c_new);
+    else tc = tanh_q_fast(c_new, p.m_bits);
+    return sat8(rescale_any<FS>(o * tc, p.eff_m, p.f_m) + p.zp_m);                      // Section 3.2.7
 }
 
 // One pair of the block's own cells (local pair k of row b), gate sums in shared memory.
-template <int G, bool PEEP, bool TAB>
+template <int G, bool PEEP, bool TAB, bool FS>
 __device__ __forceinline__ void own_cell_pair(const RecParams &p, const OwnCells &oc, const ActTabs &at, int b, int k, int t,
                                               int8_t *h_next)
 {
@@ -470,9 +482,9 @@ __device__ __forceinline__ void own_cell_pair(const RecParams &p, const OwnCells
         int32_t ao = a[q][SO];
         if (PEEP) {
             const int32_t H = oc.ho_s[(size_t)b * p.cpc + ul + q], P = oc.P_s[nl + q * G + SO];
-            ao = sat16(ao + H + sat16(rescale_any(P * c_new[q], p.eff_c[SO], p.f_c[SO])));   // Eq. 5: o sees c^t
+            ao = sat16(ao + H + sat16(rescale_any<FS>(P * c_new[q], p.eff_c[SO], p.f_c[SO])));   // Eq. 5: o sees c^t
         }
-        m[q] = hidden_of<TAB>(p, at, gate_sigmoid<TAB>(at, ao), c_new[q]);
+        m[q] = hidden_of<TAB, FS>(p, at, gate_sigmoid<TAB>(at, ao), c_new[q]);
     }
     *reinterpret_cast<uint32_t *>(c_ptr) = pack16(c_new[0], c_new[1]);
     store_hidden_pair(p, b, u, t, m[0], m[1], h_next);
@@ -480,13 +492,13 @@ __device__ __forceinline__ void own_cell_pair(const RecParams &p, const OwnCells
 
 // All (row, cell pair) tasks of the block, consecutive threads on consecutive pairs of a row: the gate sums of a row's
 // pairs are contiguous in shared memory.
-template <int G, bool PEEP, bool TAB>
+template <int G, bool PEEP, bool TAB, bool FS>
 __device__ __forceinline__ void phase_b_own(const RecParams &p, const OwnCells &oc, const ActTabs &at, int t, int8_t *h_next)
 {
     const int pairs = oc.cells >> 1, total = p.B * pairs;
     for (int i = threadIdx.x; i < total; i += RTHREADS) {
         const int b = i / pairs, k = i - b * pairs;
-        own_cell_pair<G, PEEP, TAB>(p, oc, at, b, k, t, h_next);
+        own_cell_pair<G, PEEP, TAB, FS>(p, oc, at, b, k, t, h_next);
     }
 }
 
@@ -536,7 +548,7 @@ __device__ __forceinline__ void load_pair_i32_cg(const int32_t *ptr, int32_t (&v
 }
 
 // Two adjacent cells (u even) of row b, every step after the gate sums (layer norm without peephole).
-template <int G, bool LN, bool PEEP, bool TAB>
+template <int G, bool LN, bool PEEP, bool TAB, bool FS>
 __device__ __forceinline__ void flat_cell_pair(const RecParams &p, const ActTabs &at, const LnRow *lr, int b, int u, int t,
                                                int8_t *h_next)
 {
@@ -556,7 +568,7 @@ __device__ __forceinline__ void flat_cell_pair(const RecParams &p, const ActTabs
             for (int g = 0; g < G; ++g) {
                 if (g == SO) continue;
                 int32_t v = a[k][g];
-                if (g != SZ) v += sat16(rescale_any(P[k][g] * c_old[k], p.eff_c[g], p.f_c[g]));
+                if (g != SZ) v += sat16(rescale_any<FS>(P[k][g] * c_old[k], p.eff_c[g], p.f_c[g]));
                 a[k][g] = sat16(v);
             }
     } else {
@@ -568,7 +580,7 @@ __device__ __forceinline__ void flat_cell_pair(const RecParams &p, const ActTabs
 #pragma unroll
             for (int k = 0; k < 2; ++k)
 #pragma unroll
-                for (int g = 0; g < G; ++g) a[k][g] = ln_apply_fast(a[k][g], lr[g], L[k][g], bl[k][g], p.eff_ln[g], p.f_ln[g]);
+                for (int g = 0; g < G; ++g) a[k][g] = ln_apply_sel<FS>(a[k][g], lr[g], L[k][g], bl[k][g], p.eff_ln[g], p.f_ln[g]);
         }
     }
     int32_t c_new[2], m[2];
@@ -580,15 +592,15 @@ __device__ __forceinline__ void flat_cell_pair(const RecParams &p, const ActTabs
         else { i = 32768 - f; if (i > 32767) i = 32767; }          // coupled input gate, Section 3.2.9
         c_new[k] = cell_update_fast(i, z, f, c_old[k], p.m_bits);
         int32_t ao = a[k][SO];
-        if (PEEP) ao = sat16(ao + sat16(rescale_any(P[k][SO] * c_new[k], p.eff_c[SO], p.f_c[SO])));
+        if (PEEP) ao = sat16(ao + sat16(rescale_any<FS>(P[k][SO] * c_new[k], p.eff_c[SO], p.f_c[SO])));
         const int32_t o = gate_sigmoid<TAB>(at, ao);
-        m[k] = hidden_of<TAB>(p, at, o, c_new[k]);
+        m[k] = hidden_of<TAB, FS>(p, at, o, c_new[k]);
     }
     *reinterpret_cast<uint32_t *>(c_ptr) = pack16(c_new[0], c_new[1]);
     store_hidden_pair(p, b, u, t, m[0], m[1], h_next);
 }
 
-template <int G, bool LN, bool PEEP, bool TAB>
+template <int G, bool LN, bool PEEP, bool TAB, bool FS>
 __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, const ActTabs &at, int t, int8_t *h_next)
 {
     const int total = p.B * p.C;
@@ -648,7 +660,7 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, co
         int i = j0 + 2 * (int)threadIdx.x;
         int b = i / p.C, u = i - b * p.C;
         for (; i < j1; i += step) {
-            flat_cell_pair<G, LN, PEEP, TAB>(p, at, ctl->ln_rows[b - rb], b, u, t, h_next);
+            flat_cell_pair<G, LN, PEEP, TAB, FS>(p, at, ctl->ln_rows[b - rb], b, u, t, h_next);
             b += sb; u += su;
             if (u >= p.C) { u -= p.C; ++b; }
         }
@@ -658,7 +670,7 @@ __device__ __forceinline__ void phase_b_flat(const RecParams &p, RecCtl *ctl, co
 
 // Layer norm with peephole: the gate sums need their peephole term before the statistics, and the output
 // gate's statistics need c^t of the whole row, so a row is processed by one CTA in three passes.
-template <int G, bool TAB>
+template <int G, bool TAB, bool FS>
 __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl, const ActTabs &at, int t, int8_t *h_next,
                                                 int16_t *row_s)
 {
@@ -679,7 +691,7 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
                 if (g == SO) continue;
                 const int n = u * G + g;
                 int32_t v = xh[n];
-                if (g != SZ) v += sat16(rescale_any((int32_t)__ldg(p.P + n) * c_old, p.eff_c[g], p.f_c[g]));
+                if (g != SZ) v += sat16(rescale_any<FS>((int32_t)__ldg(p.P + n) * c_old, p.eff_c[g], p.f_c[g]));
                 v = sat16(v);
                 pre_s[n] = (int16_t)v;
                 sum[g] += v;
@@ -693,7 +705,7 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
             int32_t a[4];
 #pragma unroll
             for (int g = 0; g < G; ++g)
-                if (g != SO) a[g] = ln_apply_fast(pre_s[nb + g], lr[g], __ldg(p.L + nb + g), __ldg(p.bln + nb + g), p.eff_ln[g], p.f_ln[g]);
+                if (g != SO) a[g] = ln_apply_sel<FS>(pre_s[nb + g], lr[g], __ldg(p.L + nb + g), __ldg(p.bln + nb + g), p.eff_ln[g], p.f_ln[g]);
             const int32_t f = gate_sigmoid<TAB>(at, a[SF]), z = gate_tanh<TAB>(at, a[SZ]);
             int32_t i;
             if (G == 4) i = gate_sigmoid<TAB>(at, a[SI]);
@@ -701,7 +713,7 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
             const int32_t c_new = cell_update_fast(i, z, f, c_row[u], p.m_bits);
             c_row[u] = (int16_t)c_new;
             cnew_s[u] = (int16_t)c_new;
-            const int32_t v = sat16(xh[nb + SO] + sat16(rescale_any((int32_t)__ldg(p.P + nb + SO) * c_new, p.eff_c[SO], p.f_c[SO])));
+            const int32_t v = sat16(xh[nb + SO] + sat16(rescale_any<FS>((int32_t)__ldg(p.P + nb + SO) * c_new, p.eff_c[SO], p.f_c[SO])));
             pre_s[nb + SO] = (int16_t)v;
             sum_o[SO] += v;
             sq_o[SO] += (long long)(v * v);
@@ -710,9 +722,9 @@ __device__ __forceinline__ void phase_b_ln_peep(const RecParams &p, RecCtl *ctl,
         block_reduce_stats<G>(ctl, sum_o, sq_o, p.div_c, 0);
         for (int u = threadIdx.x; u < p.C; u += RTHREADS) {
             const int n = u * G + SO;
-            const int32_t ao = ln_apply_fast(pre_s[n], lr[SO], __ldg(p.L + n), __ldg(p.bln + n), p.eff_ln[SO], p.f_ln[SO]);
+            const int32_t ao = ln_apply_sel<FS>(pre_s[n], lr[SO], __ldg(p.L + n), __ldg(p.bln + n), p.eff_ln[SO], p.f_ln[SO]);
             const int32_t o = gate_sigmoid<TAB>(at, ao);
-            const int32_t m = hidden_of<TAB>(p, at, o, cnew_s[u]);
+            const int32_t m = hidden_of<TAB, FS>(p, at, o, cnew_s[u]);
             if (p.flags & F_PROJECTION) {
                 p.mbuf[operand_off(p, b, u, p.C, p.kb_c)] = (int8_t)m;
             } else {
@@ -785,7 +797,7 @@ __device__ __forceinline__ void phase_c_small(const RecParams &p, int t, int p_l
         if (lane < p.B) {
             const int b = lane, o = p_lo + r;
             const int32_t acc = add_sat(mine, __ldg(p.bp + o));
-            const int32_t hq = sat8(rescale_sel(acc, p.eff_proj, p.f_proj, p.fast_rescale_ok) + p.zp_h);
+            const int32_t hq = sat8(rescale_sel<false>(acc, p.eff_proj, p.f_proj, p.fast_rescale_ok) + p.zp_h);
             h_next[(size_t)b * p.O + o] = (int8_t)hq;
             p.y[((size_t)t * p.B + b) * p.O + o] = (int8_t)hq;
         }
@@ -888,7 +900,8 @@ __device__ __noinline__ void drain_box_requests(uint64_t *x_full)
 
 // One instantiation per variant (gates, layer norm, peephole): each keeps only its own epilogue and elementwise code,
 // which is what lets the register allocator fit them without spilling.
-template <int G, bool LN, bool PEEP, bool TAB>
+// MODE: 0 any scales, nonlinearities evaluated; 1 every scale shifts right (FS); 2 FS and the nonlinearities memoised (TAB)
+template <int G, bool LN, bool PEEP, int MODE>
 __global__ void __launch_bounds__(RTHREADS, 1)
 k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_constant__ CUtensorMap map_Wp,
                   const __grid_constant__ CUtensorMap map_X, const __grid_constant__ CUtensorMap map_pre, RecParams p)
@@ -897,6 +910,7 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const bool proj = (p.flags & F_PROJECTION) != 0;
     constexpr bool ln = LN, peep = PEEP;
+    constexpr bool TAB = MODE == 2, FS = MODE >= 1;
     // layout: [ring stages][R slice][Wproj slice][X box][H_o (peephole) | row buffer (layer norm + peephole)]
     //         [per-column constants][control]
     uint8_t *ring = smem;
@@ -1051,7 +1065,7 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
                 if (okx)
                     for (int i = threadIdx.x; i < p.B * units; i += RTHREADS) {
                         const int b = i / units, gu = i - b * units;
-                        gate_sums_row<G, LN, PEEP, false>(p, oc, 0u, acc_s + (size_t)b * p.nc_pad, b, n0, gu * gstep, (gu + 1) * gstep,
+                        gate_sums_row<G, LN, PEEP, false, FS>(p, oc, 0u, acc_s + (size_t)b * p.nc_pad, b, n0, gu * gstep, (gu + 1) * gstep,
                                                           p.c + (size_t)b * p.C + oc.u0, true);
                     }
                 if (ln) ptx::fence_proxy_async();
@@ -1096,7 +1110,7 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
                     ptx::tc_fence_after();
                     const uint32_t ta = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(mi * p.nc_pad);
                     const bool valid = b < p.B;
-                    gate_sums_row<G, LN, PEEP, true>(p, oc, ta, nullptr, b, n0, g_begin, g_end,
+                    gate_sums_row<G, LN, PEEP, true, FS>(p, oc, ta, nullptr, b, n0, g_begin, g_end,
                                                      p.c + (size_t)(valid ? b : 0) * p.C + oc.u0, valid);
                     ptx::tc_fence_before();
                     if (ln) ptx::fence_proxy_async();                      // the box leaves through the async proxy
@@ -1125,12 +1139,12 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
             if (*abort_flag) break;
             // (a wait that runs out sets the abort flag: the next barrier ends the time loop)
             if (TAB && !wait_or_abort(&ctl->tab_full, par, abort_flag)) {}
-            else if (peep) phase_b_ln_peep<G, TAB>(p, ctl, at, t, h_next, row_s);
-            else phase_b_flat<G, true, false, TAB>(p, ctl, at, t, h_next);
+            else if (peep) phase_b_ln_peep<G, TAB, FS>(p, ctl, at, t, h_next, row_s);
+            else phase_b_flat<G, true, false, TAB, FS>(p, ctl, at, t, h_next);
             ptx::cta_sync();
         } else {
             // same block, same cells, straight from shared memory
-            if (!TAB || !has_cells || wait_or_abort(&ctl->tab_full, par, abort_flag)) phase_b_own<G, PEEP, TAB>(p, oc, at, t, h_next);
+            if (!TAB || !has_cells || wait_or_abort(&ctl->tab_full, par, abort_flag)) phase_b_own<G, PEEP, TAB, FS>(p, oc, at, t, h_next);
             ptx::fence_proxy_async();                        // X box and ring scratch go back to the async proxy
             ptx::cta_sync();
             if (has_cells && threadIdx.x == 0 && t + 1 < p.T && !*abort_flag) fetch_x(t + 1);
@@ -1178,7 +1192,7 @@ k_recurrent_sm100(const __grid_constant__ CUtensorMap map_R, const __grid_consta
                         if (__all_sync(0xffffffffu, wait_or_abort(&ctl->acc_full[2], par, abort_flag))) {
                             ptx::tc_fence_after();
                             const int b = tile_mi * 128 + quarter * 32 + lane;
-                            phase_c_row(p, tmem_base + ((uint32_t)(quarter * 32) << 16) + acc_cols_a, n_issue_c, b, t, tile_p0, c_begin,
+                            phase_c_row<FS>(p, tmem_base + ((uint32_t)(quarter * 32) << 16) + acc_cols_a, n_issue_c, b, t, tile_p0, c_begin,
                                         c_end, h_next, b < p.B);
                             ptx::tc_fence_before();
                         }
@@ -1247,19 +1261,32 @@ size_t rec_smem_bytes(const LayerParams &p, int stages, int nc_pad, int pn, int 
 
 int round_up(int v, int m) { return (v + m - 1) / m * m; }
 
-// the instantiation for a layer's variant; tab: with the memoised nonlinearities
-template <bool TAB>
+// the instantiation for a layer's variant and mode (see the kernel)
+template <int MODE>
 const void *recurrent_kernel_of(const LayerParams &p)
 {
     const bool ln = (p.flags & F_LAYERNORM) != 0, peep = (p.flags & F_PEEPHOLE) != 0;
     if (p.G == 4) {
-        if (ln) return peep ? (const void *)k_recurrent_sm100<4, true, true, TAB> : (const void *)k_recurrent_sm100<4, true, false, TAB>;
-        return peep ? (const void *)k_recurrent_sm100<4, false, true, TAB> : (const void *)k_recurrent_sm100<4, false, false, TAB>;
+        if (ln) return peep ? (const void *)k_recurrent_sm100<4, true, true, MODE> : (const void *)k_recurrent_sm100<4, true, false, MODE>;
+        return peep ? (const void *)k_recurrent_sm100<4, false, true, MODE> : (const void *)k_recurrent_sm100<4, false, false, MODE>;
     }
-    if (ln) return peep ? (const void *)k_recurrent_sm100<3, true, true, TAB> : (const void *)k_recurrent_sm100<3, true, false, TAB>;
-    return peep ? (const void *)k_recurrent_sm100<3, false, true, TAB> : (const void *)k_recurrent_sm100<3, false, false, TAB>;
+    if (ln) return peep ? (const void *)k_recurrent_sm100<3, true, true, MODE> : (const void *)k_recurrent_sm100<3, true, false, MODE>;
+    return peep ? (const void *)k_recurrent_sm100<3, false, true, MODE> : (const void *)k_recurrent_sm100<3, false, false, MODE>;
 }
-const void *recurrent_kernel(const LayerParams &p, bool tab) { return tab ? recurrent_kernel_of<true>(p) : recurrent_kernel_of<false>(p); }
+const void *recurrent_kernel(const LayerParams &p, int mode)
+{
+    return mode == 2 ? recurrent_kernel_of<2>(p) : (mode == 1 ? recurrent_kernel_of<1>(p) : recurrent_kernel_of<0>(p));
+}
+
+// every scale the recurrent kernel applies for this layer shifts right (shift <= 0)
+bool scales_shift_right(const LayerParams &p)
+{
+    const bool proj = (p.flags & F_PROJECTION) != 0, peep = (p.flags & F_PEEPHOLE) != 0, ln = (p.flags & F_LAYERNORM) != 0;
+    bool ok = p.eff_m.shift <= 0 && (!proj || p.eff_proj.shift <= 0);
+    for (int g = 0; g < p.G; ++g)
+        ok = ok && p.eff_h[g].shift <= 0 && (!peep || p.eff_c[g].shift <= 0) && (!ln || p.eff_ln[g].shift <= 0);
+    return ok;
+}
 
 // contig: n_own operand tiles of `per` chunks each, one owner per tile; else n_total chunks of one tile dealt round-robin
 RingPlan make_ring_plan(int stages, int n_own, bool contig, int per, int n_total)
@@ -1343,11 +1370,11 @@ int fast_recurrent_init(FastLayer &f, const LayerParams &p, const FastScratch &s
     } else {
         f.map_Wp = f.map_R;
     }
-    for (int tab = 0; tab < 2; ++tab) {
+    for (int mode = 0; mode < 3; ++mode) {
         int per_sm = 0;
-        if (cudaFuncSetAttribute(recurrent_kernel(p, tab != 0), cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(recurrent_kernel(p, mode), cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem) != cudaSuccess)
             return QLSTM_OK;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, recurrent_kernel(p, tab != 0), RTHREADS, f.smem) != cudaSuccess ||
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, recurrent_kernel(p, mode), RTHREADS, f.smem) != cudaSuccess ||
             per_sm < 1)
             return QLSTM_OK;
     }
@@ -1431,7 +1458,10 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
     rp.f_proj = make_fast_scale(p.eff_proj);
     rp.f_m = make_fast_scale(p.eff_m);
     rp.phase_ns = phase_ns;
-    const bool tab = f.act_tab != nullptr && !rp.small && !f.dbg_no_tables;
+    // tables only with right-shifting scales (a layer with a left shift keeps the general kernel)
+    const bool fs = scales_shift_right(p) && !f.dbg_general_kernel;
+    const bool tab = fs && f.act_tab != nullptr && !rp.small && !f.dbg_no_tables;
+    const int mode = tab ? 2 : (fs ? 1 : 0);
     rp.tab = tab ? f.act_tab : nullptr;
     rp.tab_lay = f.act_lay;
     rp.spin_limit_ns = f.dbg_spin_limit_ns ? f.dbg_spin_limit_ns : SPIN_LIMIT_NS;
@@ -1461,7 +1491,7 @@ int launch_recurrent_fast(const FastLayer &f, const LayerParams &p, const FastSc
         !make_tensor_map_i16(&map_pre, s.pre, (uint64_t)B, (uint64_t)p.N, (uint32_t)rp.x_rows, (uint32_t)rp.npc))
         return QLSTM_ERR_CUDA;
     void *args[] = {(void *)&f.map_R, (void *)&f.map_Wp, (void *)&map_X, (void *)&map_pre, (void *)&rp};
-    cudaError_t e = cudaLaunchCooperativeKernel(recurrent_kernel(p, tab), dim3(f.grid), dim3(RTHREADS), args, f.smem, st);
+    cudaError_t e = cudaLaunchCooperativeKernel(recurrent_kernel(p, mode), dim3(f.grid), dim3(RTHREADS), args, f.smem, st);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return e == cudaErrorCooperativeLaunchTooLarge ? QLSTM_ERR_LAUNCH : QLSTM_ERR_CUDA;

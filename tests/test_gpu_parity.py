@@ -517,7 +517,7 @@ def test_tables_and_arithmetic_agree(idx, B):
     q = qlstm.QLSTM(w.layers, T, B, device=0)
     q.set_impl(2, 2)
     res = []
-    for enable in (True, False):
+    for enable in (1, 0, 2):                  # tables; definition evaluated; general instantiation (any scale)
         n_tab = q.activation_tables(enable)
         assert n_tab == len(w.layers)                 # every layer of these configurations has room for its tables
         h0, c0 = w.initial_state()
@@ -529,8 +529,34 @@ def test_tables_and_arithmetic_agree(idx, B):
         res.append((y.cpu().numpy(), h.cpu().numpy(), c.cpu().numpy()))
     q.close()
     check_equal(res[0], res[1], f"config {idx} batch {B}: tables against arithmetic")
+    check_equal(res[0], res[2], f"config {idx} batch {B}: tables against the general instantiation")
     if B <= 64:
         check_equal(res[0], oracle(w), f"config {idx} batch {B}: tables against the oracle")
+
+
+@pytest.mark.parametrize("kw", VARIANTS, ids=lambda k: "+".join(sorted(k)) or "basic")
+@pytest.mark.parametrize("B", [2, 40])
+def test_scales_with_a_left_shift(B, kw):
+    """Effective scales of 1 and above (shift > 0, Section 3.2.4's rescale with its saturating left shift) in every
+    place the recurrent part rescales: the layers then take the general instantiation of the persistent kernel and the
+    general epilogue of the projection GEMM.  Everything saturates early; the result is still the oracle's, bit for bit."""
+    w = random_layer_stack(900 + B, 2, 32, 112, 48, T=5, B=B, **kw)
+    for q in w.layers:
+        for g in range(4):
+            if q.eff_h[g] is not None and q.eff_h[g][0]:
+                q.eff_h[g] = (q.eff_h[g][0], 1)
+            if g == 1 and q.eff_x[g] is not None and q.eff_x[g][0]:
+                q.eff_x[g] = (q.eff_x[g][0], 2)
+            if getattr(q, "eff_c", None) and q.eff_c[g] is not None and q.eff_c[g][0]:
+                q.eff_c[g] = (q.eff_c[g][0], 1)
+            if getattr(q, "eff_ln", None) and q.eff_ln[g] is not None and q.eff_ln[g][0] and g == 2:
+                q.eff_ln[g] = (q.eff_ln[g][0], 1)
+        q.eff_m = (q.eff_m[0], 1)
+        if q.eff_proj[0]:
+            q.eff_proj = (q.eff_proj[0], 1)
+    want = oracle(w)
+    check_equal(run_gpu(w, impl=(FAST, FAST)), want, f"left shifts, fast kernels, B={B} {kw}")
+    check_equal(run_gpu(w, impl=(SIMPLE, SIMPLE)), want, f"left shifts, simple kernels, B={B} {kw}")
 
 
 @pytest.mark.parametrize("seed", range(10))
