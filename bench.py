@@ -95,16 +95,16 @@ class ClockSampler:
 
 
 # DRAM traffic of the recurrent kernel from one ncu capture of full-size launches (three counters, one pass; its
-# summary is kept with the other profile summaries): dram__bytes_read.sum + dram__bytes_write.sum = 1267.6 + 52.7 MB
+# summary is kept with the other profile summaries): dram__bytes_read.sum + dram__bytes_write.sum = 1269.9 + 52.8 MB
 # per launch (one layer, 300 steps) of config 5 at batch 256, against 1309.9 MB algorithmic (X read once, y written
 # once).  Valid only for the kernel sources the counters were taken from and for that launch shape: otherwise null.
-NCU_RECURRENT = {"bytes": 1320.3e6, "steps": 300, "config": 5, "batch": 256, "source_sha": "48da413db92aeb40"}
+NCU_RECURRENT = {"bytes": 1322.7e6, "steps": 300, "config": 5, "batch": 256, "source_sha": "41be06a06a9b908e"}
 
 # DRAM traffic of the input-projection kernel from one ncu capture of a full-size launch (three counters, one pass):
 # dram__bytes_read.sum + dram__bytes_write.sum = 54.5 + 1204.1 MB at 76800 rows of config 5 (algorithmic: 49.2 MB of x,
 # 5.2 MB of W, 1258.3 MB of int16 output, part of which is still in L2 when the kernel ends).  Valid only for the
 # kernel sources the counters were taken from and for that launch shape: otherwise reported as null.
-NCU_PROJECTION = {"bytes": 1258.6e6, "rows": 76800, "config": 5, "source_sha": "028cc3e7e43c5a67"}
+NCU_PROJECTION = {"bytes": 1258.6e6, "rows": 76800, "config": 5, "source_sha": "b04867077a26bd59"}
 
 # The recurrent kernel is bound by plain integer arithmetic (the fixed-point epilogues), not by its matmuls or by
 # memory.  Peak: 148 SMs x 64 int32 lanes (4 schedulers x 16-lane integer pipe) x the SM clock; a microbenchmark of
