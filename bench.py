@@ -502,7 +502,7 @@ def main():
                 line["barrier_floor"] = {"error": str(exc)}
             # the other batch sizes of the configuration's sweep, then the other configurations
             per = {}
-            for Bs in (1, 8, 64):
+            for Bs in (1, 8, 16, 64):
                 per[f"config5_batch{Bs}"] = config_entry(5, Bs, with_oracle=False)
             line["batch_sweep"] = {k.split("batch")[1]: {"value": v["value"], "unit": UNIT, "ms_per_pass": v["ms_per_pass"],
                                                          "us_per_layer_step": 1e3 * v["ms_per_pass"] / (T * n_l)}
